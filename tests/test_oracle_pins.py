@@ -1,0 +1,362 @@
+"""Pins for the CPU oracle: each check ties an oracle function to something other than itself
+(hand-worked cases, closed forms, invariants, a library routine, brute force on tiny inputs)."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import focus_oracle as fo
+from paper_2602_02159_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _cases(name):
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                yield [p.split() for p in line.split("|")]
+
+
+# ------------------------------------------------------------------ select_queries (Eq. 4, Eq. 5)
+def test_indicator_hand_worked_cases():
+    n = 0
+    for conf, masked, par, focus, active in _cases("indicator_cases.txt"):
+        conf = np.array(conf, dtype=np.float32)
+        masked = np.array(masked, dtype=np.uint8)
+        blk_lo, blk_hi, k, w, clip_lo, clip_hi = map(int, par)
+        f, a = fo.select_queries(conf, masked, blk_lo, blk_hi, k, w, clip_lo, clip_hi)
+        assert f.tolist() == list(map(int, focus))
+        assert a.tolist() == list(map(int, active))
+        n += 1
+    assert n == 5
+
+
+def test_indicator_brute_force_subsets():
+    """On tiny inputs with distinct confidences the top-k set is the k-subset of the masked
+    candidates with the largest confidence sum (a definition that involves no sorting)."""
+    rng = np.random.default_rng(1)
+    for _ in range(30):
+        L = int(rng.integers(4, 10))
+        conf = rng.permutation(L).astype(np.float32) / L
+        masked = (rng.random(L) < 0.7).astype(np.uint8)
+        cand = [i for i in range(L) if masked[i]]
+        k = int(rng.integers(0, 4))
+        f, _ = fo.select_queries(conf, masked, 0, L, k, 0, 0, L)
+        kk = min(k, len(cand))
+        best = max(itertools.combinations(cand, kk), key=lambda c: sum(conf[list(c)])) if kk else ()
+        assert f.tolist() == sorted(best)
+
+
+def test_indicator_window_count_closed_form():
+    """Picks further apart than w and away from the clip edges: |I_active| = k * (2*floor(w/2) + 1)."""
+    L = 400
+    conf = np.zeros(L, dtype=np.float32)
+    masked = np.ones(L, dtype=np.uint8)
+    picks = [50, 90, 130, 170, 300]
+    conf[picks] = [0.9, 0.8, 0.7, 0.95, 0.6]
+    for w in (0, 1, 2, 7, 8, 9):
+        f, a = fo.select_queries(conf, masked, 0, L, 5, w, 0, L)
+        assert f.tolist() == picks
+        assert len(a) == 5 * (2 * (w // 2) + 1)
+    # paper's setting rho=4, n=2 -> k=8 and w=8 -> 9 positions per pick (Eq. 5 has both ends inclusive)
+    assert len(fo.select_queries(conf, masked, 0, L, 1, 8, 0, L)[1]) == 9
+
+
+def test_indicator_all_equal_takes_lowest_masked_indices_and_nan_last():
+    conf = np.full(12, 0.25, dtype=np.float32)
+    masked = np.array([0, 1, 1, 0, 1, 1, 1, 0, 1, 1, 1, 1], dtype=np.uint8)
+    f, _ = fo.select_queries(conf, masked, 0, 12, 3, 0, 0, 12)
+    assert f.tolist() == [1, 2, 4]
+    conf2 = conf.copy()
+    conf2[1] = np.nan
+    f, _ = fo.select_queries(conf2, masked, 0, 12, 3, 0, 0, 12)
+    assert f.tolist() == [2, 4, 5]
+
+
+# ------------------------------------------------------------------ sink scores (Eq. 6)
+def _small(seed=0, L=40, M=32, H=4, Hkv=2, d=8, n=5):
+    rng = np.random.default_rng(seed)
+    Q = rng.standard_normal((n, H, d))
+    K = rng.standard_normal((Hkv, L, d))
+    V = rng.standard_normal((Hkv, L, d))
+    return Q, K, V
+
+
+def test_sink_scores_sum_to_one_and_uniform_for_zero_queries():
+    Q, K, _ = _small()
+    S = fo.sink_scores(Q, K, 0.3)
+    assert abs(S.sum() - 1.0) < 1e-12
+    S0 = fo.sink_scores(np.zeros_like(Q), K, 0.3)
+    assert np.array_equal(S0, np.full(K.shape[1], 1.0 / K.shape[1]))
+    # equal scores: the tie rule returns the first n_sink candidates
+    assert fo.find_sinks(S0, 3, 2, 30).tolist() == [2, 3, 4]
+
+
+def test_sink_scores_single_row_is_library_softmax():
+    from scipy.special import softmax
+    rng = np.random.default_rng(3)
+    q = rng.standard_normal((1, 1, 6))
+    K = rng.standard_normal((1, 17, 6))
+    S = fo.sink_scores(q, K, 0.5)
+    ref = softmax(0.5 * (K[0] @ q[0, 0]))
+    assert np.allclose(S, ref, rtol=0, atol=1e-14)
+
+
+def test_sink_scores_use_the_kv_head_of_each_query_head():
+    """GQA mapping g(h) = h // (H/Hkv): with 4 query heads on 2 KV heads, zeroing KV head 1 must
+    make heads 2,3 uniform and leave heads 0,1 alone."""
+    Q, K, _ = _small(H=4, Hkv=2)
+    K2 = K.copy()
+    K2[1] = 0.0
+    S = fo.sink_scores(Q, K2, 1.0)
+    S_a = fo.sink_scores(Q[:, :2], K[:1], 1.0)           # heads 0,1 on KV head 0
+    L = K.shape[1]
+    assert np.allclose(S, 0.5 * S_a + 0.5 / L, atol=1e-14)
+
+
+def test_sink_scores_match_column_mean_of_exp_logit_minus_lse():
+    """Cross-check of two stages: S_j is the mean over rows and heads of exp(s_ij - lse_i) with the
+    lse reported by dense attention."""
+    Q, K, V = _small(seed=5)
+    scale = 0.37
+    _, lse = fo.dense_attn(Q, K, V, scale)
+    n, H, _ = Q.shape
+    acc = np.zeros(K.shape[1])
+    for h in range(H):
+        for i in range(n):
+            acc += np.exp(scale * (K[h // 2] @ Q[i, h]) - lse[h, i])
+    assert np.allclose(fo.sink_scores(Q, K, scale), acc / (n * H), atol=1e-14)
+
+
+@pytest.mark.parametrize("cfg", [0])
+def test_planted_sinks_recovered_small_config(cfg):
+    w = wl.config(cfg)
+    s = w.shape
+    t = wl.gen_qkv(s, w.seed, variant="fix", threads=1)
+    Q = wl.storage_to_f64(t["Q"], s.dtype)
+    K = wl.storage_to_f64(t["K"], s.dtype)
+    c_prev, _ = wl.gen_confidence(w.seed, s.N)
+    masked = wl.gen_masked(w)
+    _, active = fo.select_queries(wl.full_conf(s, c_prev), masked, w.blk_lo, w.blk_hi, w.k, w.w, s.M, s.L)
+    S = fo.sink_scores(Q[active - s.M], K, 1.0 / math.sqrt(s.d))
+    sinks = fo.find_sinks(S, w.n_sink, 0, s.M)
+    assert set(t["sink_pos"].tolist()) <= set(sinks.tolist())
+    # and they stand clear of the selection threshold (well outside the 1e-3 relative band)
+    tau = np.sort(S[:s.M])[::-1][w.n_sink - 1]
+    assert all(S[p] > 1.5 * tau for p in t["sink_pos"])
+
+
+def test_find_sinks_brute_force():
+    rng = np.random.default_rng(7)
+    for _ in range(20):
+        L = int(rng.integers(5, 12))
+        S = rng.integers(0, 4, size=L).astype(np.float64)      # many ties
+        lo, hi = 1, L - 1
+        n = int(rng.integers(0, hi - lo + 1))
+        got = fo.find_sinks(S, n, lo, hi).tolist()
+        # brute force: repeatedly take the max (first occurrence = lowest index)
+        pool = list(range(lo, hi))
+        exp = []
+        for _ in range(n):
+            j = max(pool, key=lambda t: (S[t], -t))
+            exp.append(j)
+            pool.remove(j)
+        assert got == sorted(exp)
+
+
+# ------------------------------------------------------------------ pooled keys, block relevance (Eq. 7)
+def test_pool_keys_constant_blocks_and_short_tail():
+    Hkv, M, B, d = 2, 11, 4, 3
+    K = np.zeros((Hkv, 16, d))
+    for b in range(3):
+        K[:, b * B:(b + 1) * B, :] = b + 1.0
+    K[:, 11:, :] = 1e9                                    # response keys must not leak into the last block
+    Kb = fo.pool_keys(K, M, B)
+    assert Kb.shape == (Hkv, 3, d)
+    assert np.array_equal(Kb[:, 0], np.full((Hkv, d), 1.0))
+    assert np.array_equal(Kb[:, 2], np.full((Hkv, d), 3.0))   # tail block has 3 tokens, all equal 3
+    K[0, 8, :] = 6.0                                      # tail mean over 3 real tokens: (6+3+3)/3
+    assert np.allclose(fo.pool_keys(K, M, B)[0, 2], 4.0)
+
+
+def test_block_scores_linearity_and_modes():
+    rng = np.random.default_rng(11)
+    nf, H, Hkv, d, M, B = 3, 4, 2, 5, 24, 8
+    Qf = rng.standard_normal((nf, H, d))
+    K = rng.standard_normal((Hkv, 30, d))
+    Kb = fo.pool_keys(K, M, B)
+    Rg = fo.score_blocks(Qf, Kb, fo.PER_KV_GROUP)
+    Ra = fo.score_blocks(Qf, Kb, fo.ALL_HEADS)
+    assert Rg.shape == (Hkv, 3) and Ra.shape == (1, 3)
+    # R_b = mean over tokens of the block of (mean query) . k_j   -- no pooling needed
+    for g in range(Hkv):
+        qbar = Qf[:, 2 * g:2 * g + 2, :].mean(axis=(0, 1))
+        for b in range(3):
+            direct = np.mean([qbar @ K[g, j] for j in range(b * B, (b + 1) * B)])
+            assert abs(Rg[g, b] - direct) < 1e-12
+    # Eq. 7 as printed is the mean over all heads = mean of the equally sized groups
+    assert np.allclose(Ra[0], Rg.mean(axis=0), atol=1e-14)
+    # no 1/sqrt(d) and no softmax: doubling the queries doubles the scores
+    assert np.allclose(fo.score_blocks(2 * Qf, Kb, fo.ALL_HEADS), 2 * Ra, atol=1e-13)
+
+
+def test_block_aligned_with_queries_ranks_first():
+    rng = np.random.default_rng(13)
+    nf, H, d, M, B = 4, 2, 16, 64, 8
+    Qf = rng.standard_normal((nf, H, d)) + 1.0
+    K = 0.1 * rng.standard_normal((2, M, d))
+    for g in range(2):
+        K[g, 5 * B:6 * B] += 3.0 * Qf[:, g].mean(axis=0)
+    R = fo.score_blocks(Qf, fo.pool_keys(K, M, B), fo.PER_KV_GROUP)
+    blocks, _ = fo.select_blocks(R, 1, np.array([], dtype=np.int64), B)
+    assert [b.tolist() for b in blocks] == [[5], [5]]
+
+
+def test_select_blocks_brute_force_and_sink_keep():
+    rng = np.random.default_rng(17)
+    for _ in range(20):
+        nb = int(rng.integers(3, 9))
+        R = rng.integers(0, 3, size=(2, nb)).astype(np.float64)
+        C = int(rng.integers(0, nb + 1))
+        B = 4
+        sinks = np.sort(rng.choice(nb * B, size=3, replace=False))
+        blocks, keep = fo.select_blocks(R, C, sinks, B)
+        for g in range(2):
+            pool = list(range(nb))
+            exp = []
+            for _ in range(C):
+                j = max(pool, key=lambda t: (R[g, t], -t))
+                exp.append(j)
+                pool.remove(j)
+            assert blocks[g].tolist() == sorted(exp)
+            assert keep[g].tolist() == [0 if (s // B) in exp else 1 for s in sinks]
+        full, _ = fo.select_blocks(R, nb, sinks, B)
+        assert all(b.tolist() == list(range(nb)) for b in full)
+        bl, _ = fo.select_blocks(R, C, sinks, B, fo.SINK_BLOCKS)
+        for g in range(2):
+            assert set(bl[g].tolist()) == set(blocks[g].tolist()) | {int(s) // B for s in sinks}
+
+
+# ------------------------------------------------------------------ attention (Eq. 9)
+def test_attention_closed_form_cases():
+    n = 0
+    for q, keys, vals, out, z in _cases("attention_cases.txt"):
+        K = np.log(np.array(keys, dtype=np.float64)).reshape(1, -1, 1)
+        V = np.array(vals, dtype=np.float64).reshape(1, -1, 1)
+        Q = np.array(q, dtype=np.float64).reshape(1, 1, 1)
+        O, lse = fo.dense_attn(Q, K, V, 1.0)
+        assert abs(O[0, 0, 0] - float(out[0])) < 1e-12
+        assert abs(math.exp(lse[0, 0]) - float(z[0])) < 1e-12
+        n += 1
+    assert n == 3
+
+
+def test_dense_equals_library_sdpa():
+    torch = pytest.importorskip("torch")
+    Q, K, V = _small(seed=21, L=50, H=4, Hkv=2, d=8, n=6)
+    scale = 0.41
+    O, _ = fo.dense_attn(Q, K, V, scale)
+    q = torch.from_numpy(Q).permute(1, 0, 2)                                   # [H, n, d]
+    k = torch.from_numpy(K).repeat_interleave(2, dim=0)
+    v = torch.from_numpy(V).repeat_interleave(2, dim=0)
+    ref = torch.nn.functional.scaled_dot_product_attention(q, k, v, scale=scale).permute(1, 0, 2).numpy()
+    assert np.allclose(O, ref, rtol=0, atol=1e-13)
+
+
+def test_keep_ratio_one_is_dense_bit_for_bit():
+    Q, K, V = _small(seed=23, L=45, M=37, H=4, Hkv=2, d=8)
+    M, B = 37, 8                      # ragged last block (5 tokens)
+    nb = 5
+    blocks = [np.arange(nb), np.arange(nb)]
+    Os, ls = fo.sparse_attn(Q, K, V, M, B, blocks, np.array([3, 20]), 0.3)
+    Od, ld = fo.dense_attn(Q, K, V, 0.3)
+    assert np.array_equal(Os, Od) and np.array_equal(ls, ld)
+
+
+def test_softmax_rows_sum_to_one_and_constant_values():
+    Q, K, V = _small(seed=29)
+    M, B = 32, 8
+    blocks = [np.array([1, 3]), np.array([0])]
+    sinks = np.array([9, 17])         # 9 is inside block 1 for group 0, outside for group 1
+    O, lse = fo.sparse_attn(Q, K, np.ones_like(V), M, B, blocks, sinks, 0.5)
+    assert np.allclose(O, 1.0, atol=1e-14)
+    for h in range(4):
+        ks = fo.key_set(M, 40, B, blocks[h // 2], sinks)
+        for i in range(Q.shape[0]):
+            assert abs(np.exp(0.5 * (K[h // 2, ks] @ Q[i, h]) - lse[h, i]).sum() - 1.0) < 1e-12
+
+
+def test_zero_queries_give_plain_mean_of_the_retained_values():
+    """Pins the exact key set: with Q = 0 every retained key has the same weight, so the output is the
+    plain mean of the retained V rows, each counted once (a sink inside a selected block must not be
+    counted twice; response tokens are always there; the short last block has only its real tokens)."""
+    _, K, V = _small(seed=31, L=45, M=37, H=2, Hkv=2, d=8)
+    Q = np.zeros((2, 2, 8))
+    M, B = 37, 8
+    blocks = [np.array([1, 4]), np.array([0])]
+    sinks = np.array([2, 10, 36])
+    O, lse = fo.sparse_attn(Q, K, V, M, B, blocks, sinks, 0.5)
+    exp_keys = [sorted(set(range(8, 16)) | set(range(32, 37)) | {2, 10, 36} | set(range(37, 45))),
+                sorted(set(range(0, 8)) | {2, 10, 36} | set(range(37, 45)))]
+    assert len(exp_keys[0]) == 8 + 5 + 1 + 8 and len(exp_keys[1]) == 8 + 2 + 8
+    for g in range(2):
+        assert np.allclose(O[0, g], V[g, exp_keys[g]].mean(axis=0), atol=1e-14)
+        assert abs(lse[g, 0] - math.log(len(exp_keys[g]))) < 1e-14
+
+
+def test_block_order_does_not_matter_and_heads_argument():
+    Q, K, V = _small(seed=37)
+    a, _ = fo.sparse_attn(Q, K, V, 32, 8, [np.array([0, 2, 3])] * 2, np.array([12]), 0.2)
+    b, _ = fo.sparse_attn(Q, K, V, 32, 8, [np.array([3, 0, 2])] * 2, np.array([12]), 0.2)
+    assert np.allclose(a, b, atol=1e-15)
+    c, _ = fo.sparse_attn(Q, K, V, 32, 8, [np.array([0, 2, 3])] * 2, np.array([12]), 0.2, heads=[2])
+    assert np.array_equal(c[:, 2], a[:, 2]) and not c[:, 0].any()
+    # a single shared list (ALL_HEADS mode) serves every head
+    d, _ = fo.sparse_attn(Q, K, V, 32, 8, [np.array([0, 2, 3])], np.array([12]), 0.2)
+    assert np.array_equal(d, a)
+
+
+def test_sparse_output_approaches_dense_when_dropped_keys_carry_no_mass():
+    """Eq. 9 restricted to a key set equals dense attention when the dropped keys have negligible
+    weight: push the dropped blocks' logits to -inf-like values."""
+    Q, K, V = _small(seed=41, L=40, M=32, H=2, Hkv=2, d=8, n=3)
+    Q = np.abs(Q)
+    K2 = K.copy()
+    K2[:, 8:16] = -50.0                       # block 1 gets hugely negative logits for positive queries
+    blocks = [np.array([0, 2, 3])] * 2
+    Os, _ = fo.sparse_attn(Q, K2, V, 32, 8, blocks, np.array([], dtype=np.int64), 1.0)
+    Od, _ = fo.dense_attn(Q, K2, V, 1.0)
+    assert np.allclose(Os, Od, atol=1e-12)
+
+
+# ------------------------------------------------------------------ generators (inputs only)
+def test_bf16_round_trip_and_rne():
+    x = np.array([1.0, 1.00390625, 1.01171875, -2.5, 3.140625], dtype=np.float32)   # 1+2^-8 ties to even
+    b = wl.f32_to_bf16_bits(x)
+    back = wl.bf16_bits_to_f32(b)
+    assert back[0] == 1.0 and back[1] == 1.0 and back[2] == np.float32(1.015625) and back[3] == -2.5
+    assert np.array_equal(wl.f32_to_bf16_bits(back), b)
+    torch = pytest.importorskip("torch")
+    r = np.random.default_rng(0).standard_normal(1000).astype(np.float32)
+    t = torch.from_numpy(r).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(wl.f32_to_bf16_bits(r), t)
+
+
+def test_generators_are_seeded_and_shaped():
+    w = wl.config(0)
+    a = wl.gen_qkv(w.shape, 0, threads=1)
+    b = wl.gen_qkv(w.shape, 0, threads=4)
+    assert all(np.array_equal(a[k], b[k]) for k in ("Q", "K", "V"))
+    assert a["Q"].shape == (128, 8, 64) and a["K"].shape == (8, 1024, 64)
+    assert not np.array_equal(a["K"], wl.gen_qkv(w.shape, 1, threads=1)["K"])
+    kn = np.linalg.norm(a["K"][:, a["sink_pos"], :], axis=2)
+    assert np.allclose(kn, wl.SINK_NORM, rtol=1e-5)
+    m = wl.gen_masked(w)
+    assert m[:896].sum() == 0 and m[896:].sum() == 64
+    for i in (1, 2, 3):
+        c = wl.config(i)
+        assert c.C == {1: 7, 2: 15, 3: 15}[i] and c.n_sink == c.shape.M // 100
