@@ -1,0 +1,181 @@
+/*
+ * libfocus -- the per-denoising-step sparse-attention path of Focus-dLLM on NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  One non-block-entry denoising step of one layer is
+ *     focus_select_queries  ->  [probe layer: focus_dense_attn (emits LSE) -> focus_find_sinks]
+ *     ->  focus_score_blocks  ->  focus_select_blocks  ->  focus_sparse_attn
+ *
+ * Conventions shared by every entry point
+ *   - Positions are 0-indexed: prompt [0, M), response / gen region [M, L).  Prompt block b is
+ *     [b*kv_block, min((b+1)*kv_block, M)); there are nb = ceil(M / kv_block) blocks.
+ *   - Query head h reads KV head g(h) = h / (n_q_heads / n_kv_heads).
+ *   - All data pointers are DEVICE pointers owned by the caller unless a comment says "host".
+ *     Q/K/V base pointers must be 16-byte aligned; the innermost (head_dim) dimension is contiguous;
+ *     token and head strides are in elements and must be multiples of 8 elements.
+ *   - Index outputs are int32, ascending, padded with -1.  Counts are written to device int32 so a
+ *     whole step can be enqueued without a host round trip.
+ *   - Every call validates its arguments on the host, enqueues its kernels on the caller's stream and
+ *     returns without synchronising.  Nothing is allocated after focus_create: scratch comes from the
+ *     context's workspace (FOCUS_ERR_WORKSPACE_TOO_SMALL if it does not fit).  Calls on one context
+ *     must be issued on one stream at a time (they share the workspace).
+ *   - Results are deterministic run to run (fixed reduction order, no floating-point atomics).
+ *   - A device-side anomaly (index out of range, a bounded wait that ran out) never traps: the kernel
+ *     skips the access, records a code in the context's device status word and returns; read it with
+ *     focus_poll_status.
+ *   - There is no CPU fallback: without a CUDA device every compute entry point fails.
+ */
+#ifndef FOCUS_H_
+#define FOCUS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct focus_ctx focus_ctx;          /* opaque: device, SM count, workspace, status word */
+typedef struct CUstream_st* focus_stream;    /* same type as cudaStream_t */
+
+typedef enum {
+  FOCUS_OK = 0,
+  FOCUS_ERR_INVALID_ARG = 1,
+  FOCUS_ERR_UNSUPPORTED = 2,
+  FOCUS_ERR_WORKSPACE_TOO_SMALL = 3,
+  FOCUS_ERR_CUDA = 4,
+  FOCUS_ERR_TIMEOUT = 5
+} focus_status;
+
+typedef enum { FOCUS_F32 = 0, FOCUS_BF16 = 1 } focus_dtype;
+
+/* How block scores are reduced over heads.  PER_KV_GROUP: one block set per KV head, scored by the
+ * mean over the query heads of that group (for MHA: per head).  ALL: one block set for the layer,
+ * scored by the mean over all heads (Eq. 7 as printed). */
+typedef enum { FOCUS_HEADS_PER_KV_GROUP = 0, FOCUS_HEADS_ALL = 1 } focus_head_reduce;
+
+/* How sink tokens join the key set.  TOKENS: as single tokens (Eq. 8 as printed).  BLOCKS: the prompt
+ * block around each sink token is added to the block list. */
+typedef enum { FOCUS_SINK_TOKENS = 0, FOCUS_SINK_BLOCKS = 1 } focus_sink_mode;
+
+typedef struct {
+  int32_t L, M;                    /* total positions, prompt length */
+  int32_t n_q_heads, n_kv_heads;   /* H, Hkv; H % Hkv == 0 */
+  int32_t head_dim;                /* 64 or 128 */
+  int32_t kv_block;                /* prompt block size B: 64 or 128 */
+  int32_t dtype;                   /* focus_dtype of Q, K, V and O */
+  float softmax_scale;             /* 0 => 1/sqrt(head_dim) */
+  int64_t q_stride_row, q_stride_head;    /* Q[(pos - q_base)*q_stride_row + h*q_stride_head + c] */
+  int64_t kv_stride_tok, kv_stride_head;  /* K[g*kv_stride_head + j*kv_stride_tok + c], same for V */
+} focus_shape;
+
+/* ---- context ------------------------------------------------------------------------------- */
+
+/* Creates a context on `device` and allocates its workspace (workspace_bytes == 0: 256 MiB) and a
+ * 4-byte status word.  The only entry point that allocates.  Errors: INVALID_ARG (null out pointer),
+ * CUDA (no such device / allocation failed). */
+focus_status focus_create(focus_ctx** out, int device, size_t workspace_bytes);
+focus_status focus_destroy(focus_ctx* ctx);
+
+/* Upper bound of the scratch any single call needs for this shape with at most n_q query rows,
+ * max_blocks blocks per group and n_sink sink tokens. */
+focus_status focus_workspace_bytes(const focus_shape* shape, int32_t n_q, int32_t max_blocks, int32_t n_sink,
+                                   size_t* out_bytes);
+
+/* Synchronises `stream`, copies the device status word to *device_status (0 = clean, else the
+ * focus_status code of the first anomaly) and clears it. */
+focus_status focus_poll_status(focus_ctx* ctx, focus_stream stream, int32_t* device_status);
+const char* focus_status_string(focus_status s);
+
+/* Selects the attention implementation for bf16 / head_dim 128 inputs: 0 = automatic (tensor-core
+ * kernel where supported), 1 = force the generic SIMT kernels.  Returns the previous value. */
+int32_t focus_set_force_simt(focus_ctx* ctx, int32_t force);
+
+/* ---- stage 1: past-confidence indicator (Eq. 4) and window expansion (Eq. 5) ---------------- */
+
+/* I_focus = the k positions i in [blk_lo, blk_hi) with masked[i] != 0 that have the highest
+ * conf_prev[i] (ties: lower index; NaN ranks last); n_focus = min(k, number of candidates).
+ * I_active = union over i in I_focus of [i - w/2, i + w/2] (integer division) clipped to
+ * [clip_lo, clip_hi).
+ *   conf_prev  float[L], masked uint8[L]
+ *   focus_idx  int32[k]; active_idx int32[k * (2*(w/2) + 1)]; n_focus, n_active int32[1]
+ * Requires 0 <= blk_lo <= blk_hi <= L, blk_hi - blk_lo <= 4096, 0 <= k <= 1024, w >= 0. */
+focus_status focus_select_queries(focus_ctx* ctx, const float* conf_prev, const uint8_t* masked, int32_t L,
+                                  int32_t blk_lo, int32_t blk_hi, int32_t k, int32_t w,
+                                  int32_t clip_lo, int32_t clip_hi,
+                                  int32_t* focus_idx, int32_t* n_focus,
+                                  int32_t* active_idx, int32_t* n_active, focus_stream stream);
+
+/* ---- stage 2: attention-sink identification (Eq. 6) ----------------------------------------- */
+
+/* S_j = mean over heads h and active rows i of softmax_j(scale * q_i^h . k_j^{g(h)}), the softmax
+ * taken over all L keys; I_sink = the n_sink positions of [cand_lo, cand_hi) with the highest S_j
+ * (ties: lower index).
+ *   Q          rows for positions [q_base, ...): the row of position p starts at (p - q_base)*q_stride_row
+ *   active_idx int32[max_active] positions (from focus_select_queries), n_active int32[1] on device
+ *   K          [Hkv, L, d] by strides
+ *   lse        float[H * max_active] (lse[h*max_active + r], natural log, as written by focus_dense_attn
+ *              for the same rows) or NULL: the library then computes it (one more pass over K)
+ *   sink_idx   int32[n_sink]; scores float[L] or NULL (receives S)
+ * n_active == 0 on the device is recorded as INVALID_ARG in the status word (outputs are -1). */
+focus_status focus_find_sinks(focus_ctx* ctx, const focus_shape* shape, const void* Q, int32_t q_base,
+                              const int32_t* active_idx, const int32_t* n_active, int32_t max_active,
+                              const void* K, const float* lse, int32_t n_sink,
+                              int32_t cand_lo, int32_t cand_hi,
+                              int32_t* sink_idx, float* scores, focus_stream stream);
+
+/* ---- stage 3: block relevance (Eq. 7) and Top-C selection (Eq. 8) --------------------------- */
+
+/* K-bar[g, b, :] = mean of the keys of prompt block b (float[Hkv * nb * d]); run once per KV-cache
+ * refresh so that focus_score_blocks need not stream K again. */
+focus_status focus_pool_keys(focus_ctx* ctx, const focus_shape* shape, const void* K, float* Kbar,
+                             focus_stream stream);
+
+/* R[g, b] = mean over the focus rows i and the heads h of group g of q_i^h . K-bar_b^{g(h)} (no
+ * softmax, no 1/sqrt(d)); G = Hkv rows (PER_KV_GROUP) or one row holding the mean over all heads (ALL).
+ * Exactly one of K (pooled on the fly, one pass over the prompt keys) and Kbar (from
+ * focus_pool_keys) must be non-NULL.  focus_idx int32[max_focus], n_focus int32[1] on device.
+ * R float[G * nb]. */
+focus_status focus_score_blocks(focus_ctx* ctx, const focus_shape* shape, const void* Q, int32_t q_base,
+                                const int32_t* focus_idx, const int32_t* n_focus, int32_t max_focus,
+                                const void* K, const float* Kbar, int32_t head_reduce,
+                                float* R, focus_stream stream);
+
+/* Per row g of R: the C highest-scoring blocks (ties: lower index), ascending, into
+ * block_idx[g*max_blocks ...] (padded -1), count into block_cnt[g].
+ * SINK_TOKENS: sink_keep[g*n_sink + s] = 1 iff sink token s lies outside every selected block of g.
+ * SINK_BLOCKS: the blocks containing the sink tokens are merged into the list (sink_keep all 0);
+ *              needs max_blocks >= min(nb, C + n_sink).
+ * Requires 0 <= C <= nb, max_blocks >= C, nb <= 8192.  sink_idx int32[n_sink] on device. */
+focus_status focus_select_blocks(focus_ctx* ctx, const focus_shape* shape, const float* R, int32_t head_reduce,
+                                 int32_t C, const int32_t* sink_idx, int32_t n_sink, int32_t sink_mode,
+                                 int32_t* block_idx, int32_t max_blocks, int32_t* block_cnt,
+                                 uint8_t* sink_keep, focus_stream stream);
+
+/* ---- stage 4: sparse attention (Eq. 9) and the dense attention of the dense layers ---------- */
+
+/* o_i^h = sum_{j in keys(h)} softmax_j(scale * q_i^h . k_j) v_j with keys(h) = tokens of the selected
+ * blocks of the head's group + kept sink tokens + every response position [M, L), each counted once.
+ *   Q        rows for positions [q_base, q_base + n_q)
+ *   q_rows   int32[max_rows] positions to compute (device) with n_rows int32[1] (device), or both NULL:
+ *            all n_q rows (then max_rows is ignored)
+ *   block_idx/block_cnt/sink_idx/sink_keep as written by focus_select_blocks (head_reduce tells whether
+ *            there is one list per KV head or one shared list); sink_keep may be NULL when n_sink == 0
+ *   O        [rows, H, d] contiguous, input dtype; output row r belongs to q_rows[r]
+ *   lse      float[H * rows_bound] (lse[h*rows_bound + r], rows_bound = max_rows or n_q) or NULL */
+focus_status focus_sparse_attn(focus_ctx* ctx, const focus_shape* shape, const void* Q, int32_t q_base, int32_t n_q,
+                               const int32_t* q_rows, const int32_t* n_rows, int32_t max_rows,
+                               const void* K, const void* V, int32_t head_reduce,
+                               const int32_t* block_idx, int32_t max_blocks, const int32_t* block_cnt,
+                               const int32_t* sink_idx, const uint8_t* sink_keep, int32_t n_sink,
+                               void* O, float* lse, focus_stream stream);
+
+/* Bidirectional softmax attention of the same rows over all L keys ("FullAttn" of Algorithm 1): the
+ * dense layers, the probe layer (its lse feeds focus_find_sinks) and the baseline of the benchmark. */
+focus_status focus_dense_attn(focus_ctx* ctx, const focus_shape* shape, const void* Q, int32_t q_base, int32_t n_q,
+                              const int32_t* q_rows, const int32_t* n_rows, int32_t max_rows,
+                              const void* K, const void* V, void* O, float* lse, focus_stream stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FOCUS_H_ */

@@ -1,0 +1,133 @@
+// Shared host/device helpers of libfocus (internal; the public ABI is include/focus.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "focus.h"
+
+struct focus_ctx {
+  int device;
+  int sm_count;
+  char* ws;            // workspace (device)
+  size_t ws_bytes;
+  int32_t* d_status;   // device status word: 0 = clean, else first anomaly's focus_status code
+  int force_simt;
+  void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime (no libcuda link)
+};
+
+// Bump allocator over the context workspace; one per API call.
+struct WsAlloc {
+  char* base;
+  size_t cap, off;
+  bool ok;
+  explicit WsAlloc(focus_ctx* c) : base(c->ws), cap(c->ws_bytes), off(0), ok(true) {}
+  template <typename T>
+  T* get(size_t n) {
+    size_t bytes = (n * sizeof(T) + 255) & ~size_t(255);
+    if (off + bytes > cap) { ok = false; return nullptr; }
+    T* p = reinterpret_cast<T*>(base + off);
+    off += bytes;
+    return p;
+  }
+};
+
+#define FOCUS_CHECK_LAUNCH()                                   \
+  do {                                                         \
+    if (cudaGetLastError() != cudaSuccess) return FOCUS_ERR_CUDA; \
+  } while (0)
+
+static inline bool shape_ok_basic(const focus_shape* s) {
+  if (!s) return false;
+  if (s->L <= 0 || s->M < 0 || s->M > s->L) return false;
+  if (s->n_q_heads <= 0 || s->n_kv_heads <= 0 || s->n_q_heads % s->n_kv_heads) return false;
+  if (s->dtype != FOCUS_F32 && s->dtype != FOCUS_BF16) return false;
+  if (s->kv_block <= 0) return false;
+  if (s->q_stride_row < s->head_dim || s->q_stride_head < s->head_dim) return false;
+  if (s->kv_stride_tok < s->head_dim || s->kv_stride_head < s->head_dim) return false;
+  if ((s->q_stride_row | s->q_stride_head | s->kv_stride_tok | s->kv_stride_head) & 7) return false;
+  return true;
+}
+static inline bool shape_supported(const focus_shape* s) {
+  return (s->head_dim == 64 || s->head_dim == 128) && (s->kv_block == 64 || s->kv_block == 128);
+}
+static inline float shape_scale(const focus_shape* s) {
+  return s->softmax_scale != 0.f ? s->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
+}
+static inline int shape_nb(const focus_shape* s) { return (s->M + s->kv_block - 1) / s->kv_block; }
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
+
+// Order-preserving map float -> uint32 (larger float => larger key).  NaN ranks below everything;
+// -0 and +0 compare equal.
+__device__ __forceinline__ uint32_t float_key(float x) {
+  if (x != x) return 0u;
+  if (x == 0.f) x = 0.f;
+  uint32_t u = __float_as_uint(x);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return u == 0u ? 1u : u;   // keep 0 for NaN only (~0xFFFFFFFF is a NaN pattern anyway)
+}
+
+__device__ __forceinline__ float load_as_float(const float* p) { return *p; }
+__device__ __forceinline__ float load_as_float(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+// Exclusive prefix sum over the thread block of one int per thread; returns the exclusive prefix and the
+// block total through `total`.  `warp_tot` is shared scratch of at least 33 ints.  All threads must call.
+__device__ __forceinline__ int block_excl_scan(int v, int* warp_tot, int& total) {
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  int x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  __syncthreads();   // protect warp_tot from a previous call's readers
+  if (lane == 31) warp_tot[wid] = x;
+  __syncthreads();
+  if (wid == 0) {
+    int t = lane < nw ? warp_tot[lane] : 0;
+    int s = t;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int y = __shfl_up_sync(0xffffffffu, s, o);
+      if (lane >= o) s += y;
+    }
+    if (lane < nw) warp_tot[lane] = s - t;
+    if (lane == 31) warp_tot[32] = s;
+  }
+  __syncthreads();
+  total = warp_tot[32];
+  return warp_tot[wid] + x - v;
+}
+#endif
+
+// ---- internal launchers (defined in the .cu files) -------------------------------------------
+struct AttnArgs {
+  focus_shape sh;
+  float scale;
+  const void* Q;
+  int q_base, n_q;
+  const int32_t* q_rows;
+  const int32_t* n_rows;
+  int max_rows;       // host bound on rows (n_q when q_rows == NULL)
+  const void* K;
+  const void* V;
+  int dense;          // 1: key set = [0, L)
+  int group_stride;   // block list row of KV head g = g * group_stride (1 per-group lists, 0 shared list)
+  const int32_t* block_idx;
+  int max_blocks;
+  const int32_t* block_cnt;
+  const int32_t* sink_idx;
+  const uint8_t* sink_keep;
+  int n_sink;
+  void* O;            // may be NULL (lse only)
+  float* lse;         // may be NULL
+  int lse_stride;
+};
+
+focus_status launch_attn_simt(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st);
+focus_status launch_attn_tc(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st);
+bool attn_tc_supported(const focus_ctx* ctx, const AttnArgs& a);
+size_t attn_tc_workspace(const focus_shape* s, int n_q, int max_blocks, int n_sink);

@@ -1,0 +1,267 @@
+// Index-set selection kernels: past-confidence indicator + window expansion (Eq. 4, Eq. 5), Top-C block
+// selection (Eq. 8) and Top-N_sink token selection (Section "Dynamic attention sinks identification").
+// All three are comparison-only: scores are mapped to order-preserving integer keys, ties go to the
+// lower index, outputs come out ascending through a block-wide prefix sum.
+#include "focus_common.cuh"
+
+// ------------------------------------------------------------------------------------------------
+// Stage 1.  One CTA.  Candidates = masked positions of [blk_lo, blk_hi); rank by counting.
+// ------------------------------------------------------------------------------------------------
+constexpr int SQ_THREADS = 256;
+constexpr int SQ_MAX_RANGE = 4096;
+constexpr int SQ_MAX_K = 1024;
+
+__global__ void __launch_bounds__(SQ_THREADS)
+select_queries_kernel(const float* __restrict__ conf, const uint8_t* __restrict__ masked, int blk_lo, int blk_hi,
+                      int k, int hw, int clip_lo, int clip_hi, int32_t* __restrict__ focus_idx,
+                      int32_t* __restrict__ n_focus, int32_t* __restrict__ active_idx, int32_t* __restrict__ n_active) {
+  __shared__ uint32_t key[SQ_MAX_RANGE];     // 0xFFFFFFFF-coded validity lives in `valid`
+  __shared__ uint8_t valid[SQ_MAX_RANGE];
+  __shared__ uint8_t sel[SQ_MAX_RANGE];
+  __shared__ int focus_s[SQ_MAX_K];
+  __shared__ int scan_s[33];
+  const int n = blk_hi - blk_lo;
+  const int tid = threadIdx.x;
+  for (int i = tid; i < n; i += SQ_THREADS) {
+    key[i] = float_key(conf[blk_lo + i]);
+    valid[i] = masked[blk_lo + i] != 0;
+  }
+  __syncthreads();
+  for (int i = tid; i < n; i += SQ_THREADS) {
+    int rank = 0;
+    if (valid[i]) {
+      const uint32_t ki = key[i];
+      for (int j = 0; j < n; ++j) {
+        const uint32_t kj = key[j];
+        rank += (valid[j] && (kj > ki || (kj == ki && j < i))) ? 1 : 0;
+      }
+    }
+    sel[i] = valid[i] && rank < k;
+  }
+  __syncthreads();
+  // ascending compaction of the selected positions
+  int base = 0;
+  for (int c0 = 0; c0 < n; c0 += SQ_THREADS) {
+    const int i = c0 + tid;
+    const int f = (i < n && sel[i]) ? 1 : 0;
+    int tot;
+    const int pre = block_excl_scan(f, scan_s, tot);
+    if (f) {
+      focus_s[base + pre] = blk_lo + i;
+      focus_idx[base + pre] = blk_lo + i;
+    }
+    base += tot;
+  }
+  const int nf = base;                       // = min(k, #candidates)
+  for (int i = nf + tid; i < k; i += SQ_THREADS) focus_idx[i] = -1;
+  if (tid == 0) *n_focus = nf;
+  __syncthreads();
+  // windows: pick i contributes the part of [f_i - hw, f_i + hw] not already covered by pick i-1
+  const int span = 2 * hw + 1;
+  int abase = 0;
+  for (int c0 = 0; c0 < nf; c0 += SQ_THREADS) {
+    const int i = c0 + tid;
+    int lo = 0, cnt = 0;
+    if (i < nf) {
+      const int f = focus_s[i];
+      lo = max(f - hw, clip_lo);
+      if (i > 0) lo = max(lo, focus_s[i - 1] + hw + 1);
+      const int hi = min(f + hw, clip_hi - 1);
+      cnt = max(0, hi - lo + 1);
+    }
+    int tot;
+    const int pre = block_excl_scan(cnt, scan_s, tot);
+    for (int t = 0; t < cnt; ++t) active_idx[abase + pre + t] = lo + t;
+    abase += tot;
+  }
+  for (int i = abase + tid; i < k * span; i += SQ_THREADS) active_idx[i] = -1;
+  if (tid == 0) *n_active = abase;
+}
+
+extern "C" focus_status focus_select_queries(focus_ctx* ctx, const float* conf_prev, const uint8_t* masked, int32_t L,
+                                             int32_t blk_lo, int32_t blk_hi, int32_t k, int32_t w, int32_t clip_lo,
+                                             int32_t clip_hi, int32_t* focus_idx, int32_t* n_focus,
+                                             int32_t* active_idx, int32_t* n_active, focus_stream stream) {
+  if (!ctx || !conf_prev || !masked || !focus_idx || !n_focus || !active_idx || !n_active) return FOCUS_ERR_INVALID_ARG;
+  if (L <= 0 || blk_lo < 0 || blk_hi < blk_lo || blk_hi > L || k < 0 || w < 0) return FOCUS_ERR_INVALID_ARG;
+  if (clip_lo < 0 || clip_hi > L || clip_hi < clip_lo) return FOCUS_ERR_INVALID_ARG;
+  if (blk_hi - blk_lo > SQ_MAX_RANGE || k > SQ_MAX_K) return FOCUS_ERR_UNSUPPORTED;
+  select_queries_kernel<<<1, SQ_THREADS, 0, stream>>>(conf_prev, masked, blk_lo, blk_hi, k, w / 2, clip_lo, clip_hi,
+                                                      focus_idx, n_focus, active_idx, n_active);
+  FOCUS_CHECK_LAUNCH();
+  return FOCUS_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Stage 3b.  One CTA per group: rank-by-counting Top-C over nb <= 8192 block scores.
+// ------------------------------------------------------------------------------------------------
+constexpr int SB_THREADS = 1024;
+constexpr int SB_MAX_NB = 8192;
+
+__global__ void __launch_bounds__(SB_THREADS)
+select_blocks_kernel(const float* __restrict__ R, int nb, int C, int B, const int32_t* __restrict__ sink_idx,
+                     int n_sink, int sink_blocks_mode, int32_t* __restrict__ block_idx, int max_blocks,
+                     int32_t* __restrict__ block_cnt, uint8_t* __restrict__ sink_keep, int32_t* status) {
+  __shared__ uint32_t key[SB_MAX_NB];
+  __shared__ uint8_t sel[SB_MAX_NB];
+  __shared__ int scan_s[33];
+  const int g = blockIdx.x, tid = threadIdx.x;
+  const float* Rg = R + (size_t)g * nb;
+  for (int i = tid; i < nb; i += SB_THREADS) key[i] = float_key(Rg[i]);
+  __syncthreads();
+  for (int i = tid; i < nb; i += SB_THREADS) {
+    const uint32_t ki = key[i];
+    int rank = 0;
+    for (int j = 0; j < nb; ++j) {
+      const uint32_t kj = key[j];
+      rank += (kj > ki || (kj == ki && j < i)) ? 1 : 0;
+    }
+    sel[i] = rank < C;
+  }
+  __syncthreads();
+  for (int s = tid; s < n_sink; s += SB_THREADS) {
+    const int j = sink_idx[s];
+    const int b = j / B;
+    if (j < 0 || b >= nb) {
+      set_status(status, FOCUS_ERR_INVALID_ARG);
+      if (sink_keep) sink_keep[(size_t)g * n_sink + s] = 0;
+      continue;
+    }
+    if (sink_blocks_mode) {
+      sel[b] = 1;                                   // benign race: every writer stores 1
+      if (sink_keep) sink_keep[(size_t)g * n_sink + s] = 0;
+    } else {
+      sink_keep[(size_t)g * n_sink + s] = sel[b] ? 0 : 1;
+    }
+  }
+  __syncthreads();
+  int base = 0;
+  int32_t* out = block_idx + (size_t)g * max_blocks;
+  for (int c0 = 0; c0 < nb; c0 += SB_THREADS) {
+    const int i = c0 + tid;
+    const int f = (i < nb && sel[i]) ? 1 : 0;
+    int tot;
+    const int pre = block_excl_scan(f, scan_s, tot);
+    if (f && base + pre < max_blocks) out[base + pre] = i;
+    base += tot;
+  }
+  if (base > max_blocks) {
+    if (tid == 0) set_status(status, FOCUS_ERR_INVALID_ARG);
+    base = max_blocks;
+  }
+  for (int i = base + tid; i < max_blocks; i += SB_THREADS) out[i] = -1;
+  if (tid == 0) block_cnt[g] = base;
+}
+
+extern "C" focus_status focus_select_blocks(focus_ctx* ctx, const focus_shape* shape, const float* R,
+                                            int32_t head_reduce, int32_t C, const int32_t* sink_idx, int32_t n_sink,
+                                            int32_t sink_mode, int32_t* block_idx, int32_t max_blocks,
+                                            int32_t* block_cnt, uint8_t* sink_keep, focus_stream stream) {
+  if (!ctx || !shape_ok_basic(shape) || !R || !block_idx || !block_cnt) return FOCUS_ERR_INVALID_ARG;
+  const int nb = shape_nb(shape);
+  if (C < 0 || C > nb || max_blocks < C || n_sink < 0) return FOCUS_ERR_INVALID_ARG;
+  if (n_sink > 0 && !sink_idx) return FOCUS_ERR_INVALID_ARG;
+  if (head_reduce != FOCUS_HEADS_PER_KV_GROUP && head_reduce != FOCUS_HEADS_ALL) return FOCUS_ERR_INVALID_ARG;
+  if (sink_mode != FOCUS_SINK_TOKENS && sink_mode != FOCUS_SINK_BLOCKS) return FOCUS_ERR_INVALID_ARG;
+  if (sink_mode == FOCUS_SINK_TOKENS && n_sink > 0 && !sink_keep) return FOCUS_ERR_INVALID_ARG;
+  if (sink_mode == FOCUS_SINK_BLOCKS && max_blocks < (nb < C + n_sink ? nb : C + n_sink)) return FOCUS_ERR_INVALID_ARG;
+  if (nb > SB_MAX_NB) return FOCUS_ERR_UNSUPPORTED;
+  if (nb == 0 && max_blocks == 0) {
+    // nothing to select; counts still have to be defined
+  }
+  const int G = head_reduce == FOCUS_HEADS_ALL ? 1 : shape->n_kv_heads;
+  select_blocks_kernel<<<G, SB_THREADS, 0, stream>>>(R, nb, C, shape->kv_block, sink_idx, n_sink,
+                                                     sink_mode == FOCUS_SINK_BLOCKS, block_idx, max_blocks, block_cnt,
+                                                     sink_keep, ctx->d_status);
+  FOCUS_CHECK_LAUNCH();
+  return FOCUS_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Stage 2, selection half.  sink_reduce_heads: S[j] = inv * sum_h part[h][j] in fixed head order.
+// sink_topn: one CTA, 8-bit radix select of the n-th largest key, then ascending ordered compaction.
+// ------------------------------------------------------------------------------------------------
+__global__ void sink_reduce_heads_kernel(const float* __restrict__ part, int H, int L, const int32_t* n_active,
+                                         float* __restrict__ S) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= L) return;
+  float acc = 0.f;
+  for (int h = 0; h < H; ++h) acc += part[(size_t)h * L + j];
+  const int n = *n_active;
+  S[j] = n > 0 ? acc / ((float)H * (float)n) : 0.f;
+}
+
+constexpr int TN_THREADS = 1024;
+
+__global__ void __launch_bounds__(TN_THREADS)
+sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const int32_t* n_active,
+                 int32_t* __restrict__ sink_idx, int32_t* status) {
+  __shared__ int hist[256];
+  __shared__ int scan_s[33];
+  __shared__ uint32_t s_prefix;
+  __shared__ int s_remaining;
+  const int tid = threadIdx.x;
+  const int n = hi - lo;
+  const int want = min(n_sink, n);
+  if (*n_active <= 0) {                      // undefined scores: report and emit an empty set
+    if (tid == 0) set_status(status, FOCUS_ERR_INVALID_ARG);
+    for (int i = tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
+    return;
+  }
+  if (want == 0) {
+    for (int i = tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
+    return;
+  }
+  // radix select: find the key T of the want-th largest element, MSB first
+  uint32_t prefix = 0, pmask = 0;
+  int remaining = want;                       // rank (1-based) still to locate inside the current bucket
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int b = tid; b < 256; b += TN_THREADS) hist[b] = 0;
+    __syncthreads();
+    for (int i = tid; i < n; i += TN_THREADS) {
+      const uint32_t k = float_key(S[lo + i]);
+      if ((k & pmask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int acc = 0, b = 255;
+      for (; b > 0; --b) {
+        if (acc + hist[b] >= remaining) break;
+        acc += hist[b];
+      }
+      s_prefix = prefix | ((uint32_t)b << shift);
+      s_remaining = remaining - acc;
+    }
+    __syncthreads();
+    prefix = s_prefix;
+    remaining = s_remaining;
+    pmask |= 255u << shift;
+    __syncthreads();
+  }
+  const uint32_t T = prefix;                 // threshold key; `remaining` = how many == T to take (lowest index first)
+  int base = 0, eq_taken = 0;
+  for (int c0 = 0; c0 < n; c0 += TN_THREADS) {
+    const int i = c0 + tid;
+    uint32_t k = 0;
+    if (i < n) k = float_key(S[lo + i]);
+    const int is_eq = (i < n && k == T) ? 1 : 0;
+    int tot_eq;
+    const int pre_eq = block_excl_scan(is_eq, scan_s, tot_eq);
+    const int f = (i < n && (k > T || (is_eq && eq_taken + pre_eq < remaining))) ? 1 : 0;
+    int tot;
+    const int pre = block_excl_scan(f, scan_s, tot);
+    if (f) sink_idx[base + pre] = lo + i;
+    base += tot;
+    eq_taken += tot_eq;
+  }
+  for (int i = base + tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
+}
+
+focus_status launch_sink_select(focus_ctx* ctx, const float* part, int H, int L, const int32_t* n_active, float* S,
+                                int cand_lo, int cand_hi, int n_sink, int32_t* sink_idx, cudaStream_t st) {
+  sink_reduce_heads_kernel<<<(L + 255) / 256, 256, 0, st>>>(part, H, L, n_active, S);
+  FOCUS_CHECK_LAUNCH();
+  sink_topn_kernel<<<1, TN_THREADS, 0, st>>>(S, cand_lo, cand_hi, n_sink, n_active, sink_idx, ctx->d_status);
+  FOCUS_CHECK_LAUNCH();
+  return FOCUS_OK;
+}

@@ -1,0 +1,107 @@
+"""Device-buffer bookkeeping for one Focus-dLLM denoising step (harness level).
+
+`StepBuffers` owns the caller-side buffers the C ABI writes into (index sets, counts, block scores, outputs)
+and `run_layer_*` issue the library calls of one layer in the order of Algorithm 1.  No arithmetic happens
+here; torch tensors are device memory only.
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import binding as fb
+from .workloads import Shape, Workload
+
+
+def torch_dtype(dtype: str):
+    return torch.float32 if dtype == "f32" else torch.bfloat16
+
+
+def to_device(a: np.ndarray, dtype: str, device="cuda") -> torch.Tensor:
+    """Storage array (float32, or uint16 bf16 bit patterns) -> device tensor of the matching torch dtype."""
+    if dtype == "f32":
+        return torch.from_numpy(np.ascontiguousarray(a)).to(device)
+    return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+def from_device(t: torch.Tensor) -> np.ndarray:
+    """Device tensor -> float64 numpy (exact widening)."""
+    return t.detach().to(torch.float64).cpu().numpy()
+
+
+def c_shape(s: Shape) -> fb.focus_shape:
+    return fb.make_shape(s.L, s.M, s.H, s.Hkv, s.d, s.B, fb.F32 if s.dtype == "f32" else fb.BF16)
+
+
+@dataclasses.dataclass
+class StepBuffers:
+    """Caller-owned outputs of the selection stages and of attention for one workload."""
+    wl: Workload
+    head_reduce: int = fb.HEADS_PER_KV_GROUP
+    sink_mode: int = fb.SINK_TOKENS
+    rows: str = "active"              # "active": attention rows are I_active (the paper); "gen": all N gen rows
+    device: str = "cuda"
+
+    def __post_init__(self):
+        w, s = self.wl, self.wl.shape
+        dev = self.device
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.shape = c_shape(s)
+        self.max_active = max(1, w.k * (2 * (w.w // 2) + 1))
+        self.G = 1 if self.head_reduce == fb.HEADS_ALL else s.Hkv
+        self.max_blocks = max(1, min(s.nb, w.C + w.n_sink) if self.sink_mode == fb.SINK_BLOCKS else w.C)
+        self.focus_idx = torch.full((max(1, w.k),), -1, **i32)
+        self.n_focus = torch.zeros(1, **i32)
+        self.active_idx = torch.full((self.max_active,), -1, **i32)
+        self.n_active = torch.zeros(1, **i32)
+        self.sink_idx = torch.full((max(1, w.n_sink),), -1, **i32)
+        self.sink_scores = torch.zeros(s.L, dtype=torch.float32, device=dev)
+        self.R = torch.zeros(self.G * max(1, s.nb), dtype=torch.float32, device=dev)
+        self.block_idx = torch.full((self.G * self.max_blocks,), -1, **i32)
+        self.block_cnt = torch.zeros(self.G, **i32)
+        self.sink_keep = torch.zeros(self.G * max(1, w.n_sink), dtype=torch.uint8, device=dev)
+        self.max_rows = self.max_active if self.rows == "active" else s.N
+        self.O = torch.zeros(self.max_rows, s.H, s.d, dtype=torch_dtype(s.dtype), device=dev)
+        self.lse = torch.zeros(s.H, self.max_rows, dtype=torch.float32, device=dev)
+
+    # rows argument triple of the attention calls
+    def _rows(self):
+        if self.rows == "active":
+            return self.active_idx, self.n_active, self.max_active
+        return None, None, 0
+
+
+def select_queries(ctx, b: StepBuffers, conf_prev: torch.Tensor, masked: torch.Tensor, stream=None):
+    w, s = b.wl, b.wl.shape
+    fb.focus_select_queries(ctx, conf_prev, masked, s.L, w.blk_lo, w.blk_hi, w.k, w.w, s.M, s.L,
+                            b.focus_idx, b.n_focus, b.active_idx, b.n_active, stream)
+
+
+def dense_layer(ctx, b: StepBuffers, Q, K, V, O=None, lse=None, stream=None):
+    s = b.wl.shape
+    q_rows, n_rows, max_rows = b._rows()
+    fb.focus_dense_attn(ctx, b.shape, Q, s.M, s.N, q_rows, n_rows, max_rows, K, V, b.O if O is None else O,
+                        b.lse if lse is None else lse, stream)
+
+
+def find_sinks(ctx, b: StepBuffers, Q, K, lse: Optional[torch.Tensor], stream=None):
+    """lse must be the [H, max_active] log-sum-exp of a dense pass over the I_active rows, or None."""
+    w, s = b.wl, b.wl.shape
+    fb.focus_find_sinks(ctx, b.shape, Q, s.M, b.active_idx, b.n_active, b.max_active, K, lse, w.n_sink, 0, s.M,
+                        b.sink_idx, b.sink_scores, stream)
+
+
+def sparse_layer(ctx, b: StepBuffers, Q, K, V, Kbar: Optional[torch.Tensor] = None, O=None, lse=None, stream=None):
+    """score_blocks -> select_blocks -> sparse_attn for one sparse layer (Algorithm 1, sparse branch)."""
+    w, s = b.wl, b.wl.shape
+    fb.focus_score_blocks(ctx, b.shape, Q, s.M, b.focus_idx, b.n_focus, max(1, w.k), None if Kbar is not None else K,
+                          Kbar, b.head_reduce, b.R, stream)
+    fb.focus_select_blocks(ctx, b.shape, b.R, b.head_reduce, w.C, b.sink_idx, w.n_sink, b.sink_mode, b.block_idx,
+                           b.max_blocks, b.block_cnt, b.sink_keep, stream)
+    q_rows, n_rows, max_rows = b._rows()
+    fb.focus_sparse_attn(ctx, b.shape, Q, s.M, s.N, q_rows, n_rows, max_rows, K, V, b.head_reduce, b.block_idx,
+                         b.max_blocks, b.block_cnt, b.sink_idx, b.sink_keep, w.n_sink, b.O if O is None else O,
+                         b.lse if lse is None else lse, stream)

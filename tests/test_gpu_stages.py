@@ -1,0 +1,338 @@
+"""GPU parity: every stage of the path, called through the C ABI, against the CPU oracle on the same seeded
+inputs.  Small shapes span several key tiles, a ragged last prompt block and a ragged response tail."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import focus_oracle as fo
+from paper_2602_02159_b200 import binding as fb
+from paper_2602_02159_b200 import step as fstep
+from paper_2602_02159_b200 import workloads as wl
+from tests.helpers import check_topk_band, max_abs, rel_rms
+
+pytestmark = pytest.mark.gpu
+
+TOL_ABS = {"f32": 1e-5, "bf16": 2e-2}       # contractual max-abs on attention outputs
+TOL_RMS = {"f32": 1e-5, "bf16": 1e-2}       # self-imposed relative RMS (outputs are ~1e-3..1e-2 in size)
+TOL_LSE = {"f32": 1e-4, "bf16": 1e-3}
+BAND = 1e-3
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = fb.Context(0)
+    yield c
+    assert c.poll_status() == 0
+    c.close()
+
+
+def small_workload(dtype, d, B, H=4, Hkv=4, L=1500, M=1100, k=6, w=8, n_sink=9, C=3, seed=3, blk=None):
+    s = wl.Shape(L, M, H, Hkv, d, B, dtype)
+    lo, hi = blk if blk else (M, min(L, M + 96))
+    return wl.Workload(f"small_{dtype}_{d}_{B}", s, k=k, w=w, n_sink=n_sink, C=C, blk_lo=lo, blk_hi=hi, seed=seed)
+
+
+SHAPES = [
+    pytest.param(("f32", 64, 64, 4, 4), id="f32_d64_B64"),
+    pytest.param(("f32", 128, 128, 4, 2), id="f32_d128_gqa"),
+    pytest.param(("bf16", 128, 128, 4, 4), id="bf16_d128_B128_mha"),
+    pytest.param(("bf16", 128, 128, 8, 2), id="bf16_d128_B128_gqa"),
+    pytest.param(("bf16", 64, 64, 4, 4), id="bf16_d64_B64"),
+    pytest.param(("bf16", 128, 64, 4, 4), id="bf16_d128_B64"),
+]
+
+
+def make_inputs(w, variant="fix"):
+    s = w.shape
+    t = wl.gen_qkv(s, w.seed, variant=variant, threads=4)
+    c_prev, _ = wl.gen_confidence(w.seed, s.N)
+    masked = wl.gen_masked(w)
+    rng = np.random.default_rng(w.seed + 100)
+    masked[s.M:][rng.random(s.N) < 0.3] = 0            # some gen positions already decoded
+    host = dict(Q=wl.storage_to_f64(t["Q"], s.dtype), K=wl.storage_to_f64(t["K"], s.dtype),
+                V=wl.storage_to_f64(t["V"], s.dtype), conf=wl.full_conf(s, c_prev), masked=masked,
+                sink_pos=t["sink_pos"])
+    dev = dict(Q=fstep.to_device(t["Q"], s.dtype), K=fstep.to_device(t["K"], s.dtype),
+               V=fstep.to_device(t["V"], s.dtype), conf=torch.from_numpy(host["conf"]).cuda(),
+               masked=torch.from_numpy(masked).cuda())
+    return host, dev
+
+
+def oracle_chain(w, host, head_reduce, sink_mode):
+    s = w.shape
+    scale = 1.0 / math.sqrt(s.d)
+    focus, active = fo.select_queries(host["conf"], host["masked"], w.blk_lo, w.blk_hi, w.k, w.w, s.M, s.L)
+    Qa = host["Q"][active - s.M]
+    S = fo.sink_scores(Qa, host["K"], scale)
+    sinks = fo.find_sinks(S, w.n_sink, 0, s.M)
+    Kbar = fo.pool_keys(host["K"], s.M, s.B)
+    R = fo.score_blocks(host["Q"][focus - s.M], Kbar, head_reduce)
+    blocks, keep = fo.select_blocks(R, w.C, sinks, s.B, sink_mode)
+    return dict(focus=focus, active=active, S=S, sinks=sinks, Kbar=Kbar, R=R, blocks=blocks, keep=keep, scale=scale)
+
+
+# --------------------------------------------------------------------------------------------------
+def test_select_queries_exact(ctx):
+    """Comparison-only stage: bit-exact, no band.  Includes ties, NaN, k > candidates, k = 0, clipping."""
+    rng = np.random.default_rng(0)
+    cases = []
+    for trial in range(12):
+        L = int(rng.integers(40, 3000))
+        M = int(rng.integers(0, L // 2))
+        conf = rng.beta(2, 5, size=L).astype(np.float32)
+        if trial % 3 == 0:
+            conf = np.round(conf * 8) / 8                     # many ties
+        if trial % 4 == 1:
+            conf[rng.integers(0, L, size=5)] = np.nan
+        if trial % 5 == 2:
+            conf[rng.integers(0, L, size=5)] = -0.0
+        masked = (rng.random(L) < 0.6).astype(np.uint8)
+        lo = int(rng.integers(M, L))
+        hi = int(rng.integers(lo, min(L, lo + 600) + 1))
+        k = int(rng.integers(0, 40))
+        w = int(rng.integers(0, 12))
+        cases.append((conf, masked, L, lo, hi, k, w, M, L))
+    conf = np.full(64, 0.5, dtype=np.float32)
+    cases.append((conf, np.ones(64, dtype=np.uint8), 64, 0, 64, 8, 8, 0, 64))            # all equal
+    cases.append((conf, np.zeros(64, dtype=np.uint8), 64, 0, 64, 8, 8, 0, 64))           # nothing masked
+    cases.append((conf, np.ones(64, dtype=np.uint8), 64, 10, 10, 8, 8, 0, 64))           # empty block
+    cases.append((conf, np.ones(64, dtype=np.uint8), 64, 0, 64, 4, 8, 20, 30))           # clip excludes everything near picks
+    for conf, masked, L, lo, hi, k, w, clo, chi in cases:
+        span = 2 * (w // 2) + 1
+        f = torch.full((max(1, k),), -7, dtype=torch.int32, device="cuda")
+        a = torch.full((max(1, k * span),), -7, dtype=torch.int32, device="cuda")
+        nf = torch.zeros(1, dtype=torch.int32, device="cuda")
+        na = torch.zeros(1, dtype=torch.int32, device="cuda")
+        fb.focus_select_queries(ctx, torch.from_numpy(conf).cuda(), torch.from_numpy(masked).cuda(), L, lo, hi, k, w,
+                                clo, chi, f, nf, a, na)
+        ef, ea = fo.select_queries(conf, masked, lo, hi, k, w, clo, chi)
+        assert nf.item() == len(ef) and na.item() == len(ea)
+        assert f.cpu().numpy()[:len(ef)].tolist() == ef.tolist()
+        assert a.cpu().numpy()[:len(ea)].tolist() == ea.tolist()
+        if k > 0:
+            assert (f.cpu().numpy()[len(ef):k] == -1).all() and (a.cpu().numpy()[len(ea):k * span] == -1).all()
+
+
+@pytest.mark.parametrize("cfg", SHAPES)
+@pytest.mark.parametrize("force_simt", [False, True], ids=["auto", "simt"])
+def test_stages_against_oracle(ctx, cfg, force_simt):
+    """Each stage is fed the ORACLE's upstream index sets so that stages are judged in isolation."""
+    dtype, d, B, H, Hkv = cfg
+    w = small_workload(dtype, d, B, H=H, Hkv=Hkv)
+    s = w.shape
+    ctx.set_force_simt(force_simt)
+    try:
+        for head_reduce in (fb.HEADS_PER_KV_GROUP, fb.HEADS_ALL):
+            host, dev = make_inputs(w)
+            ora = oracle_chain(w, host, head_reduce, fb.SINK_TOKENS)
+            b = fstep.StepBuffers(w, head_reduce=head_reduce)
+            # stage 1
+            fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
+            assert b.focus_idx.cpu().numpy()[:b.n_focus.item()].tolist() == ora["focus"].tolist()
+            assert b.active_idx.cpu().numpy()[:b.n_active.item()].tolist() == ora["active"].tolist()
+            na = len(ora["active"])
+            # dense attention over the active rows (+ LSE)
+            fstep.dense_layer(ctx, b, dev["Q"], dev["K"], dev["V"])
+            Od, lsed = fo.dense_attn(host["Q"][ora["active"] - s.M], host["K"], host["V"], ora["scale"])
+            got = fstep.from_device(b.O)[:na]
+            assert max_abs(got, Od) <= TOL_ABS[dtype] and rel_rms(got, Od) <= TOL_RMS[dtype]
+            assert max_abs(fstep.from_device(b.lse)[:, :na], lsed) <= TOL_LSE[dtype]
+            # stage 2, with the dense pass's LSE and with the library computing its own
+            for lse_in in (b.lse, None):
+                b.sink_idx.fill_(-5)
+                fstep.find_sinks(ctx, b, dev["Q"], dev["K"], lse_in)
+                S_gpu = fstep.from_device(b.sink_scores)
+                assert abs(S_gpu.sum() - 1.0) < 1e-3
+                assert np.max(np.abs(S_gpu - ora["S"]) / ora["S"]) < 2e-3
+                check_topk_band(b.sink_idx.cpu().numpy(), ora["sinks"], ora["S"], range(0, s.M), BAND, what="sinks")
+                assert set(host["sink_pos"].tolist()) <= set(b.sink_idx.cpu().numpy().tolist())
+            # stage 3a cold (streams K) and warm (cached K-bar)
+            b.sink_idx.copy_(torch.from_numpy(ora["sinks"].astype(np.int32)))
+            Kbar = torch.zeros(s.Hkv, s.nb, s.d, dtype=torch.float32, device="cuda")
+            fb.focus_pool_keys(ctx, b.shape, dev["K"], Kbar)
+            assert max_abs(fstep.from_device(Kbar), ora["Kbar"]) < 1e-5
+            for kbar_in in (None, Kbar):
+                b.R.zero_()
+                fb.focus_score_blocks(ctx, b.shape, dev["Q"], s.M, b.focus_idx, b.n_focus, w.k,
+                                      dev["K"] if kbar_in is None else None, kbar_in, head_reduce, b.R)
+                Rg = fstep.from_device(b.R).reshape(b.G, s.nb)
+                assert max_abs(Rg, ora["R"]) <= 1e-5 * max(1.0, np.abs(ora["R"]).max())
+            # stage 3b from the GPU's own scores
+            fb.focus_select_blocks(ctx, b.shape, b.R, head_reduce, w.C, b.sink_idx, w.n_sink, fb.SINK_TOKENS,
+                                   b.block_idx, b.max_blocks, b.block_cnt, b.sink_keep)
+            bi = b.block_idx.cpu().numpy().reshape(b.G, b.max_blocks)
+            for g in range(b.G):
+                assert b.block_cnt[g].item() == w.C
+                check_topk_band(bi[g], ora["blocks"][g], ora["R"][g], range(s.nb), BAND,
+                                scale_ref=np.abs(ora["R"][g]).max(), what=f"blocks g{g}")
+            # stage 4 on the oracle's sets
+            b.block_idx.copy_(torch.from_numpy(np.stack(ora["blocks"]).astype(np.int32).reshape(-1)))
+            b.sink_keep.copy_(torch.from_numpy(ora["keep"].reshape(-1)))
+            q_rows, n_rows, max_rows = b._rows()
+            fb.focus_sparse_attn(ctx, b.shape, dev["Q"], s.M, s.N, q_rows, n_rows, max_rows, dev["K"], dev["V"],
+                                 head_reduce, b.block_idx, b.max_blocks, b.block_cnt, b.sink_idx, b.sink_keep,
+                                 w.n_sink, b.O, b.lse)
+            Os, lses = fo.sparse_attn(host["Q"][ora["active"] - s.M], host["K"], host["V"], s.M, s.B, ora["blocks"],
+                                      ora["sinks"], ora["scale"])
+            got = fstep.from_device(b.O)[:na]
+            assert max_abs(got, Os) <= TOL_ABS[dtype] and rel_rms(got, Os) <= TOL_RMS[dtype]
+            assert max_abs(fstep.from_device(b.lse)[:, :na], lses) <= TOL_LSE[dtype]
+            assert ctx.poll_status() == 0
+    finally:
+        ctx.set_force_simt(False)
+
+
+@pytest.mark.parametrize("cfg", SHAPES)
+def test_gen_rows_keep_all_equals_dense_and_sharp_logits(ctx, cfg):
+    """All N gen rows as queries (q_rows = NULL); keep ratio 1 must reproduce dense attention; Q, K ~ N(0,1)
+    gives peaky softmax rows where the 2e-2 bound on bf16 outputs is a meaningful test."""
+    dtype, d, B, H, Hkv = cfg
+    s = wl.Shape(1400, 1000, H, Hkv, d, B, dtype)
+    rng = np.random.default_rng(5)
+    Qs = wl.to_storage(rng.standard_normal((s.N, H, d)).astype(np.float32) * 0.6, dtype)
+    Ks = wl.to_storage(rng.standard_normal((Hkv, s.L, d)).astype(np.float32) * 0.6, dtype)
+    Vs = wl.to_storage(rng.standard_normal((Hkv, s.L, d)).astype(np.float32), dtype)
+    Q, K, V = (wl.storage_to_f64(x, dtype) for x in (Qs, Ks, Vs))
+    dQ, dK, dV = (fstep.to_device(x, dtype) for x in (Qs, Ks, Vs))
+    sh = fstep.c_shape(s)
+    O = torch.zeros(s.N, H, d, dtype=fstep.torch_dtype(dtype), device="cuda")
+    lse = torch.zeros(H, s.N, dtype=torch.float32, device="cuda")
+    scale = 1.0 / math.sqrt(d)
+    fb.focus_dense_attn(ctx, sh, dQ, s.M, s.N, None, None, 0, dK, dV, O, lse)
+    Od, ld = fo.dense_attn(Q, K, V, scale)
+    assert np.sqrt(np.mean(Od ** 2)) > 0.05
+    tol = 2e-2 if dtype == "bf16" else 2e-5
+    assert max_abs(fstep.from_device(O), Od) <= tol
+    assert max_abs(fstep.from_device(lse), ld) <= (2e-3 if dtype == "bf16" else 1e-4)
+    dense_out = O.clone()
+    # keep every block, plus sinks that all lie inside kept blocks -> identical key set
+    G = Hkv
+    nb = s.nb
+    bidx = torch.arange(nb, dtype=torch.int32, device="cuda").repeat(G)
+    bcnt = torch.full((G,), nb, dtype=torch.int32, device="cuda")
+    sinks = torch.tensor([0, 77, 999], dtype=torch.int32, device="cuda")
+    keep = torch.zeros(G * 3, dtype=torch.uint8, device="cuda")
+    fb.focus_sparse_attn(ctx, sh, dQ, s.M, s.N, None, None, 0, dK, dV, fb.HEADS_PER_KV_GROUP, bidx, nb, bcnt, sinks,
+                         keep, 3, O, lse)
+    assert max_abs(fstep.from_device(O), Od) <= tol
+    assert max_abs(fstep.from_device(O), fstep.from_device(dense_out)) <= tol
+    assert ctx.poll_status() == 0
+
+
+def test_degenerate_cases(ctx):
+    """C = 0 with no sinks (response keys only), n_sink = 0, Q = 0 (uniform weights pin the key set),
+    a single query row, block list given in descending order."""
+    dtype, d, B, H, Hkv = "bf16", 128, 128, 4, 2
+    s = wl.Shape(900, 700, H, Hkv, d, B, dtype)          # nb = 6, last block 60 tokens; response 200 (ragged)
+    rng = np.random.default_rng(9)
+    Ks = wl.to_storage(rng.standard_normal((Hkv, s.L, d)).astype(np.float32), dtype)
+    Vs = wl.to_storage(rng.standard_normal((Hkv, s.L, d)).astype(np.float32), dtype)
+    K, V = wl.storage_to_f64(Ks, dtype), wl.storage_to_f64(Vs, dtype)
+    dK, dV = fstep.to_device(Ks, dtype), fstep.to_device(Vs, dtype)
+    sh = fstep.c_shape(s)
+    for force in (False, True):
+        ctx.set_force_simt(force)
+        for nrow in (1, 200):
+            Qz = torch.zeros(s.N, H, d, dtype=torch.bfloat16, device="cuda")
+            O = torch.zeros(nrow, H, d, dtype=torch.bfloat16, device="cuda")
+            lse = torch.zeros(H, nrow, dtype=torch.float32, device="cuda")
+            blocks = [np.array([5, 2]), np.array([0])]
+            bidx = torch.tensor([5, 2, 0, -1], dtype=torch.int32, device="cuda")
+            bcnt = torch.tensor([2, 1], dtype=torch.int32, device="cuda")
+            sinks_np = np.array([3, 300, 650])                                  # 300 in block 2, 650 in block 5
+            sinks = torch.from_numpy(sinks_np.astype(np.int32)).cuda()
+            keep = torch.tensor([1, 0, 0, 0, 1, 1], dtype=torch.uint8, device="cuda")
+            fb.focus_sparse_attn(ctx, sh, Qz, s.M, nrow, None, None, 0, dK, dV, fb.HEADS_PER_KV_GROUP, bidx, 2, bcnt,
+                                 sinks, keep, 3, O, lse)
+            got = fstep.from_device(O)
+            for h in range(H):
+                ks = fo.key_set(s.M, s.L, B, blocks[h // 2], sinks_np)
+                assert max_abs(got[0, h], V[h // 2, ks].mean(axis=0)) < 4e-3
+                assert abs(lse[h, 0].item() - math.log(len(ks))) < 1e-4
+            # nothing kept from the prompt
+            bcnt0 = torch.zeros(2, dtype=torch.int32, device="cuda")
+            fb.focus_sparse_attn(ctx, sh, Qz, s.M, nrow, None, None, 0, dK, dV, fb.HEADS_PER_KV_GROUP, bidx, 2, bcnt0,
+                                 None, None, 0, O, lse)
+            got = fstep.from_device(O)
+            for h in range(H):
+                assert max_abs(got[0, h], V[h // 2, s.M:].mean(axis=0)) < 4e-3
+        ctx.set_force_simt(False)
+    assert ctx.poll_status() == 0
+
+
+def test_sink_blocks_mode_and_bad_indices_are_reported(ctx):
+    w = small_workload("f32", 64, 64)
+    s = w.shape
+    host, dev = make_inputs(w)
+    ora = oracle_chain(w, host, fb.HEADS_PER_KV_GROUP, fb.SINK_BLOCKS)
+    b = fstep.StepBuffers(w, sink_mode=fb.SINK_BLOCKS)
+    R = torch.from_numpy(ora["R"].astype(np.float32).reshape(-1)).cuda()
+    b.sink_idx.copy_(torch.from_numpy(ora["sinks"].astype(np.int32)))
+    fb.focus_select_blocks(ctx, b.shape, R, fb.HEADS_PER_KV_GROUP, w.C, b.sink_idx, w.n_sink, fb.SINK_BLOCKS,
+                           b.block_idx, b.max_blocks, b.block_cnt, b.sink_keep)
+    bi = b.block_idx.cpu().numpy().reshape(b.G, b.max_blocks)
+    for g in range(b.G):
+        n = b.block_cnt[g].item()
+        assert bi[g, :n].tolist() == ora["blocks"][g].tolist() and (bi[g, n:] == -1).all()
+    assert b.sink_keep.sum().item() == 0
+    assert ctx.poll_status() == 0
+    # a block index out of range is skipped and reported, not dereferenced
+    b.block_idx[0] = 10 ** 6
+    fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
+    q_rows, n_rows, max_rows = b._rows()
+    fb.focus_sparse_attn(ctx, b.shape, dev["Q"], s.M, s.N, q_rows, n_rows, max_rows, dev["K"], dev["V"],
+                         fb.HEADS_PER_KV_GROUP, b.block_idx, b.max_blocks, b.block_cnt, b.sink_idx, b.sink_keep,
+                         w.n_sink, b.O, b.lse)
+    assert ctx.poll_status() == fb.ERR_INVALID_ARG
+    assert ctx.poll_status() == 0
+
+
+def test_host_side_argument_matrix(ctx):
+    w = small_workload("f32", 64, 64)
+    s = w.shape
+    _, dev = make_inputs(w)
+    b = fstep.StepBuffers(w)
+    lib = ctx._lib
+    import ctypes as C
+    sh = b.shape
+    st = torch.cuda.current_stream().cuda_stream
+    p = lambda t: t.data_ptr()
+    # k beyond the supported maximum, block range beyond the supported maximum
+    assert lib.focus_select_queries(ctx.handle, p(dev["conf"]), p(dev["masked"]), s.L, 0, s.L, 5000, 8, 0, s.L,
+                                    p(b.focus_idx), p(b.n_focus), p(b.active_idx), p(b.n_active), st) == fb.ERR_UNSUPPORTED
+    assert lib.focus_select_queries(ctx.handle, p(dev["conf"]), p(dev["masked"]), s.L, 5, 3, 4, 8, 0, s.L,
+                                    p(b.focus_idx), p(b.n_focus), p(b.active_idx), p(b.n_active), st) == fb.ERR_INVALID_ARG
+    # C > nb
+    assert lib.focus_select_blocks(ctx.handle, C.byref(sh), p(b.R), 0, s.nb + 1, p(b.sink_idx), w.n_sink, 0,
+                                   p(b.block_idx), s.nb + 1, p(b.block_cnt), p(b.sink_keep), st) == fb.ERR_INVALID_ARG
+    # both / neither of K and Kbar
+    assert lib.focus_score_blocks(ctx.handle, C.byref(sh), p(dev["Q"]), s.M, p(b.focus_idx), p(b.n_focus), w.k,
+                                  None, None, 0, p(b.R), st) == fb.ERR_INVALID_ARG
+    # head_dim the kernels are not built for
+    bad = fb.make_shape(s.L, s.M, 4, 4, 96, 64, fb.F32)
+    assert lib.focus_dense_attn(ctx.handle, C.byref(bad), p(dev["Q"]), s.M, s.N, None, None, 0, p(dev["K"]),
+                                p(dev["V"]), p(b.O), None, st) == fb.ERR_UNSUPPORTED
+    # workspace too small is reported, not overrun
+    tiny = fb.Context(0, workspace_bytes=4096)
+    assert tiny._lib.focus_find_sinks(tiny.handle, C.byref(sh), p(dev["Q"]), s.M, p(b.active_idx), p(b.n_active),
+                                      b.max_active, p(dev["K"]), None, w.n_sink, 0, s.M, p(b.sink_idx), None,
+                                      st) == fb.ERR_WORKSPACE_TOO_SMALL
+    tiny.close()
+
+
+def test_results_are_deterministic(ctx):
+    w = small_workload("bf16", 128, 128, H=8, Hkv=2)
+    host, dev = make_inputs(w)
+    outs = []
+    for _ in range(2):
+        b = fstep.StepBuffers(w)
+        fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
+        fstep.dense_layer(ctx, b, dev["Q"], dev["K"], dev["V"])
+        fstep.find_sinks(ctx, b, dev["Q"], dev["K"], b.lse)
+        fstep.sparse_layer(ctx, b, dev["Q"], dev["K"], dev["V"])
+        torch.cuda.synchronize()
+        outs.append([t.clone() for t in (b.sink_idx, b.sink_scores, b.R, b.block_idx, b.O.view(torch.int16), b.lse)])
+    for a, c in zip(*outs):
+        assert torch.equal(a, c)
