@@ -1,8 +1,577 @@
-// placeholder until the tensor-core kernels land
-#include "focus_common.cuh"
-bool attn_tc_supported(const focus_ctx*, const AttnArgs&) { return false; }
-focus_status launch_attn_tc(focus_ctx*, const AttnArgs&, cudaStream_t) { return FOCUS_ERR_UNSUPPORTED; }
-size_t attn_tc_workspace(const focus_shape*, int, int, int) { return 0; }
+// Block-sparse / dense bidirectional attention on the 5th-generation tensor cores (Eq. 9; FullAttn of
+// Algorithm 1).  bf16 inputs, head_dim 128, fp32 accumulation in TMEM.
+//
+// One CTA = one 128-row query tile of one KV head (GQA: the rows of all query heads of the group are
+// stacked, so every K/V tile is read once per group) x one contiguous range ("split") of that head's key
+// tiles.  Key tiles are 128 keys wide and are enumerated on the fly from the selected block list, the
+// gathered sink tokens and the response region; K/V tiles arrive by TMA through a six-slot ring.
+//
+// Warp roles (192 threads):
+//   warp 0        TMA producer (one lane): K_j, V_{j-1}, K_{j+1}, ... in the order the MMA warp consumes them
+//   warp 1        tcgen05.mma issuer (one lane) + TMEM allocation: S_b = Q K_j^T (b = j mod 2), O += P_j V_j
+//   warps 2..5    online softmax, one query row per thread: S_b -> registers, exp2, bf16 P back into TMEM
+//                 (aliasing S_b), lazy rescale of O, final normalisation and the epilogue
+// Split partials (unnormalised O, running max, running sum) go to scratch and are merged by a second kernel in
+// fixed split order, so results are deterministic.
+#include "tc_common.cuh"
+
+using namespace tc;
+
+namespace {
+
+constexpr int TM = 128;            // query rows per CTA
+constexpr int TN = 128;            // keys per tile
+constexpr int HD = 128;            // head dim
+constexpr int NSLOT = 6;           // K/V ring slots
+constexpr int SLOT_BYTES = TN * HD * 2;
+constexpr int HALF_BYTES = SLOT_BYTES / 2;     // one 64-wide half of a tile: 128 rows x 128 bytes
+constexpr int Q_BYTES = TM * HD * 2;
+constexpr int NBAR = 2 * NSLOT + 5;
+constexpr int SMEM_BYTES = 1024 + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8 + 64;
+constexpr int NTHREADS = 192;
+constexpr float RESCALE_THRESHOLD = 8.0f;      // log2 units: O is rescaled only when the row max grew by more
+
+struct TcParams {
+  const __nv_bfloat16* Q;
+  __nv_bfloat16* O;
+  float* lse;
+  const int32_t* q_rows;
+  const int32_t* n_rows;
+  const int32_t* block_idx;
+  const int32_t* block_cnt;
+  const uint8_t* sink_mask;    // [Hkv][ns_pad]: 1 = attend this gathered sink column
+  float* part_O;               // [cta][128][128] unnormalised partial outputs (n_splits > 1)
+  float* part_ml;              // [cta][128][2] running max (log2 domain) and running sum
+  long long q_stride_row, q_stride_head;
+  int q_base, n_q, rows_bound, L, M, H, Hkv, hpg, B, nb, dense, group_stride, max_blocks, n_sink, ns_pad;
+  int n_mtiles, n_splits, lse_stride;
+  float scale_log2;            // softmax scale * log2(e)
+  int32_t* status;
+};
+
+struct TileInfo {
+  int kind;     // 0: tile of the K/V tensors, 1: tile of the gathered sink rows
+  int start;    // first key row of the tile in its tensor
+  int nvalid;   // leading columns that are real keys (the rest is masked out)
+};
+
+struct TileEnum {
+  int n_blk, n_sinkt, n_resp, total;
+  const int32_t* blocks;
+};
+
+__device__ __forceinline__ TileEnum make_enum(const TcParams& p, int g) {
+  TileEnum e;
+  if (p.dense) {
+    e.n_blk = 0; e.n_sinkt = 0; e.n_resp = (p.L + TN - 1) / TN; e.blocks = nullptr;
+  } else {
+    const int row = g * p.group_stride;
+    e.n_blk = min(max(p.block_cnt[row], 0), p.max_blocks);
+    e.n_sinkt = p.ns_pad / TN;
+    e.n_resp = (p.L - p.M + TN - 1) / TN;
+    e.blocks = p.block_idx + (size_t)row * p.max_blocks;
+  }
+  e.total = e.n_blk + e.n_sinkt + e.n_resp;
+  return e;
+}
+
+__device__ __forceinline__ TileInfo tile_info(const TcParams& p, const TileEnum& e, int t) {
+  TileInfo ti;
+  if (p.dense) {
+    ti.kind = 0; ti.start = t * TN; ti.nvalid = min(TN, p.L - ti.start);
+  } else if (t < e.n_blk) {
+    const int b = e.blocks[t];
+    ti.kind = 0;
+    if (b < 0 || b >= p.nb) {               // reported once by the producer; the tile is fully masked
+      ti.start = 0; ti.nvalid = 0;
+    } else {
+      ti.start = b * p.B; ti.nvalid = min(p.B, p.M - ti.start);
+    }
+  } else if (t < e.n_blk + e.n_sinkt) {
+    const int s = t - e.n_blk;
+    ti.kind = 1; ti.start = s * TN; ti.nvalid = min(TN, p.n_sink - s * TN);
+  } else {
+    const int r = t - e.n_blk - e.n_sinkt;
+    ti.kind = 0; ti.start = p.M + r * TN; ti.nvalid = min(TN, p.L - ti.start);
+  }
+  return ti;
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+               const __grid_constant__ CUtensorMap tmSK, const __grid_constant__ CUtensorMap tmSV, const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
+
+  const int nrows = p.q_rows ? min(max(*p.n_rows, 0), p.rows_bound) : p.n_q;
+  const int total_fr = nrows * p.hpg;                    // stacked (row, head-of-group) rows of this KV head
+  if (mt * TM >= total_fr) return;                       // uniform: nothing to compute for this tile
+
+  const TileEnum te = make_enum(p, g);
+  const int t0 = (int)(((long long)te.total * split) / p.n_splits);
+  const int t1 = (int)(((long long)te.total * (split + 1)) / p.n_splits);
+  const int nt = t1 - t0;
+  const int cta_lin = blockIdx.x * p.n_splits + split;
+
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sptr = smem_raw + (sbase - smem_u32(smem_raw));
+  const uint32_t sQ = sbase;
+  const uint32_t sSlot = sbase + Q_BYTES;
+  const uint32_t sBar = sSlot + NSLOT * SLOT_BYTES;
+  auto bar_full = [&](int s) { return sBar + 8u * s; };
+  auto bar_empty = [&](int s) { return sBar + 8u * (NSLOT + s); };
+  auto bar_sfull = [&](int b) { return sBar + 8u * (2 * NSLOT + b); };
+  auto bar_pready = [&](int b) { return sBar + 8u * (2 * NSLOT + 2 + b); };
+  const uint32_t bar_pvdone = sBar + 8u * (2 * NSLOT + 4);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(sptr + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+
+  if (nt <= 0) {                                          // empty split: publish a neutral partial
+    if (p.n_splits > 1 && warp >= 2) {
+      const int row = (warp & 3) * 32 + lane;
+      p.part_ml[((size_t)cta_lin * TM + row) * 2 + 0] = -INFINITY;
+      p.part_ml[((size_t)cta_lin * TM + row) * 2 + 1] = 0.f;
+    }
+    return;
+  }
+
+  // ---- set-up -------------------------------------------------------------------------------------
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < NSLOT; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pready(b), 128); }
+    mbar_init(bar_pvdone, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+    prefetch_tmap(&tmK); prefetch_tmap(&tmV);
+    if (!p.dense && p.ns_pad > 0) { prefetch_tmap(&tmSK); prefetch_tmap(&tmSV); }
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_holder), 512);
+    tmem_relinquish();
+  }
+  // Q tile -> shared memory in the 128-byte-swizzled K-major layout the MMA descriptor expects:
+  // half h (columns 64h..64h+63) at h*16 KB, row r at r*128 bytes, 16-byte chunk c at ((c ^ (r & 7)) * 16).
+  for (int idx = threadIdx.x; idx < TM * 16; idx += NTHREADS) {
+    const int r = idx >> 4, c = idx & 15;
+    const int fr = mt * TM + r;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (fr < total_fr) {
+      const int qr = fr / p.hpg, hh = fr % p.hpg;
+      const int pos = p.q_rows ? p.q_rows[qr] : p.q_base + qr;
+      if (pos >= p.q_base && pos < p.q_base + p.n_q) {
+        const __nv_bfloat16* src = p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
+                                   (long long)(g * p.hpg + hh) * p.q_stride_head + c * 8;
+        v = __ldg(reinterpret_cast<const uint4*>(src));
+      } else if (c == 0) {
+        set_status(p.status, FOCUS_ERR_INVALID_ARG);
+      }
+    }
+    const int half = c >> 3, cc = c & 7;
+    *reinterpret_cast<uint4*>(sptr + half * HALF_BYTES + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+  }
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_holder;
+  const uint32_t tmem_O = tmem + 256;
+
+  if (warp == 0) {
+    // ================================ TMA producer ================================================
+    if (lane == 0) {
+      uint32_t q = 0;
+      int issued = 0;
+      auto load = [&](int t, bool isV) -> bool {
+        const int slot = q % NSLOT;
+        const uint32_t ph = (q / NSLOT) & 1u;
+        if (!mbar_wait(bar_empty(slot), ph ^ 1u, abort_flag, p.status)) return false;
+        const TileInfo ti = tile_info(p, te, t);
+        if (!p.dense && !isV && t < te.n_blk) {
+          const int b = te.blocks[t];
+          if (b < 0 || b >= p.nb) set_status(p.status, FOCUS_ERR_INVALID_ARG);
+        }
+        const CUtensorMap* map = ti.kind ? (isV ? &tmSV : &tmSK) : (isV ? &tmV : &tmK);
+        const uint32_t dst = sSlot + slot * SLOT_BYTES;
+        mbar_expect_tx(bar_full(slot), SLOT_BYTES);
+        tma_load_3d(dst, map, bar_full(slot), 0, ti.start, g);
+        tma_load_3d(dst + HALF_BYTES, map, bar_full(slot), 64, ti.start, g);
+        ++q; ++issued;
+        return true;
+      };
+      bool ok = true;
+      for (int j = t0; j < t1 && ok; ++j) {
+        ok = load(j, false);
+        if (ok && j > t0) ok = load(j - 1, true);
+      }
+      if (ok) ok = load(t1 - 1, true);
+      if (!ok) {
+        // unwinding: let the copies already issued land before the CTA's shared memory is released
+        const uint32_t first = issued > NSLOT ? (uint32_t)(issued - NSLOT) : 0u;
+        for (uint32_t i = first; i < (uint32_t)issued; ++i) {
+          uint64_t t_start = global_ns();
+          while (!mbar_try_wait(bar_full(i % NSLOT), (i / NSLOT) & 1u)) {
+            if (global_ns() - t_start > WAIT_LIMIT_NS) break;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ================================ MMA issuer ==================================================
+    if (lane == 0) {
+      constexpr uint32_t IDESC_QK = make_idesc(TM, TN, 0);
+      constexpr uint32_t IDESC_PV = make_idesc(TM, HD, 1);
+      const uint64_t qdesc = make_sdesc(sQ, 16, 1024);
+      uint32_t q = 0;
+      bool ok = true;
+      auto do_pv = [&](int idx) -> bool {
+        const int b = idx & 1;
+        if (!mbar_wait(bar_pready(b), (uint32_t)(idx >> 1) & 1u, abort_flag, p.status)) return false;
+        const int slot = q % NSLOT;
+        if (!mbar_wait(bar_full(slot), (q / NSLOT) & 1u, abort_flag, p.status)) return false;
+        tc_fence_after();
+        const uint64_t vdesc = make_sdesc(sSlot + slot * SLOT_BYTES, HALF_BYTES, 1024);
+        const uint32_t pt = tmem + b * 128;
+#pragma unroll
+        for (int ks = 0; ks < TN / 16; ++ks)
+          mma_ts(tmem_O, pt + ks * 8, vdesc + (uint64_t)(ks * (2048 >> 4)), IDESC_PV, (idx > 0 || ks > 0) ? 1u : 0u);
+        tc_commit(bar_empty(slot));
+        tc_commit(bar_pvdone);
+        ++q;
+        return true;
+      };
+      for (int idx = 0; idx < nt && ok; ++idx) {
+        const int b = idx & 1;
+        const int slot = q % NSLOT;
+        if (!mbar_wait(bar_full(slot), (q / NSLOT) & 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint64_t kdesc = make_sdesc(sSlot + slot * SLOT_BYTES, 16, 1024);
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t off = (uint64_t)((half * HALF_BYTES + ks * 32) >> 4);
+            mma_ss(tmem + b * 128, qdesc + off, kdesc + off, IDESC_QK, (half | ks) ? 1u : 0u);
+          }
+        tc_commit(bar_empty(slot));
+        tc_commit(bar_sfull(b));
+        ++q;
+        if (idx > 0) ok = do_pv(idx - 1);
+      }
+      if (ok) ok = do_pv(nt - 1);
+    }
+  } else {
+    // ================================ softmax / epilogue ==========================================
+    const int rq = warp & 3;                         // TMEM lane quarter this warp may access
+    const int row = rq * 32 + lane;                  // query row of this thread inside the tile
+    const uint32_t lane_off = (uint32_t)(rq * 32) << 16;
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int idx = 0; idx < nt; ++idx) {
+      const int b = idx & 1;
+      // votes keep the warp together: the TMEM loads and stores below are warp-collective
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(b), (uint32_t)(idx >> 1) & 1u, abort_flag, p.status))) { ok = false; break; }
+      tc_fence_after();
+      uint32_t sreg[128];
+      const uint32_t ts = tmem + lane_off + b * 128;
+      TC_LD32(ts, (sreg + 0));
+      TC_LD32(ts + 32, (sreg + 32));
+      TC_LD32(ts + 64, (sreg + 64));
+      TC_LD32(ts + 96, (sreg + 96));
+      tc_wait_ld();
+      const TileInfo ti = tile_info(p, te, t0 + idx);
+      float tmax = -INFINITY;
+      if (ti.kind == 0 && ti.nvalid == TN) {
+#pragma unroll
+        for (int c = 0; c < 128; ++c) tmax = fmaxf(tmax, __uint_as_float(sreg[c]));
+      } else if (ti.kind == 0) {
+#pragma unroll
+        for (int c = 0; c < 128; ++c) {
+          const float v = c < ti.nvalid ? __uint_as_float(sreg[c]) : -INFINITY;
+          sreg[c] = __float_as_uint(v);
+          tmax = fmaxf(tmax, v);
+        }
+      } else {
+        const uint32_t* mk = reinterpret_cast<const uint32_t*>(p.sink_mask + (size_t)g * p.ns_pad + ti.start);
+#pragma unroll
+        for (int c4 = 0; c4 < 32; ++c4) {
+          const uint32_t mword = __ldg(mk + c4);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int c = c4 * 4 + e;
+            const float v = ((mword >> (8 * e)) & 0xffu) ? __uint_as_float(sreg[c]) : -INFINITY;
+            sreg[c] = __float_as_uint(v);
+            tmax = fmaxf(tmax, v);
+          }
+        }
+      }
+      tmax *= p.scale_log2;                          // scale > 0: max commutes with the scaling
+      float alpha = 1.f;
+      bool rescale = false;
+      if (tmax > m_ref + RESCALE_THRESHOLD) {        // also true for the first finite maximum (m_ref = -inf)
+        if (m_ref != -INFINITY) {
+          alpha = ex2(m_ref - tmax);
+          rescale = true;
+        }
+        m_ref = tmax;
+      }
+      // p = 2^(s*scale_log2 - m_ref); a fully masked row so far (m_ref = -inf) contributes zeros
+      const float mneg = m_ref == -INFINITY ? 0.f : -m_ref;
+      uint32_t preg[64];
+      float lsum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 64; ++c) {
+        const float p0 = ex2(fmaf(__uint_as_float(sreg[2 * c]), p.scale_log2, mneg));
+        const float p1 = ex2(fmaf(__uint_as_float(sreg[2 * c + 1]), p.scale_log2, mneg));
+        lsum += p0 + p1;
+        preg[c] = pack_bf16(p0, p1);
+      }
+      l = l * alpha + lsum;
+      if (idx > 0) {
+        // P_{idx-1} V_{idx-1} must have left the tensor core before O is touched; waiting for every phase in
+        // order also keeps the parity of this barrier unambiguous
+        if (!__all_sync(0xffffffffu, mbar_wait(bar_pvdone, (uint32_t)(idx - 1) & 1u, abort_flag, p.status))) { ok = false; break; }
+        if (__any_sync(0xffffffffu, rescale)) {   // tcgen05.ld/st are warp-collective: the whole warp takes the branch
+          tc_fence_after();
+#pragma unroll
+          for (int cb = 0; cb < 4; ++cb) {
+            uint32_t oreg[32];
+            TC_LD32(tmem_O + lane_off + cb * 32, oreg);
+            tc_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * alpha);
+            TC_ST32(tmem_O + lane_off + cb * 32, oreg);
+          }
+        }
+      }
+      TC_ST32(ts, (preg + 0));
+      TC_ST32(ts + 32, (preg + 32));
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_pready(b));
+    }
+    // ---- epilogue: wait for the last P V, normalise, write out -----------------------------------
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_pvdone, (uint32_t)(nt - 1) & 1u, abort_flag, p.status));
+    if (ok) {
+      tc_fence_after();
+      const int fr = mt * TM + row;
+      const bool valid = fr < total_fr;
+      if (p.n_splits == 1) {
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        const int qr = valid ? fr / p.hpg : 0, hh = valid ? fr % p.hpg : 0;
+        __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD;
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t oreg[32];
+          TC_LD32(tmem_O + lane_off + cb * 32, oreg);
+          tc_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int c = 0; c < 32; c += 8) {
+              uint4 v;
+              v.x = pack_bf16(__uint_as_float(oreg[c + 0]) * inv, __uint_as_float(oreg[c + 1]) * inv);
+              v.y = pack_bf16(__uint_as_float(oreg[c + 2]) * inv, __uint_as_float(oreg[c + 3]) * inv);
+              v.z = pack_bf16(__uint_as_float(oreg[c + 4]) * inv, __uint_as_float(oreg[c + 5]) * inv);
+              v.w = pack_bf16(__uint_as_float(oreg[c + 6]) * inv, __uint_as_float(oreg[c + 7]) * inv);
+              *reinterpret_cast<uint4*>(orow + cb * 32 + c) = v;
+            }
+          }
+        }
+        if (valid && p.lse)
+          p.lse[(size_t)(g * p.hpg + hh) * p.lse_stride + qr] = (m_ref + log2f(l)) * 0.6931471805599453f;
+      } else {
+        float* po = p.part_O + ((size_t)cta_lin * TM + row) * HD;
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t oreg[32];
+          TC_LD32(tmem_O + lane_off + cb * 32, oreg);
+          tc_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; c += 4)
+            *reinterpret_cast<uint4*>(po + cb * 32 + c) = make_uint4(oreg[c], oreg[c + 1], oreg[c + 2], oreg[c + 3]);
+        }
+        p.part_ml[((size_t)cta_lin * TM + row) * 2 + 0] = m_ref;
+        p.part_ml[((size_t)cta_lin * TM + row) * 2 + 1] = l;
+      }
+    }
+  }
+  // ---- teardown: every role converges here, also after a timed-out wait --------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+// Merge of the split partials: out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s, one warp per stacked row.
+__global__ void __launch_bounds__(256)
+attn_combine_kernel(const float* __restrict__ part_O, const float* __restrict__ part_ml, int n_splits, int n_mtiles,
+                    int hpg, int H, const int32_t* q_rows, const int32_t* n_rows, int rows_bound, int n_q,
+                    __nv_bfloat16* __restrict__ O, float* __restrict__ lse, int lse_stride) {
+  const int lane = threadIdx.x & 31;
+  const int wrow = blockIdx.x * 8 + (threadIdx.x >> 5);        // global stacked-row slot: tile * 128 + row
+  const int tile = wrow / TM, row = wrow % TM;
+  const int g = tile / n_mtiles, mt = tile % n_mtiles;
+  const int nrows = q_rows ? min(max(*n_rows, 0), rows_bound) : n_q;
+  const int fr = mt * TM + row;
+  if (fr >= nrows * hpg) return;
+  float m = -INFINITY;
+  for (int s = 0; s < n_splits; ++s) {
+    const float* ml = part_ml + ((size_t)(tile * n_splits + s) * TM + row) * 2;
+    if (ml[1] > 0.f) m = fmaxf(m, ml[0]);
+  }
+  float tot = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < n_splits; ++s) {
+    const size_t base = (size_t)(tile * n_splits + s) * TM + row;
+    const float ls = part_ml[base * 2 + 1];
+    if (!(ls > 0.f)) continue;
+    const float wgt = exp2f(part_ml[base * 2] - m);
+    tot += wgt * ls;
+    const float4 o = *reinterpret_cast<const float4*>(part_O + base * HD + lane * 4);
+    acc.x += wgt * o.x; acc.y += wgt * o.y; acc.z += wgt * o.z; acc.w += wgt * o.w;
+  }
+  const float inv = tot > 0.f ? 1.f / tot : 0.f;
+  const int qr = fr / hpg, hh = fr % hpg;
+  __nv_bfloat16* orow = O + ((size_t)qr * H + (size_t)(g * hpg + hh)) * HD + lane * 4;
+  uint2 v;
+  v.x = pack_bf16(acc.x * inv, acc.y * inv);
+  v.y = pack_bf16(acc.z * inv, acc.w * inv);
+  *reinterpret_cast<uint2*>(orow) = v;
+  if (lse && lane == 0) lse[(size_t)(g * hpg + hh) * lse_stride + qr] = (m + log2f(tot)) * 0.6931471805599453f;
+}
+
+// Gathers the sink tokens' K and V rows into compact, zero-padded per-KV-head tiles and builds the
+// column mask: attend column s iff the token is kept for this head's group, is valid and is a prompt token
+// (response tokens are attended through the response tiles; every key is counted once).
+__global__ void __launch_bounds__(256)
+sink_gather_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V, long long kv_stride_tok,
+                   long long kv_stride_head, const int32_t* __restrict__ sink_idx, const uint8_t* __restrict__ sink_keep,
+                   int n_sink, int ns_pad, int group_stride, int M, int L, __nv_bfloat16* __restrict__ gK,
+                   __nv_bfloat16* __restrict__ gV, uint8_t* __restrict__ mask, int32_t* status) {
+  const int g = blockIdx.y;
+  const int s = blockIdx.x * 16 + (threadIdx.x >> 4), c = threadIdx.x & 15;
+  if (s >= ns_pad) return;
+  uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
+  uint8_t mk = 0;
+  if (s < n_sink) {
+    const int j = sink_idx[s];
+    if (j < 0 || j >= L) {
+      if (c == 0) set_status(status, FOCUS_ERR_INVALID_ARG);
+    } else {
+      const size_t off = (size_t)g * kv_stride_head + (size_t)j * kv_stride_tok + c * 8;
+      kv = __ldg(reinterpret_cast<const uint4*>(K + off));
+      vv = __ldg(reinterpret_cast<const uint4*>(V + off));
+      mk = (j < M && sink_keep[(size_t)g * group_stride * n_sink + s]) ? 1 : 0;
+    }
+  }
+  const size_t o = ((size_t)g * ns_pad + s) * HD + c * 8;
+  *reinterpret_cast<uint4*>(gK + o) = kv;
+  *reinterpret_cast<uint4*>(gV + o) = vv;
+  if (c == 0) mask[(size_t)g * ns_pad + s] = mk;
+}
+
+int pick_splits(const focus_ctx* ctx, int base_ctas, int max_tiles) {
+  int s = ctx->sm_count / (base_ctas > 0 ? base_ctas : 1);
+  if (s < 1) s = 1;
+  const int cap = max_tiles / 2 > 1 ? max_tiles / 2 : 1;
+  return s < cap ? s : cap;
+}
+
+}  // namespace
+
+bool attn_tc_supported(const focus_ctx* ctx, const AttnArgs& a) {
+  return ctx->encode_tiled != nullptr && a.sh.dtype == FOCUS_BF16 && a.sh.head_dim == HD && a.O != nullptr &&
+         (a.sh.n_q_heads / a.sh.n_kv_heads) <= TM && a.sh.L >= 1;
+}
+
+size_t attn_tc_workspace(const focus_shape* s, int n_q, int max_blocks, int n_sink) {
+  const size_t ns_pad = ((size_t)n_sink + TN - 1) / TN * TN;
+  const size_t gather = 2 * (size_t)s->n_kv_heads * ns_pad * HD * 2 + (size_t)s->n_kv_heads * ns_pad + 1024;
+  const int hpg = s->n_q_heads / s->n_kv_heads;
+  const size_t mtiles = ((size_t)n_q * hpg + TM - 1) / TM;
+  const size_t ctas = mtiles * s->n_kv_heads;
+  const size_t part = (ctas < 160 ? 320 : ctas) * ((size_t)TM * HD * 4 + TM * 8) + 1024;
+  return gather + part;
+}
+
+focus_status launch_attn_tc(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st) {
+  const focus_shape& sh = a.sh;
+  const int Hkv = sh.n_kv_heads, hpg = sh.n_q_heads / Hkv;
+  const int n_mtiles = (int)(((long long)a.max_rows * hpg + TM - 1) / TM);
+  if (n_mtiles == 0) return FOCUS_OK;
+  const int base = n_mtiles * Hkv;
+  const int ns_pad = a.dense ? 0 : (a.n_sink + TN - 1) / TN * TN;
+  const int n_resp = a.dense ? (sh.L + TN - 1) / TN : (sh.L - sh.M + TN - 1) / TN;
+  const int max_tiles = a.dense ? n_resp : a.max_blocks + ns_pad / TN + n_resp;
+  const int n_splits = pick_splits(ctx, base, max_tiles);
+
+  WsAlloc ws(ctx);
+  __nv_bfloat16* gK = nullptr; __nv_bfloat16* gV = nullptr; uint8_t* mask = nullptr;
+  if (ns_pad > 0) {
+    gK = ws.get<__nv_bfloat16>((size_t)Hkv * ns_pad * HD);
+    gV = ws.get<__nv_bfloat16>((size_t)Hkv * ns_pad * HD);
+    mask = ws.get<uint8_t>((size_t)Hkv * ns_pad);
+  }
+  float* part_O = nullptr; float* part_ml = nullptr;
+  if (n_splits > 1) {
+    part_O = ws.get<float>((size_t)base * n_splits * TM * HD);
+    part_ml = ws.get<float>((size_t)base * n_splits * TM * 2);
+  }
+  if (!ws.ok) return FOCUS_ERR_WORKSPACE_TOO_SMALL;
+
+  CUtensorMap tmK, tmV, tmSK, tmSV;
+  if (!encode_kv_map(ctx->encode_tiled, &tmK, a.K, HD, sh.L, Hkv, sh.kv_stride_tok, sh.kv_stride_head, 64, TN) ||
+      !encode_kv_map(ctx->encode_tiled, &tmV, a.V, HD, sh.L, Hkv, sh.kv_stride_tok, sh.kv_stride_head, 64, TN))
+    return FOCUS_ERR_INVALID_ARG;
+  if (ns_pad > 0) {
+    if (!encode_kv_map(ctx->encode_tiled, &tmSK, gK, HD, ns_pad, Hkv, HD, (long long)ns_pad * HD, 64, TN) ||
+        !encode_kv_map(ctx->encode_tiled, &tmSV, gV, HD, ns_pad, Hkv, HD, (long long)ns_pad * HD, 64, TN))
+      return FOCUS_ERR_CUDA;
+    dim3 gg((ns_pad + 15) / 16, Hkv);
+    sink_gather_kernel<<<gg, 256, 0, st>>>((const __nv_bfloat16*)a.K, (const __nv_bfloat16*)a.V, sh.kv_stride_tok,
+                                           sh.kv_stride_head, a.sink_idx, a.sink_keep, a.n_sink, ns_pad,
+                                           a.group_stride, sh.M, sh.L, gK, gV, mask, ctx->d_status);
+    FOCUS_CHECK_LAUNCH();
+  } else {
+    tmSK = tmK; tmSV = tmV;
+  }
+
+  TcParams p;
+  p.Q = (const __nv_bfloat16*)a.Q; p.O = (__nv_bfloat16*)a.O; p.lse = a.lse;
+  p.q_rows = a.q_rows; p.n_rows = a.n_rows; p.block_idx = a.block_idx; p.block_cnt = a.block_cnt;
+  p.sink_mask = mask; p.part_O = part_O; p.part_ml = part_ml;
+  p.q_stride_row = sh.q_stride_row; p.q_stride_head = sh.q_stride_head;
+  p.q_base = a.q_base; p.n_q = a.n_q; p.rows_bound = a.max_rows; p.L = sh.L; p.M = sh.M; p.H = sh.n_q_heads;
+  p.Hkv = Hkv; p.hpg = hpg; p.B = sh.kv_block; p.nb = shape_nb(&sh); p.dense = a.dense;
+  p.group_stride = a.group_stride; p.max_blocks = a.max_blocks; p.n_sink = a.n_sink; p.ns_pad = ns_pad;
+  p.n_mtiles = n_mtiles; p.n_splits = n_splits; p.lse_stride = a.lse_stride;
+  p.scale_log2 = a.scale * 1.4426950408889634f;
+  p.status = ctx->d_status;
+
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+      return FOCUS_ERR_CUDA;
+    attr_set = true;
+  }
+  attn_tc_kernel<<<dim3(base, n_splits), NTHREADS, SMEM_BYTES, st>>>(tmK, tmV, tmSK, tmSV, p);
+  FOCUS_CHECK_LAUNCH();
+  if (n_splits > 1) {
+    const int rows_total = base * TM;
+    attn_combine_kernel<<<rows_total / 8, 256, 0, st>>>(part_O, part_ml, n_splits, n_mtiles, hpg, sh.n_q_heads,
+                                                        a.q_rows, a.n_rows, a.max_rows, a.n_q,
+                                                        (__nv_bfloat16*)a.O, a.lse, a.lse_stride);
+    FOCUS_CHECK_LAUNCH();
+  }
+  return FOCUS_OK;
+}
+
+// The tensor-core sink column-sum is not built yet: the SIMT kernel serves every shape.
 bool sink_tc_supported(const focus_ctx*, const focus_shape*, int) { return false; }
 focus_status launch_sink_colsum_tc(focus_ctx*, const focus_shape*, const void*, int, const int32_t*, const int32_t*, int,
-                                   const void*, const float*, float*, WsAlloc&, cudaStream_t) { return FOCUS_ERR_UNSUPPORTED; }
+                                   const void*, const float*, float*, WsAlloc&, cudaStream_t) {
+  return FOCUS_ERR_UNSUPPORTED;
+}
