@@ -86,6 +86,9 @@ focus_status focus_workspace_bytes(const focus_shape* shape, int32_t n_q, int32_
 focus_status focus_poll_status(focus_ctx* ctx, focus_stream stream, int32_t* device_status);
 const char* focus_status_string(focus_status s);
 
+/* Number of kernels this library has launched in this process so far (all contexts). */
+uint64_t focus_launch_count(void);
+
 /* Selects the attention implementation for bf16 / head_dim 128 inputs: 0 = automatic (tensor-core
  * kernel where supported), 1 = force the generic SIMT kernels.  Returns the previous value. */
 int32_t focus_set_force_simt(focus_ctx* ctx, int32_t force);

@@ -42,6 +42,7 @@ _SIGS = {
     "focus_poll_status": (_I, [_P, _P, C.POINTER(_I)]),
     "focus_status_string": (C.c_char_p, [_I]),
     "focus_set_force_simt": (_I, [_P, _I]),
+    "focus_launch_count": (C.c_uint64, []),
     "focus_select_queries": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P, _P, _P, _P, _P]),
     "focus_find_sinks": (_I, [_P, _SH, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _P, _P, _P]),
     "focus_pool_keys": (_I, [_P, _SH, _P, _P, _P]),
@@ -134,6 +135,10 @@ class Context:
 
     def set_force_simt(self, force: bool) -> int:
         return self._lib.focus_set_force_simt(self.handle, 1 if force else 0)
+
+
+def focus_launch_count() -> int:
+    return int(load_library().focus_launch_count())
 
 
 def focus_workspace_bytes(shape: focus_shape, n_q: int, max_blocks: int, n_sink: int) -> int:

@@ -568,10 +568,3 @@ focus_status launch_attn_tc(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st) 
   }
   return FOCUS_OK;
 }
-
-// The tensor-core sink column-sum is not built yet: the SIMT kernel serves every shape.
-bool sink_tc_supported(const focus_ctx*, const focus_shape*, int) { return false; }
-focus_status launch_sink_colsum_tc(focus_ctx*, const focus_shape*, const void*, int, const int32_t*, const int32_t*, int,
-                                   const void*, const float*, float*, WsAlloc&, cudaStream_t) {
-  return FOCUS_ERR_UNSUPPORTED;
-}

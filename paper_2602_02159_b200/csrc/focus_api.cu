@@ -16,6 +16,10 @@ focus_status launch_sink_colsum_tc(focus_ctx* ctx, const focus_shape* s, const v
                                    const int32_t* active_idx, const int32_t* n_active, int max_active, const void* K,
                                    const float* lse, float* part, WsAlloc& ws, cudaStream_t st);
 
+unsigned long long g_focus_launches = 0;
+
+extern "C" uint64_t focus_launch_count(void) { return g_focus_launches; }
+
 extern "C" const char* focus_status_string(focus_status s) {
   switch (s) {
     case FOCUS_OK: return "ok";

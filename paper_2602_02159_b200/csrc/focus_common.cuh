@@ -33,8 +33,12 @@ struct WsAlloc {
   }
 };
 
-#define FOCUS_CHECK_LAUNCH()                                   \
-  do {                                                         \
+// Every kernel launch of the library goes through this macro: it counts the launch and maps a failed
+// launch to FOCUS_ERR_CUDA.
+extern unsigned long long g_focus_launches;
+#define FOCUS_CHECK_LAUNCH()                                      \
+  do {                                                            \
+    ++g_focus_launches;                                           \
     if (cudaGetLastError() != cudaSuccess) return FOCUS_ERR_CUDA; \
   } while (0)
 

@@ -1,0 +1,232 @@
+// Attention-sink column sums on the tensor cores (Eq. 6): part[h][j] = sum_i exp(scale * q_i^h . k_j - lse_i^h)
+// over the active query rows i.  bf16 inputs, head_dim 128.
+//
+// The product is taken transposed, S^T = K_tile Q^T, so that TMEM lanes are keys and TMEM columns are query
+// rows: each consumer thread owns one key and adds up its probabilities over the columns serially -- the
+// column sum needs no cross-thread reduction and no second pass over the tile.  K streams once through a TMA
+// ring (this kernel is HBM-bound); the query rows of one KV group stay resident in shared memory.
+//
+// Warp roles (192 threads): warp 0 TMA producer, warp 1 tcgen05.mma issuer + TMEM owner, warps 2..5 consumers.
+#include "tc_common.cuh"
+
+using namespace tc;
+
+namespace {
+
+constexpr int TK = 128;               // keys per tile (MMA M)
+constexpr int HD = 128;
+constexpr int SLOT_BYTES = TK * HD * 2;
+constexpr int HALF_BYTES = SLOT_BYTES / 2;
+constexpr int NTHREADS = 192;
+constexpr int MAX_SLOTS = 6;
+constexpr int MAX_NPAD = 256;
+
+struct SinkParams {
+  const __nv_bfloat16* Q;
+  const int32_t* active_idx;
+  const int32_t* n_active;
+  const float* lse;             // [H][lse_stride], natural log
+  float* part;                  // [H][L]
+  long long q_stride_row, q_stride_head;
+  int q_base, L, hpg, max_active, n_pad, n_slots, lse_stride, chunks;
+  float scale_log2;
+  int32_t* status;
+};
+
+#define TC_LD16(taddr, r)                                                                                         \
+  asm volatile(                                                                                                   \
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"     \
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), \
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])                  \
+      : "r"(taddr)                                                                                                \
+      : "memory")
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = blockIdx.y, chunk = blockIdx.x;
+  const int T = (p.L + TK - 1) / TK;
+  const int t0 = (int)(((long long)T * chunk) / p.chunks), t1 = (int)(((long long)T * (chunk + 1)) / p.chunks);
+  const int nt = t1 - t0;
+  if (nt <= 0) return;
+  const int n = min(max(*p.n_active, 0), p.max_active);
+  const int q_head_bytes = p.n_pad * 256;              // two swizzled halves of n_pad rows x 128 bytes
+  const int q_bytes = p.hpg * q_head_bytes;
+
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sptr = smem_raw + (sbase - smem_u32(smem_raw));
+  const uint32_t sQ = sbase;
+  const uint32_t sSlot = sbase + q_bytes;
+  const uint32_t sBar = sSlot + p.n_slots * SLOT_BYTES;
+  auto bar_full = [&](int s) { return sBar + 8u * s; };
+  auto bar_empty = [&](int s) { return sBar + 8u * (MAX_SLOTS + s); };
+  auto bar_sfull = [&](int b) { return sBar + 8u * (2 * MAX_SLOTS + b); };
+  auto bar_sempty = [&](int b) { return sBar + 8u * (2 * MAX_SLOTS + 2 + b); };
+  uint8_t* tail = sptr + q_bytes + p.n_slots * SLOT_BYTES + (2 * MAX_SLOTS + 4) * 8;
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
+  float* neg_lse2 = reinterpret_cast<float*>(tail + 16);       // [hpg][n_pad]: -lse * log2(e)
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.n_slots; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_sempty(b), 128); }
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+    prefetch_tmap(&tmK);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_holder), 512);
+    tmem_relinquish();
+  }
+  // query rows of every head of the group -> swizzled K-major B operand; rows >= n are zero
+  for (int idx = threadIdx.x; idx < p.hpg * p.n_pad * 16; idx += NTHREADS) {
+    const int c = idx & 15, r = (idx >> 4) % p.n_pad, hh = (idx >> 4) / p.n_pad;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (r < n) {
+      const int pos = p.active_idx[r];
+      if (pos >= p.q_base && pos < p.L) {
+        v = __ldg(reinterpret_cast<const uint4*>(p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
+                                                 (long long)(g * p.hpg + hh) * p.q_stride_head + c * 8));
+      } else if (c == 0) {
+        set_status(p.status, FOCUS_ERR_INVALID_ARG);
+      }
+    }
+    const int half = c >> 3, cc = c & 7;
+    *reinterpret_cast<uint4*>(sptr + hh * q_head_bytes + half * (p.n_pad * 128) + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+  }
+  for (int idx = threadIdx.x; idx < p.hpg * p.n_pad; idx += NTHREADS) {
+    const int r = idx % p.n_pad, hh = idx / p.n_pad;
+    neg_lse2[idx] = r < n ? -p.lse[(size_t)(g * p.hpg + hh) * p.lse_stride + r] * 1.4426950408889634f : 0.f;
+  }
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_holder;
+  const int units = nt * p.hpg;                  // one unit = (key tile, query head of the group)
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int issued = 0;
+      bool ok = true;
+      for (int i = 0; i < nt && ok; ++i) {
+        const int slot = i % p.n_slots;
+        const uint32_t ph = (uint32_t)(i / p.n_slots) & 1u;
+        if (!mbar_wait(bar_empty(slot), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        const uint32_t dst = sSlot + slot * SLOT_BYTES;
+        mbar_expect_tx(bar_full(slot), SLOT_BYTES);
+        tma_load_3d(dst, &tmK, bar_full(slot), 0, (t0 + i) * TK, g);
+        tma_load_3d(dst + HALF_BYTES, &tmK, bar_full(slot), 64, (t0 + i) * TK, g);
+        ++issued;
+      }
+      if (!ok) {
+        const int first = issued > p.n_slots ? issued - p.n_slots : 0;
+        for (int i = first; i < issued; ++i) {
+          const uint64_t t_start = global_ns();
+          while (!mbar_try_wait(bar_full(i % p.n_slots), (uint32_t)(i / p.n_slots) & 1u))
+            if (global_ns() - t_start > WAIT_LIMIT_NS) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(TK, p.n_pad, 0);
+      bool ok = true;
+      for (int u = 0; u < units && ok; ++u) {
+        const int i = u / p.hpg, hh = u % p.hpg;
+        const int slot = i % p.n_slots, b = u & 1;
+        if (!mbar_wait(bar_sempty(b), ((uint32_t)(u >> 1) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        if (hh == 0 && !mbar_wait(bar_full(slot), (uint32_t)(i / p.n_slots) & 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint64_t kdesc = make_sdesc(sSlot + slot * SLOT_BYTES, 16, 1024);
+        const uint64_t qdesc = make_sdesc(sQ + hh * q_head_bytes, 16, 1024);
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            mma_ss(tmem + b * 256, kdesc + (uint64_t)((half * HALF_BYTES + ks * 32) >> 4),
+                   qdesc + (uint64_t)((half * (p.n_pad * 128) + ks * 32) >> 4), idesc, (half | ks) ? 1u : 0u);
+        tc_commit(bar_sfull(b));
+        if (hh == p.hpg - 1) tc_commit(bar_empty(slot));
+      }
+    }
+  } else {
+    const int rq = warp & 3;
+    const int krow = rq * 32 + lane;                          // key of this thread inside the tile
+    const uint32_t lane_off = (uint32_t)(rq * 32) << 16;
+    for (int u = 0; u < units; ++u) {
+      const int i = u / p.hpg, hh = u % p.hpg, b = u & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(b), (uint32_t)(u >> 1) & 1u, abort_flag, p.status))) break;
+      tc_fence_after();
+      const float* nl = neg_lse2 + hh * p.n_pad;
+      float acc = 0.f;
+      for (int c0 = 0; c0 < n; c0 += 16) {
+        uint32_t r[16];
+        TC_LD16(tmem + lane_off + b * 256 + c0, r);
+        tc_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+          if (c0 + c < n) acc += ex2(fmaf(__uint_as_float(r[c]), p.scale_log2, nl[c0 + c]));
+      }
+      tc_fence_before();
+      mbar_arrive(bar_sempty(b));
+      const int key = (t0 + i) * TK + krow;
+      if (key < p.L) p.part[(size_t)(g * p.hpg + hh) * p.L + key] = acc;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+}  // namespace
+
+static int sink_npad(int max_active) { return (max_active + 15) / 16 * 16; }
+static int sink_slots(int hpg, int n_pad) {
+  const int fixed = 1024 + hpg * n_pad * 256 + (2 * MAX_SLOTS + 4) * 8 + 16 + hpg * n_pad * 4 + 64;
+  int s = (232448 - fixed) / SLOT_BYTES;
+  return s > MAX_SLOTS ? MAX_SLOTS : s;
+}
+
+bool sink_tc_supported(const focus_ctx* ctx, const focus_shape* s, int max_active) {
+  if (!ctx->encode_tiled || s->dtype != FOCUS_BF16 || s->head_dim != HD) return false;
+  const int n_pad = sink_npad(max_active), hpg = s->n_q_heads / s->n_kv_heads;
+  return n_pad <= MAX_NPAD && sink_slots(hpg, n_pad) >= 2;
+}
+
+focus_status launch_sink_colsum_tc(focus_ctx* ctx, const focus_shape* s, const void* Q, int q_base,
+                                   const int32_t* active_idx, const int32_t* n_active, int max_active, const void* K,
+                                   const float* lse, float* part, WsAlloc&, cudaStream_t st) {
+  const int Hkv = s->n_kv_heads, hpg = s->n_q_heads / Hkv;
+  SinkParams p;
+  p.Q = (const __nv_bfloat16*)Q; p.active_idx = active_idx; p.n_active = n_active; p.lse = lse; p.part = part;
+  p.q_stride_row = s->q_stride_row; p.q_stride_head = s->q_stride_head;
+  p.q_base = q_base; p.L = s->L; p.hpg = hpg; p.max_active = max_active; p.n_pad = sink_npad(max_active);
+  p.n_slots = sink_slots(hpg, p.n_pad); p.lse_stride = max_active;
+  const int T = (s->L + TK - 1) / TK;
+  int chunks = ctx->sm_count / Hkv;
+  if (chunks < 1) chunks = 1;
+  if (chunks > T) chunks = T;
+  p.chunks = chunks;
+  p.scale_log2 = shape_scale(s) * 1.4426950408889634f;
+  p.status = ctx->d_status;
+  CUtensorMap tmK;
+  if (!encode_kv_map(ctx->encode_tiled, &tmK, K, HD, s->L, Hkv, s->kv_stride_tok, s->kv_stride_head, 64, TK))
+    return FOCUS_ERR_INVALID_ARG;
+  const int smem = 1024 + hpg * p.n_pad * 256 + p.n_slots * SLOT_BYTES + (2 * MAX_SLOTS + 4) * 8 + 16 +
+                   hpg * p.n_pad * 4 + 64;
+  static int attr_smem = 0;
+  if (smem > attr_smem) {
+    if (cudaFuncSetAttribute(sink_colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+      return FOCUS_ERR_CUDA;
+    attr_smem = smem;
+  }
+  sink_colsum_tc_kernel<<<dim3(chunks, Hkv), NTHREADS, smem, st>>>(tmK, p);
+  FOCUS_CHECK_LAUNCH();
+  return FOCUS_OK;
+}
