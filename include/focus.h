@@ -172,6 +172,18 @@ focus_status focus_sparse_attn(focus_ctx* ctx, const focus_shape* shape, const v
                                const int32_t* sink_idx, const uint8_t* sink_keep, int32_t n_sink,
                                void* O, float* lse, focus_stream stream);
 
+/* One whole sparse layer (Algorithm 1, sparse branch) in one call, for the default modes (one block set per
+ * KV head, sinks as tokens) with cached pooled keys: block relevance (Eq. 7) -> Top-C (Eq. 8) -> sparse
+ * attention (Eq. 9).  Same results as focus_score_blocks(Kbar) + focus_select_blocks + focus_sparse_attn with
+ * max_blocks = C, in fewer kernel launches.  Outputs: R float[Hkv*nb] (required unless the tensor-core path is
+ * taken; may then be NULL), block_idx int32[Hkv*C], block_cnt int32[Hkv], sink_keep uint8[Hkv*n_sink], O, lse. */
+focus_status focus_sparse_layer(focus_ctx* ctx, const focus_shape* shape, const void* Q, int32_t q_base, int32_t n_q,
+                                const int32_t* q_rows, const int32_t* n_rows, int32_t max_rows,
+                                const int32_t* focus_idx, const int32_t* n_focus, int32_t max_focus,
+                                const void* K, const void* V, const float* Kbar, int32_t C,
+                                const int32_t* sink_idx, int32_t n_sink, float* R, int32_t* block_idx,
+                                int32_t* block_cnt, uint8_t* sink_keep, void* O, float* lse, focus_stream stream);
+
 /* Bidirectional softmax attention of the same rows over all L keys ("FullAttn" of Algorithm 1): the
  * dense layers, the probe layer (its lse feeds focus_find_sinks) and the baseline of the benchmark. */
 focus_status focus_dense_attn(focus_ctx* ctx, const focus_shape* shape, const void* Q, int32_t q_base, int32_t n_q,

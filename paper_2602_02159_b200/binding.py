@@ -49,6 +49,8 @@ _SIGS = {
     "focus_score_blocks": (_I, [_P, _SH, _P, _I, _P, _P, _I, _P, _P, _I, _P, _P]),
     "focus_select_blocks": (_I, [_P, _SH, _P, _I, _I, _P, _I, _I, _P, _I, _P, _P, _P]),
     "focus_sparse_attn": (_I, [_P, _SH, _P, _I, _I, _P, _P, _I, _P, _P, _I, _P, _I, _P, _P, _P, _I, _P, _P, _P]),
+    "focus_sparse_layer": (_I, [_P, _SH, _P, _I, _I, _P, _P, _I, _P, _P, _I, _P, _P, _P, _I, _P, _I, _P, _P, _P, _P, _P,
+                                _P, _P]),
     "focus_dense_attn": (_I, [_P, _SH, _P, _I, _I, _P, _P, _I, _P, _P, _P, _P, _P]),
 }
 
@@ -186,6 +188,15 @@ def focus_sparse_attn(ctx, shape, Q, q_base, n_q, q_rows, n_rows, max_rows, K, V
                                       max_rows, _ptr(K), _ptr(V), head_reduce, _ptr(block_idx), max_blocks,
                                       _ptr(block_cnt), _ptr(sink_idx), _ptr(sink_keep), n_sink, _ptr(O), _ptr(lse),
                                       _stream(stream)), "focus_sparse_attn")
+
+
+def focus_sparse_layer(ctx, shape, Q, q_base, n_q, q_rows, n_rows, max_rows, focus_idx, n_focus, max_focus, K, V, Kbar,
+                       C_keep, sink_idx, n_sink, R, block_idx, block_cnt, sink_keep, O, lse=None, stream=None):
+    _check(ctx._lib.focus_sparse_layer(ctx.handle, C.byref(shape), _ptr(Q), q_base, n_q, _ptr(q_rows), _ptr(n_rows),
+                                       max_rows, _ptr(focus_idx), _ptr(n_focus), max_focus, _ptr(K), _ptr(V),
+                                       _ptr(Kbar), C_keep, _ptr(sink_idx), n_sink, _ptr(R), _ptr(block_idx),
+                                       _ptr(block_cnt), _ptr(sink_keep), _ptr(O), _ptr(lse), _stream(stream)),
+           "focus_sparse_layer")
 
 
 def focus_dense_attn(ctx, shape, Q, q_base, n_q, q_rows, n_rows, max_rows, K, V, O, lse=None, stream=None):

@@ -498,6 +498,12 @@ size_t attn_tc_workspace(const focus_shape* s, int n_q, int max_blocks, int n_si
 }
 
 focus_status launch_attn_tc(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st) {
+  WsAlloc ws(ctx);
+  return launch_attn_tc_ws(ctx, a, ws, nullptr, st);
+}
+
+// `pre` non-NULL: the sink rows and the column mask were already gathered into it by the caller (taken from `ws`).
+focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, const SinkGather* pre, cudaStream_t st) {
   const focus_shape& sh = a.sh;
   const int Hkv = sh.n_kv_heads, hpg = sh.n_q_heads / Hkv;
   const int n_mtiles = (int)(((long long)a.max_rows * hpg + TM - 1) / TM);
@@ -508,12 +514,15 @@ focus_status launch_attn_tc(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st) 
   const int max_tiles = a.dense ? n_resp : a.max_blocks + ns_pad / TN + n_resp;
   const int n_splits = pick_splits(ctx, base, max_tiles);
 
-  WsAlloc ws(ctx);
   __nv_bfloat16* gK = nullptr; __nv_bfloat16* gV = nullptr; uint8_t* mask = nullptr;
   if (ns_pad > 0) {
-    gK = ws.get<__nv_bfloat16>((size_t)Hkv * ns_pad * HD);
-    gV = ws.get<__nv_bfloat16>((size_t)Hkv * ns_pad * HD);
-    mask = ws.get<uint8_t>((size_t)Hkv * ns_pad);
+    if (pre) {
+      gK = pre->gK; gV = pre->gV; mask = pre->mask;
+    } else {
+      gK = ws.get<__nv_bfloat16>((size_t)Hkv * ns_pad * HD);
+      gV = ws.get<__nv_bfloat16>((size_t)Hkv * ns_pad * HD);
+      mask = ws.get<uint8_t>((size_t)Hkv * ns_pad);
+    }
   }
   float* part_O = nullptr; float* part_ml = nullptr;
   if (n_splits > 1) {
@@ -530,11 +539,13 @@ focus_status launch_attn_tc(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st) 
     if (!encode_kv_map(ctx->encode_tiled, &tmSK, gK, HD, ns_pad, Hkv, HD, (long long)ns_pad * HD, 64, TN) ||
         !encode_kv_map(ctx->encode_tiled, &tmSV, gV, HD, ns_pad, Hkv, HD, (long long)ns_pad * HD, 64, TN))
       return FOCUS_ERR_CUDA;
-    dim3 gg((ns_pad + 15) / 16, Hkv);
-    sink_gather_kernel<<<gg, 256, 0, st>>>((const __nv_bfloat16*)a.K, (const __nv_bfloat16*)a.V, sh.kv_stride_tok,
-                                           sh.kv_stride_head, a.sink_idx, a.sink_keep, a.n_sink, ns_pad,
-                                           a.group_stride, sh.M, sh.L, gK, gV, mask, ctx->d_status);
-    FOCUS_CHECK_LAUNCH();
+    if (!pre) {
+      dim3 gg((ns_pad + 15) / 16, Hkv);
+      sink_gather_kernel<<<gg, 256, 0, st>>>((const __nv_bfloat16*)a.K, (const __nv_bfloat16*)a.V, sh.kv_stride_tok,
+                                             sh.kv_stride_head, a.sink_idx, a.sink_keep, a.n_sink, ns_pad,
+                                             a.group_stride, sh.M, sh.L, gK, gV, mask, ctx->d_status);
+      FOCUS_CHECK_LAUNCH();
+    }
   } else {
     tmSK = tmK; tmSV = tmV;
   }

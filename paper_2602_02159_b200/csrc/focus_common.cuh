@@ -131,7 +131,14 @@ struct AttnArgs {
   int lse_stride;
 };
 
+struct SinkGather {          // sink rows of one layer gathered into compact per-KV-head tiles
+  __nv_bfloat16* gK;         // [Hkv][ns_pad][128]
+  __nv_bfloat16* gV;
+  uint8_t* mask;             // [Hkv][ns_pad]: 1 = attend this column
+};
+
 focus_status launch_attn_simt(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st);
+focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, const SinkGather* pre, cudaStream_t st);
 focus_status launch_attn_tc(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st);
 bool attn_tc_supported(const focus_ctx* ctx, const AttnArgs& a);
 size_t attn_tc_workspace(const focus_shape* s, int n_q, int max_blocks, int n_sink);

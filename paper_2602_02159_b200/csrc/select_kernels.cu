@@ -193,6 +193,15 @@ __global__ void sink_reduce_heads_kernel(const float* __restrict__ part, int H, 
 
 constexpr int TN_THREADS = 1024;
 
+// Histogram increment with warp aggregation: lanes that hit the same bin elect one leader that adds their
+// count.  Sink scores are all close to 1/L, so without this nearly every add lands on one counter.
+__device__ __forceinline__ void hist_add(int* hist, uint32_t bin, bool active) {
+  const uint32_t amask = __ballot_sync(0xffffffffu, active);
+  if (!active) return;
+  const uint32_t peers = __match_any_sync(amask, bin);
+  if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
+}
+
 __global__ void __launch_bounds__(TN_THREADS)
 sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const int32_t* n_active,
                  int32_t* __restrict__ sink_idx, int32_t* status) {
@@ -215,22 +224,43 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
   // radix select: find the key T of the want-th largest element, MSB first
   uint32_t prefix = 0, pmask = 0;
   int remaining = want;                       // rank (1-based) still to locate inside the current bucket
+  const int n_round = (n + TN_THREADS - 1) / TN_THREADS * TN_THREADS;
   for (int shift = 24; shift >= 0; shift -= 8) {
     for (int b = tid; b < 256; b += TN_THREADS) hist[b] = 0;
     __syncthreads();
-    for (int i = tid; i < n; i += TN_THREADS) {
-      const uint32_t k = float_key(S[lo + i]);
-      if ((k & pmask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1);
+    for (int i = tid; i < n_round; i += TN_THREADS) {
+      uint32_t k = 0;
+      if (i < n) k = float_key(S[lo + i]);
+      hist_add(hist, (k >> shift) & 255u, i < n && (k & pmask) == prefix);
     }
     __syncthreads();
-    if (tid == 0) {
-      int acc = 0, b = 255;
-      for (; b > 0; --b) {
-        if (acc + hist[b] >= remaining) break;
-        acc += hist[b];
+    if (tid < 32) {
+      // bucket b such that (count of keys in buckets above b) < remaining <= (that count + hist[b])
+      int above = 0, found = -1, found_above = 0;
+      for (int base = 224; base >= 0 && found < 0; base -= 32) {
+        const int b = base + 31 - tid;                       // lane 0 owns the highest bucket of the group
+        const int h = hist[b];
+        int incl = h;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, incl, o);
+          if (tid >= o) incl += y;
+        }
+        const bool hit = above + incl >= remaining;
+        const uint32_t bal = __ballot_sync(0xffffffffu, hit);
+        if (bal) {
+          const int l0 = __ffs(bal) - 1;
+          found = base + 31 - l0;
+          found_above = above + __shfl_sync(0xffffffffu, incl - h, l0);
+        } else {
+          above += __shfl_sync(0xffffffffu, incl, 31);
+        }
       }
-      s_prefix = prefix | ((uint32_t)b << shift);
-      s_remaining = remaining - acc;
+      if (tid == 0) {
+        if (found < 0) { found = 0; found_above = above - hist[0]; }
+        s_prefix = prefix | ((uint32_t)found << shift);
+        s_remaining = remaining - found_above;
+      }
     }
     __syncthreads();
     prefix = s_prefix;
@@ -239,22 +269,29 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
     __syncthreads();
   }
   const uint32_t T = prefix;                 // threshold key; `remaining` = how many == T to take (lowest index first)
-  int base = 0, eq_taken = 0;
-  for (int c0 = 0; c0 < n; c0 += TN_THREADS) {
-    const int i = c0 + tid;
-    uint32_t k = 0;
-    if (i < n) k = float_key(S[lo + i]);
-    const int is_eq = (i < n && k == T) ? 1 : 0;
-    int tot_eq;
-    const int pre_eq = block_excl_scan(is_eq, scan_s, tot_eq);
-    const int f = (i < n && (k > T || (is_eq && eq_taken + pre_eq < remaining))) ? 1 : 0;
-    int tot;
-    const int pre = block_excl_scan(f, scan_s, tot);
-    if (f) sink_idx[base + pre] = lo + i;
-    base += tot;
-    eq_taken += tot_eq;
+  // ordered compaction: thread t owns the contiguous chunk [t*cs, (t+1)*cs)
+  const int cs = (n + TN_THREADS - 1) / TN_THREADS;
+  const int c_lo = min(tid * cs, n), c_hi = min(c_lo + cs, n);
+  int n_gt = 0, n_eq = 0;
+  for (int i = c_lo; i < c_hi; ++i) {
+    const uint32_t k = float_key(S[lo + i]);
+    n_gt += k > T;
+    n_eq += k == T;
   }
-  for (int i = base + tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
+  int tot_eq, tot_gt;
+  const int pre_eq = block_excl_scan(n_eq, scan_s, tot_eq);
+  const int take_eq = max(0, min(n_eq, remaining - pre_eq));        // equals are taken in index order
+  int tot_sel;
+  const int pre_sel = block_excl_scan(n_gt + take_eq, scan_s, tot_sel);
+  (void)tot_gt;
+  int out = pre_sel, eq_seen = 0;
+  for (int i = c_lo; i < c_hi; ++i) {
+    const uint32_t k = float_key(S[lo + i]);
+    bool take = k > T;
+    if (k == T) { take = eq_seen < take_eq; ++eq_seen; }
+    if (take) sink_idx[out++] = lo + i;
+  }
+  for (int i = tot_sel + tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
 }
 
 focus_status launch_sink_select(focus_ctx* ctx, const float* part, int H, int L, const int32_t* n_active, float* S,

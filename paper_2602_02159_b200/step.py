@@ -94,14 +94,21 @@ def find_sinks(ctx, b: StepBuffers, Q, K, lse: Optional[torch.Tensor], stream=No
                         b.sink_idx, b.sink_scores, stream)
 
 
-def sparse_layer(ctx, b: StepBuffers, Q, K, V, Kbar: Optional[torch.Tensor] = None, O=None, lse=None, stream=None):
-    """score_blocks -> select_blocks -> sparse_attn for one sparse layer (Algorithm 1, sparse branch)."""
+def sparse_layer(ctx, b: StepBuffers, Q, K, V, Kbar: Optional[torch.Tensor] = None, O=None, lse=None, stream=None,
+                 fused: bool = True):
+    """score_blocks -> select_blocks -> sparse_attn for one sparse layer (Algorithm 1, sparse branch); with cached
+    pooled keys and the default modes this is the single fused call focus_sparse_layer."""
     w, s = b.wl, b.wl.shape
+    q_rows, n_rows, max_rows = b._rows()
+    if Kbar is not None and b.head_reduce == fb.HEADS_PER_KV_GROUP and b.sink_mode == fb.SINK_TOKENS and fused:
+        fb.focus_sparse_layer(ctx, b.shape, Q, s.M, s.N, q_rows, n_rows, max_rows, b.focus_idx, b.n_focus, max(1, w.k),
+                              K, V, Kbar, w.C, b.sink_idx, w.n_sink, b.R, b.block_idx, b.block_cnt, b.sink_keep,
+                              b.O if O is None else O, b.lse if lse is None else lse, stream)
+        return
     fb.focus_score_blocks(ctx, b.shape, Q, s.M, b.focus_idx, b.n_focus, max(1, w.k), None if Kbar is not None else K,
                           Kbar, b.head_reduce, b.R, stream)
     fb.focus_select_blocks(ctx, b.shape, b.R, b.head_reduce, w.C, b.sink_idx, w.n_sink, b.sink_mode, b.block_idx,
                            b.max_blocks, b.block_cnt, b.sink_keep, stream)
-    q_rows, n_rows, max_rows = b._rows()
     fb.focus_sparse_attn(ctx, b.shape, Q, s.M, s.N, q_rows, n_rows, max_rows, K, V, b.head_reduce, b.block_idx,
                          b.max_blocks, b.block_cnt, b.sink_idx, b.sink_keep, w.n_sink, b.O if O is None else O,
                          b.lse if lse is None else lse, stream)

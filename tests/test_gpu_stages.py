@@ -244,6 +244,42 @@ def test_long_key_pipeline_single_split(ctx):
     assert ctx.poll_status() == 0
 
 
+@pytest.mark.parametrize("cfg", [SHAPES[0], SHAPES[2], SHAPES[3]])
+def test_fused_sparse_layer_matches_stagewise_and_oracle(ctx, cfg):
+    """focus_sparse_layer (fused selection + attention) against the stage-by-stage calls and the oracle."""
+    dtype, d, B, H, Hkv = cfg
+    w = small_workload(dtype, d, B, H=H, Hkv=Hkv, n_sink=150, C=4, seed=8)       # two sink tiles
+    s = w.shape
+    host, dev = make_inputs(w)
+    ora = oracle_chain(w, host, fb.HEADS_PER_KV_GROUP, fb.SINK_TOKENS)
+    Kbar = torch.zeros(s.Hkv, s.nb, s.d, dtype=torch.float32, device="cuda")
+    outs = []
+    for fused in (False, True):
+        b = fstep.StepBuffers(w)
+        fb.focus_pool_keys(ctx, b.shape, dev["K"], Kbar)
+        fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
+        b.sink_idx.copy_(torch.from_numpy(ora["sinks"].astype(np.int32)))
+        fstep.sparse_layer(ctx, b, dev["Q"], dev["K"], dev["V"], Kbar=Kbar, fused=fused)
+        torch.cuda.synchronize()
+        outs.append(b)
+    a, f = outs
+    assert torch.equal(a.block_idx, f.block_idx) and torch.equal(a.block_cnt, f.block_cnt)
+    assert torch.equal(a.sink_keep, f.sink_keep)
+    assert max_abs(fstep.from_device(a.R), fstep.from_device(f.R)) <= 1e-6 * max(1.0, np.abs(ora["R"]).max())
+    na = len(ora["active"])
+    bi = f.block_idx.cpu().numpy().reshape(s.Hkv, -1)
+    for g in range(s.Hkv):
+        check_topk_band(bi[g], ora["blocks"][g], ora["R"][g], range(s.nb), BAND, scale_ref=np.abs(ora["R"][g]).max())
+    blocks = [bi[g] for g in range(s.Hkv)]
+    Os, lses = fo.sparse_attn(host["Q"][ora["active"] - s.M], host["K"], host["V"], s.M, s.B, blocks, ora["sinks"],
+                              ora["scale"])
+    for b in outs:
+        got = fstep.from_device(b.O)[:na]
+        assert max_abs(got, Os) <= TOL_ABS[dtype] and rel_rms(got, Os) <= TOL_RMS[dtype]
+        assert max_abs(fstep.from_device(b.lse)[:, :na], lses) <= TOL_LSE[dtype]
+    assert ctx.poll_status() == 0
+
+
 def test_degenerate_cases(ctx):
     """C = 0 with no sinks (response keys only), n_sink = 0, Q = 0 (uniform weights pin the key set),
     a single query row, block list given in descending order."""
