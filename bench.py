@@ -80,7 +80,7 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------------
 # CPU oracle arm (also the cpu_baseline leg of the default arm)
 # --------------------------------------------------------------------------------------------------
-def oracle_sample(w, heads=(0, 1), repeats=1):
+def oracle_sample(w, heads=tuple(range(8)), repeats=1):
     """Times the CPU oracle on a bounded sample of one step: `heads` of the H heads, one dense layer, the
     probe-layer sink scores and one sparse layer; scales to the whole step (all heads, the layer schedule)."""
     from oracle import focus_oracle as fo
@@ -275,9 +275,30 @@ def run_focus(args):
         return tot / steps, launches, marks
 
     K, W = args.steps, max(args.warmup, 3)
+    # eager pass with CUDA-event marks around every attention call: per-kernel durations for the roofline
+    ms_eager, launches, marks = timed(lambda m: step("active", marks=m), K, W, with_marks=True)
+    assert ctx.poll_status() == 0, "device status word set during the timed region"
+    # the same step captured once into a CUDA graph (counts stay on the device, so nothing needs the host)
+    graph = None
+    if not args.no_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            step("active")
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        n0 = fb.focus_launch_count()
+        with torch.cuda.graph(graph):
+            step("active")
+        launches = fb.focus_launch_count() - n0          # kernels per replayed step
     sampler = ClockSampler(local)
     sampler.start()
-    ms_step, launches, marks = timed(lambda m: step("active", marks=m), K, W, with_marks=True)
+    if graph is not None:
+        ms_step, _, _ = timed(lambda m: graph.replay(), K, W)
+        launches *= K
+    else:
+        ms_step = ms_eager
     clocks = sampler.stop()
     assert ctx.poll_status() == 0, "device status word set during the timed region"
 
@@ -357,6 +378,8 @@ def run_focus(args):
                    "pooled_keys": "cached per KV-cache refresh", "l2": "inputs larger than L2 (17 GB of K/V per step)",
                    "multi_gpu": "independent replicas, no data-path collective", "input_gen_s": round(t_gen, 1)},
         "gpu_launches": int(launches),
+        "launch_mode": "one CUDA graph replay per step" if graph is not None else "eager C-ABI calls",
+        "eager_ms_per_step": ms_eager,
         "clocks": clocks,
         "speedup_vs_own_dense": ms_dense_step / ms_step,
         "own_dense_ms_per_step": ms_dense_step,
@@ -390,6 +413,7 @@ def main():
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (quick runs)")
     ap.add_argument("--skip-gen", action="store_true", help="skip the gen-region-rows (tensor-bound) measurements")
+    ap.add_argument("--no-graph", action="store_true", help="time eager C-ABI calls instead of a CUDA graph replay")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle baseline leg")
     args = ap.parse_args()
     if args.impl == "reference":

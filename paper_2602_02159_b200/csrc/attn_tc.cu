@@ -42,6 +42,7 @@ struct TcParams {
   const uint8_t* sink_mask;    // [Hkv][ns_pad]: 1 = attend this gathered sink column
   float* part_O;               // [cta][128][128] unnormalised partial outputs (n_splits > 1)
   float* part_ml;              // [cta][128][2] running max (log2 domain) and running sum
+  int32_t* counters;           // one arrival counter per (KV head, query tile); NULL: a separate kernel merges the splits
   long long q_stride_row, q_stride_head;
   int q_base, n_q, rows_bound, L, M, H, Hkv, hpg, B, nb, dense, group_stride, max_blocks, n_sink, ns_pad;
   int n_mtiles, n_splits, lse_stride;
@@ -97,6 +98,56 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams& p, const TileEnum&
   return ti;
 }
 
+// Merge of the split partials of one (KV head, query tile): out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s,
+// splits taken in index order (deterministic whoever runs it).  One warp per stacked row.
+__device__ __forceinline__ void merge_rows(const TcParams& p, int tile, int g, int mt, int total_fr, int warp,
+                                           int n_warps, int lane) {
+  const int rows = min(TM, total_fr - mt * TM);
+  for (int row = warp; row < rows; row += n_warps) {
+    float m = -INFINITY;
+    for (int s = 0; s < p.n_splits; ++s) {
+      const float* ml = p.part_ml + ((size_t)(tile * p.n_splits + s) * TM + row) * 2;
+      if (__ldcg(ml + 1) > 0.f) m = fmaxf(m, __ldcg(ml));
+    }
+    float tot = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < p.n_splits; ++s) {
+      const size_t base = (size_t)(tile * p.n_splits + s) * TM + row;
+      const float ls = __ldcg(p.part_ml + base * 2 + 1);
+      if (!(ls > 0.f)) continue;
+      const float wgt = exp2f(__ldcg(p.part_ml + base * 2) - m);
+      tot += wgt * ls;
+      const float4 o = __ldcg(reinterpret_cast<const float4*>(p.part_O + base * HD + lane * 4));
+      acc.x += wgt * o.x; acc.y += wgt * o.y; acc.z += wgt * o.z; acc.w += wgt * o.w;
+    }
+    const float inv = tot > 0.f ? 1.f / tot : 0.f;
+    const int fr = mt * TM + row;
+    const int qr = fr / p.hpg, hh = fr % p.hpg;
+    __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD + lane * 4;
+    uint2 v;
+    v.x = pack_bf16(acc.x * inv, acc.y * inv);
+    v.y = pack_bf16(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2*>(orow) = v;
+    if (p.lse && lane == 0)
+      p.lse[(size_t)(g * p.hpg + hh) * p.lse_stride + qr] = (m + log2f(tot)) * 0.6931471805599453f;
+  }
+}
+
+// Called by every thread of every split CTA once its partial is written: the CTA that arrives last at the
+// tile's counter merges all splits and re-arms the counter for the next launch.
+__device__ __forceinline__ void finish_split(const TcParams& p, int tile, int g, int mt, int total_fr, int* s_last) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int prev = atomicAdd(&p.counters[tile], 1);
+    *s_last = prev == p.n_splits - 1;
+    if (*s_last) p.counters[tile] = 0;
+    __threadfence();
+  }
+  __syncthreads();
+  if (*s_last) merge_rows(p, tile, g, mt, total_fr, threadIdx.x >> 5, NTHREADS / 32, threadIdx.x & 31);
+}
+
 __global__ void __launch_bounds__(NTHREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                const __grid_constant__ CUtensorMap tmSK, const __grid_constant__ CUtensorMap tmSV, const TcParams p) {
@@ -127,11 +178,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(sptr + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
+  __shared__ int s_last;
   if (nt <= 0) {                                          // empty split: publish a neutral partial
-    if (p.n_splits > 1 && warp >= 2) {
-      const int row = (warp & 3) * 32 + lane;
-      p.part_ml[((size_t)cta_lin * TM + row) * 2 + 0] = -INFINITY;
-      p.part_ml[((size_t)cta_lin * TM + row) * 2 + 1] = 0.f;
+    if (p.n_splits > 1) {
+      if (warp >= 2) {
+        const int row = (warp & 3) * 32 + lane;
+        if (mt * TM + row < total_fr) {
+          p.part_ml[((size_t)cta_lin * TM + row) * 2 + 0] = -INFINITY;
+          p.part_ml[((size_t)cta_lin * TM + row) * 2 + 1] = 0.f;
+        }
+      }
+      if (p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, &s_last);
     }
     return;
   }
@@ -380,19 +437,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         }
         if (valid && p.lse)
           p.lse[(size_t)(g * p.hpg + hh) * p.lse_stride + qr] = (m_ref + log2f(l)) * 0.6931471805599453f;
-      } else {
+      } else if (__any_sync(0xffffffffu, valid)) {           // warps whose 32 rows are all padding have nothing to publish
         float* po = p.part_O + ((size_t)cta_lin * TM + row) * HD;
 #pragma unroll
         for (int cb = 0; cb < 4; ++cb) {
           uint32_t oreg[32];
           TC_LD32(tmem_O + lane_off + cb * 32, oreg);
           tc_wait_ld();
+          if (valid) {
 #pragma unroll
-          for (int c = 0; c < 32; c += 4)
-            *reinterpret_cast<uint4*>(po + cb * 32 + c) = make_uint4(oreg[c], oreg[c + 1], oreg[c + 2], oreg[c + 3]);
+            for (int c = 0; c < 32; c += 4)
+              *reinterpret_cast<uint4*>(po + cb * 32 + c) = make_uint4(oreg[c], oreg[c + 1], oreg[c + 2], oreg[c + 3]);
+          }
         }
-        p.part_ml[((size_t)cta_lin * TM + row) * 2 + 0] = m_ref;
-        p.part_ml[((size_t)cta_lin * TM + row) * 2 + 1] = l;
+        if (valid) {
+          p.part_ml[((size_t)cta_lin * TM + row) * 2 + 0] = m_ref;
+          p.part_ml[((size_t)cta_lin * TM + row) * 2 + 1] = l;
+        }
       }
     }
   }
@@ -403,9 +464,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     __syncwarp();
     tmem_dealloc(tmem, 512);
   }
+  if (p.n_splits > 1 && p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, &s_last);
 }
 
-// Merge of the split partials: out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s, one warp per stacked row.
+// Stand-alone merge (used when there are more query tiles than arrival counters): out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s, one warp per stacked row.
 __global__ void __launch_bounds__(256)
 attn_combine_kernel(const float* __restrict__ part_O, const float* __restrict__ part_ml, int n_splits, int n_mtiles,
                     int hpg, int H, const int32_t* q_rows, const int32_t* n_rows, int rows_bound, int n_q,
@@ -554,6 +616,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.Q = (const __nv_bfloat16*)a.Q; p.O = (__nv_bfloat16*)a.O; p.lse = a.lse;
   p.q_rows = a.q_rows; p.n_rows = a.n_rows; p.block_idx = a.block_idx; p.block_cnt = a.block_cnt;
   p.sink_mask = mask; p.part_O = part_O; p.part_ml = part_ml;
+  p.counters = (n_splits > 1 && base <= FOCUS_N_COUNTERS) ? ctx->d_counters : nullptr;
   p.q_stride_row = sh.q_stride_row; p.q_stride_head = sh.q_stride_head;
   p.q_base = a.q_base; p.n_q = a.n_q; p.rows_bound = a.max_rows; p.L = sh.L; p.M = sh.M; p.H = sh.n_q_heads;
   p.Hkv = Hkv; p.hpg = hpg; p.B = sh.kv_block; p.nb = shape_nb(&sh); p.dense = a.dense;
@@ -570,7 +633,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   }
   attn_tc_kernel<<<dim3(base, n_splits), NTHREADS, SMEM_BYTES, st>>>(tmK, tmV, tmSK, tmSV, p);
   FOCUS_CHECK_LAUNCH();
-  if (n_splits > 1) {
+  if (n_splits > 1 && !p.counters) {
     const int rows_total = base * TM;
     attn_combine_kernel<<<rows_total / 8, 256, 0, st>>>(part_O, part_ml, n_splits, n_mtiles, hpg, sh.n_q_heads,
                                                         a.q_rows, a.n_rows, a.max_rows, a.n_q,

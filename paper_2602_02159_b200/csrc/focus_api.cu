@@ -54,12 +54,14 @@ extern "C" focus_status focus_create(focus_ctx** out, int device, size_t workspa
         q == cudaDriverEntryPointSuccess)
       c->encode_tiled = fn;
   }
-  if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess || cudaMalloc(&c->d_status, 256) != cudaSuccess) {
+  if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess ||
+      cudaMalloc(&c->d_status, 256 + FOCUS_N_COUNTERS * sizeof(int32_t)) != cudaSuccess) {
     if (c->ws) cudaFree(c->ws);
     delete c;
     return FOCUS_ERR_CUDA;
   }
-  cudaMemset(c->d_status, 0, 256);
+  cudaMemset(c->d_status, 0, 256 + FOCUS_N_COUNTERS * sizeof(int32_t));
+  c->d_counters = c->d_status + 64;
   *out = c;
   return FOCUS_OK;
 }

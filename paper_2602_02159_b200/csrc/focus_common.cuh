@@ -13,9 +13,12 @@ struct focus_ctx {
   char* ws;            // workspace (device)
   size_t ws_bytes;
   int32_t* d_status;   // device status word: 0 = clean, else first anomaly's focus_status code
+  int32_t* d_counters; // FOCUS_N_COUNTERS arrival counters for split merges; zero between launches
   int force_simt;
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime (no libcuda link)
 };
+
+constexpr int FOCUS_N_COUNTERS = 4096;
 
 // Bump allocator over the context workspace; one per API call.
 struct WsAlloc {

@@ -192,6 +192,7 @@ __global__ void sink_reduce_heads_kernel(const float* __restrict__ part, int H, 
 }
 
 constexpr int TN_THREADS = 1024;
+constexpr int TN_MAX_SMEM_KEYS = 56 * 1024;      // keys cached in shared memory (224 KB); beyond that they are re-read
 
 // Histogram increment with warp aggregation: lanes that hit the same bin elect one leader that adds their
 // count.  Sink scores are all close to 1/L, so without this nearly every add lands on one counter.
@@ -202,14 +203,19 @@ __device__ __forceinline__ void hist_add(int* hist, uint32_t bin, bool active) {
   if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
 }
 
+// One CTA.  Keys (order-preserving integers of the scores) are staged once in shared memory, then: 4-pass 8-bit
+// radix select of the want-th largest key T, and an ordered compaction in which warp w owns the w-th contiguous
+// segment of the candidates (ballot/popc keeps index order inside a warp, one block scan orders the warps).
+template <bool CACHED>
 __global__ void __launch_bounds__(TN_THREADS)
 sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const int32_t* n_active,
                  int32_t* __restrict__ sink_idx, int32_t* status) {
+  extern __shared__ uint32_t skey[];
   __shared__ int hist[256];
   __shared__ int scan_s[33];
   __shared__ uint32_t s_prefix;
   __shared__ int s_remaining;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = hi - lo;
   const int want = min(n_sink, n);
   if (*n_active <= 0) {                      // undefined scores: report and emit an empty set
@@ -221,6 +227,12 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
     for (int i = tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
     return;
   }
+  if (CACHED) {
+#pragma unroll 8
+    for (int i = tid; i < n; i += TN_THREADS) skey[i] = float_key(S[lo + i]);
+    __syncthreads();
+  }
+  auto key_at = [&](int i) -> uint32_t { return CACHED ? skey[i] : float_key(S[lo + i]); };
   // radix select: find the key T of the want-th largest element, MSB first
   uint32_t prefix = 0, pmask = 0;
   int remaining = want;                       // rank (1-based) still to locate inside the current bucket
@@ -230,7 +242,7 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
     __syncthreads();
     for (int i = tid; i < n_round; i += TN_THREADS) {
       uint32_t k = 0;
-      if (i < n) k = float_key(S[lo + i]);
+      if (i < n) k = key_at(i);
       hist_add(hist, (k >> shift) & 255u, i < n && (k & pmask) == prefix);
     }
     __syncthreads();
@@ -269,27 +281,32 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
     __syncthreads();
   }
   const uint32_t T = prefix;                 // threshold key; `remaining` = how many == T to take (lowest index first)
-  // ordered compaction: thread t owns the contiguous chunk [t*cs, (t+1)*cs)
-  const int cs = (n + TN_THREADS - 1) / TN_THREADS;
-  const int c_lo = min(tid * cs, n), c_hi = min(c_lo + cs, n);
+  // ordered compaction: warp w owns candidates [w*seg, (w+1)*seg), seg a multiple of 32
+  const int seg = ((n + 31) / 32 + 31) / 32 * 32;
+  const int w_lo = min(warp * seg, n), w_hi = min(w_lo + seg, n);
   int n_gt = 0, n_eq = 0;
-  for (int i = c_lo; i < c_hi; ++i) {
-    const uint32_t k = float_key(S[lo + i]);
-    n_gt += k > T;
-    n_eq += k == T;
+  for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
+    const int i = i0 + lane;
+    const uint32_t k = i < w_hi ? key_at(i) : 0u;
+    n_gt += __popc(__ballot_sync(0xffffffffu, i < w_hi && k > T));
+    n_eq += __popc(__ballot_sync(0xffffffffu, i < w_hi && k == T));
   }
-  int tot_eq, tot_gt;
-  const int pre_eq = block_excl_scan(n_eq, scan_s, tot_eq);
-  const int take_eq = max(0, min(n_eq, remaining - pre_eq));        // equals are taken in index order
-  int tot_sel;
-  const int pre_sel = block_excl_scan(n_gt + take_eq, scan_s, tot_sel);
-  (void)tot_gt;
-  int out = pre_sel, eq_seen = 0;
-  for (int i = c_lo; i < c_hi; ++i) {
-    const uint32_t k = float_key(S[lo + i]);
-    bool take = k > T;
-    if (k == T) { take = eq_seen < take_eq; ++eq_seen; }
-    if (take) sink_idx[out++] = lo + i;
+  int tot_eq, tot_sel;
+  const int pre_eq = block_excl_scan(lane == 0 ? n_eq : 0, scan_s, tot_eq);          // per-warp values on lane 0
+  const int w_pre_eq = __shfl_sync(0xffffffffu, pre_eq, 0);
+  const int take_eq = max(0, min(n_eq, remaining - w_pre_eq));                       // equals are taken in index order
+  const int pre_sel = block_excl_scan(lane == 0 ? n_gt + take_eq : 0, scan_s, tot_sel);
+  int out = __shfl_sync(0xffffffffu, pre_sel, 0), eq_seen = 0;
+  for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
+    const int i = i0 + lane;
+    const uint32_t k = i < w_hi ? key_at(i) : 0u;
+    const uint32_t m_eq = __ballot_sync(0xffffffffu, i < w_hi && k == T);
+    const int my_eq_rank = eq_seen + __popc(m_eq & ((1u << lane) - 1u));
+    const bool take = i < w_hi && (k > T || (k == T && my_eq_rank < take_eq));
+    const uint32_t m_take = __ballot_sync(0xffffffffu, take);
+    if (take) sink_idx[out + __popc(m_take & ((1u << lane) - 1u))] = lo + i;
+    out += __popc(m_take);
+    eq_seen += __popc(m_eq);
   }
   for (int i = tot_sel + tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
 }
@@ -298,7 +315,20 @@ focus_status launch_sink_select(focus_ctx* ctx, const float* part, int H, int L,
                                 int cand_lo, int cand_hi, int n_sink, int32_t* sink_idx, cudaStream_t st) {
   sink_reduce_heads_kernel<<<(L + 255) / 256, 256, 0, st>>>(part, H, L, n_active, S);
   FOCUS_CHECK_LAUNCH();
-  sink_topn_kernel<<<1, TN_THREADS, 0, st>>>(S, cand_lo, cand_hi, n_sink, n_active, sink_idx, ctx->d_status);
+  const int n = cand_hi - cand_lo;
+  if (n <= TN_MAX_SMEM_KEYS) {
+    static bool attr_set = false;
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(sink_topn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               TN_MAX_SMEM_KEYS * 4) != cudaSuccess)
+        return FOCUS_ERR_CUDA;
+      attr_set = true;
+    }
+    sink_topn_kernel<true><<<1, TN_THREADS, (size_t)n * 4, st>>>(S, cand_lo, cand_hi, n_sink, n_active, sink_idx,
+                                                                ctx->d_status);
+  } else {
+    sink_topn_kernel<false><<<1, TN_THREADS, 0, st>>>(S, cand_lo, cand_hi, n_sink, n_active, sink_idx, ctx->d_status);
+  }
   FOCUS_CHECK_LAUNCH();
   return FOCUS_OK;
 }

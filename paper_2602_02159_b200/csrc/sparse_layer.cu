@@ -47,12 +47,25 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
   __shared__ float qbar[FS_HD];
   __shared__ int scan_s[33];
   const int g = blockIdx.x;
+  const int warp = tid >> 5, lane = tid & 31;
+  // Issue every load that does not depend on another one first: the kernel is a chain of global-memory
+  // latencies, not of bandwidth.
+  constexpr int KPRE = 8;
+  const float* kb = Kbar + (size_t)g * nb * FS_HD + lane * 4;
+  float4 kpre[KPRE];
+#pragma unroll
+  for (int u = 0; u < KPRE; ++u) {
+    const int b = warp + u * (FS_THREADS / 32);
+    kpre[u] = b < nb ? __ldg(reinterpret_cast<const float4*>(kb + (size_t)b * FS_HD)) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  const int my_sink = tid < n_sink ? sink_idx[tid] : -1;
+  const int c = tid & 127, y = tid >> 7;
+  const int pos0 = y < max_focus ? focus_idx[y] : -1;
   const int nf = min(max(*n_focus, 0), max_focus);
   {
-    const int c = tid & 127, y = tid >> 7;
     float acc = 0.f;
     for (int i = y; i < nf; i += 8) {
-      const int pos = focus_idx[i];
+      const int pos = i == y ? pos0 : focus_idx[i];
       if (pos < q_base || pos >= L) {
         if (c == 0) set_status(status, FOCUS_ERR_INVALID_ARG);
         continue;
@@ -66,18 +79,14 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
   if (tid < FS_HD) {
     float s = 0.f;
 #pragma unroll
-    for (int y = 0; y < 8; ++y) s += part[y][tid];
+    for (int yy = 0; yy < 8; ++yy) s += part[yy][tid];
     qbar[tid] = nf > 0 ? s / (float)(nf * hpg) : 0.f;
     if (tid == 0 && nf == 0) set_status(status, FOCUS_ERR_INVALID_ARG);
   }
   __syncthreads();
   {
-    const int warp = tid >> 5, lane = tid & 31;
     const float4 qv = *reinterpret_cast<const float4*>(&qbar[lane * 4]);
-    const float* kb = Kbar + (size_t)g * nb * FS_HD + lane * 4;
-#pragma unroll 4
-    for (int b = warp; b < nb; b += FS_THREADS / 32) {
-      const float4 kv = __ldg(reinterpret_cast<const float4*>(kb + (size_t)b * FS_HD));
+    auto score = [&](int b, const float4& kv) {
       float s = kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
@@ -85,7 +94,15 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
         key[b] = float_key(s);
         if (R) R[(size_t)g * nb + b] = s;
       }
+    };
+#pragma unroll
+    for (int u = 0; u < KPRE; ++u) {
+      const int b = warp + u * (FS_THREADS / 32);
+      if (b < nb) score(b, kpre[u]);
     }
+#pragma unroll 4
+    for (int b = warp + KPRE * (FS_THREADS / 32); b < nb; b += FS_THREADS / 32)
+      score(b, __ldg(reinterpret_cast<const float4*>(kb + (size_t)b * FS_HD)));
   }
   __syncthreads();
   for (int i = tid; i < nb; i += FS_THREADS) {
@@ -101,7 +118,7 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
   for (int s = tid; s < ns_pad; s += FS_THREADS) {
     uint8_t keep = 0, mk = 0;
     if (s < n_sink) {
-      const int j = sink_idx[s];
+      const int j = s == tid ? my_sink : sink_idx[s];
       if (j >= 0 && j < L) {
         const int b = j / B;
         keep = (b < nb && !sel[b]) ? 1 : 0;
