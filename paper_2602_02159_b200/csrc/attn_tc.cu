@@ -27,7 +27,8 @@ constexpr int SLOT_BYTES = TN * HD * 2;
 constexpr int HALF_BYTES = SLOT_BYTES / 2;     // one 64-wide half of a tile: 128 rows x 128 bytes
 constexpr int Q_BYTES = TM * HD * 2;
 constexpr int NBAR = 2 * NSLOT + 5;
-constexpr int SMEM_BYTES = 1024 + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8 + 64;
+constexpr int MAXT = 128;            // key tiles of a split whose descriptors are staged in shared memory
+constexpr int SMEM_BYTES = 1024 + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8 + 64 + MAXT * 8;
 constexpr int NTHREADS = 192;
 constexpr float RESCALE_THRESHOLD = 8.0f;      // log2 units: O is rescaled only when the row max grew by more
 
@@ -104,21 +105,37 @@ __device__ __forceinline__ void merge_rows(const TcParams& p, int tile, int g, i
                                            int n_warps, int lane) {
   const int rows = min(TM, total_fr - mt * TM);
   for (int row = warp; row < rows; row += n_warps) {
+    // the merge is a chain of L2 latencies: read the per-split (max, sum) pairs lane-parallel, and keep four
+    // partial-output loads in flight at a time; the accumulation order stays s = 0, 1, 2, ...
     float m = -INFINITY;
-    for (int s = 0; s < p.n_splits; ++s) {
-      const float* ml = p.part_ml + ((size_t)(tile * p.n_splits + s) * TM + row) * 2;
-      if (__ldcg(ml + 1) > 0.f) m = fmaxf(m, __ldcg(ml));
+    for (int s0 = 0; s0 < p.n_splits; s0 += 32) {
+      const int s = s0 + lane;
+      if (s < p.n_splits) {
+        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((size_t)(tile * p.n_splits + s) * TM + row) * 2));
+        if (ml.y > 0.f) m = fmaxf(m, ml.x);
+      }
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     float tot = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < p.n_splits; ++s) {
-      const size_t base = (size_t)(tile * p.n_splits + s) * TM + row;
-      const float ls = __ldcg(p.part_ml + base * 2 + 1);
-      if (!(ls > 0.f)) continue;
-      const float wgt = exp2f(__ldcg(p.part_ml + base * 2) - m);
-      tot += wgt * ls;
-      const float4 o = __ldcg(reinterpret_cast<const float4*>(p.part_O + base * HD + lane * 4));
-      acc.x += wgt * o.x; acc.y += wgt * o.y; acc.z += wgt * o.z; acc.w += wgt * o.w;
+    for (int s0 = 0; s0 < p.n_splits; s0 += 4) {
+      float2 ml[4];
+      float4 o[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int s = min(s0 + u, p.n_splits - 1);
+        const size_t base = (size_t)(tile * p.n_splits + s) * TM + row;
+        ml[u] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + base * 2));
+        o[u] = __ldcg(reinterpret_cast<const float4*>(p.part_O + base * HD + lane * 4));
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (s0 + u >= p.n_splits || !(ml[u].y > 0.f)) continue;
+        const float wgt = exp2f(ml[u].x - m);
+        tot += wgt * ml[u].y;
+        acc.x += wgt * o[u].x; acc.y += wgt * o[u].y; acc.z += wgt * o[u].z; acc.w += wgt * o[u].w;
+      }
     }
     const float inv = tot > 0.f ? 1.f / tot : 0.f;
     const int fr = mt * TM + row;
@@ -177,8 +194,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   const uint32_t bar_pvdone = sBar + 8u * (2 * NSLOT + 4);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(sptr + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  int* s_last_p = reinterpret_cast<int*>(tmem_holder + 2);
+  int2* tlist = reinterpret_cast<int2*>(tmem_holder + 16);      // (start | kind << 30, nvalid) per tile of this split
+  const bool use_list = !p.dense && nt <= MAXT;
+  // tile descriptor: from the staged list (sparse) or by arithmetic (dense; splits longer than the list)
+  auto get_tile = [&](int idx) -> TileInfo {
+    if (use_list) {
+      const int2 e = tlist[idx];
+      TileInfo ti; ti.kind = e.x >> 30; ti.start = e.x & 0x3FFFFFFF; ti.nvalid = e.y;
+      return ti;
+    }
+    return tile_info(p, te, t0 + idx);
+  };
 
-  __shared__ int s_last;
   if (nt <= 0) {                                          // empty split: publish a neutral partial
     if (p.n_splits > 1) {
       if (warp >= 2) {
@@ -188,21 +216,57 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           p.part_ml[((size_t)cta_lin * TM + row) * 2 + 1] = 0.f;
         }
       }
-      if (p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, &s_last);
+      if (p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p);
     }
     return;
   }
 
   // ---- set-up -------------------------------------------------------------------------------------
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < NSLOT; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pready(b), 128); }
-    mbar_init(bar_pvdone, 1);
-    *abort_flag = 0;
-    fence_barrier_init();
-    fence_proxy_async();
-    prefetch_tmap(&tmK); prefetch_tmap(&tmV);
-    if (!p.dense && p.ns_pad > 0) { prefetch_tmap(&tmSK); prefetch_tmap(&tmSV); }
+  // Warp 0 arms the barriers, stages the tile list and puts the first ring-full of K/V tiles in flight right
+  // away: those copies need nothing from the other warps, which meanwhile allocate TMEM and stage Q.
+  // Load sequence q -> (tile, K or V), the order the MMA warp consumes: K0, K1, V0, K2, V1, ..., V(nt-1).
+  auto seq_tile = [&](int q, bool& isV) -> int {
+    if (q == 0) { isV = false; return 0; }
+    if (q == 2 * nt - 1) { isV = true; return nt - 1; }
+    if (q & 1) { isV = false; return (q + 1) >> 1; }
+    isV = true; return (q >> 1) - 1;
+  };
+  auto issue = [&](int q) {
+    bool isV;
+    const int idx = seq_tile(q, isV);
+    const TileInfo ti = get_tile(idx);
+    const int slot = q % NSLOT;
+    const CUtensorMap* map = ti.kind ? (isV ? &tmSV : &tmSK) : (isV ? &tmV : &tmK);
+    const uint32_t dst = sSlot + slot * SLOT_BYTES;
+    mbar_expect_tx(bar_full(slot), SLOT_BYTES);
+    tma_load_3d(dst, map, bar_full(slot), 0, ti.start, g);
+    tma_load_3d(dst + HALF_BYTES, map, bar_full(slot), 64, ti.start, g);
+  };
+  const int n_loads = 2 * nt;
+  const int n_early = n_loads < NSLOT ? n_loads : NSLOT;
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int s = 0; s < NSLOT; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+      for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pready(b), 128); }
+      mbar_init(bar_pvdone, 1);
+      *abort_flag = 0;
+      fence_barrier_init();
+      fence_proxy_async();
+    }
+    if (use_list) {
+      for (int t = lane; t < nt; t += 32) {
+        const TileInfo ti = tile_info(p, te, t0 + t);
+        if (t0 + t < te.n_blk) {
+          const int b = te.blocks[t0 + t];
+          if (b < 0 || b >= p.nb) set_status(p.status, FOCUS_ERR_INVALID_ARG);
+        }
+        tlist[t] = make_int2(ti.start | (ti.kind << 30), ti.nvalid);
+      }
+    }
+    __syncwarp();
+    if (lane == 0)
+      for (int q = 0; q < n_early; ++q) issue(q);
+    __syncwarp();
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_holder), 512);
@@ -238,31 +302,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   if (warp == 0) {
     // ================================ TMA producer ================================================
     if (lane == 0) {
-      uint32_t q = 0;
-      int issued = 0;
-      auto load = [&](int t, bool isV) -> bool {
-        const int slot = q % NSLOT;
-        const uint32_t ph = (q / NSLOT) & 1u;
-        if (!mbar_wait(bar_empty(slot), ph ^ 1u, abort_flag, p.status)) return false;
-        const TileInfo ti = tile_info(p, te, t);
-        if (!p.dense && !isV && t < te.n_blk) {
-          const int b = te.blocks[t];
-          if (b < 0 || b >= p.nb) set_status(p.status, FOCUS_ERR_INVALID_ARG);
-        }
-        const CUtensorMap* map = ti.kind ? (isV ? &tmSV : &tmSK) : (isV ? &tmV : &tmK);
-        const uint32_t dst = sSlot + slot * SLOT_BYTES;
-        mbar_expect_tx(bar_full(slot), SLOT_BYTES);
-        tma_load_3d(dst, map, bar_full(slot), 0, ti.start, g);
-        tma_load_3d(dst + HALF_BYTES, map, bar_full(slot), 64, ti.start, g);
-        ++q; ++issued;
-        return true;
-      };
+      int issued = n_early;
       bool ok = true;
-      for (int j = t0; j < t1 && ok; ++j) {
-        ok = load(j, false);
-        if (ok && j > t0) ok = load(j - 1, true);
+      for (int q = n_early; q < n_loads; ++q) {
+        if (!mbar_wait(bar_empty(q % NSLOT), (uint32_t)((q / NSLOT) & 1) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        issue(q);
+        ++issued;
       }
-      if (ok) ok = load(t1 - 1, true);
       if (!ok) {
         // unwinding: let the copies already issued land before the CTA's shared memory is released
         const uint32_t first = issued > NSLOT ? (uint32_t)(issued - NSLOT) : 0u;
@@ -337,7 +383,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       TC_LD32(ts + 64, (sreg + 64));
       TC_LD32(ts + 96, (sreg + 96));
       tc_wait_ld();
-      const TileInfo ti = tile_info(p, te, t0 + idx);
+      const TileInfo ti = get_tile(idx);
       float tmax = -INFINITY;
       if (ti.kind == 0 && ti.nvalid == TN) {
 #pragma unroll
@@ -464,7 +510,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     __syncwarp();
     tmem_dealloc(tmem, 512);
   }
-  if (p.n_splits > 1 && p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, &s_last);
+  if (p.n_splits > 1 && p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p);
 }
 
 // Stand-alone merge (used when there are more query tiles than arrival counters): out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s, one warp per stacked row.
