@@ -62,13 +62,13 @@ struct TileEnum {
   const int32_t* blocks;
 };
 
-__device__ __forceinline__ TileEnum make_enum(const TcParams& p, int g) {
+__device__ __forceinline__ TileEnum make_enum(const TcParams& p, int g, int cnt_raw) {
   TileEnum e;
   if (p.dense) {
     e.n_blk = 0; e.n_sinkt = 0; e.n_resp = (p.L + TN - 1) / TN; e.blocks = nullptr;
   } else {
     const int row = g * p.group_stride;
-    e.n_blk = min(max(p.block_cnt[row], 0), p.max_blocks);
+    e.n_blk = min(max(cnt_raw, 0), p.max_blocks);
     e.n_sinkt = p.ns_pad / TN;
     e.n_resp = (p.L - p.M + TN - 1) / TN;
     e.blocks = p.block_idx + (size_t)row * p.max_blocks;
@@ -100,59 +100,61 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams& p, const TileEnum&
 }
 
 // Merge of the split partials of one (KV head, query tile): out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s,
-// splits taken in index order (deterministic whoever runs it).  One warp per stacked row.
-__device__ __forceinline__ void merge_rows(const TcParams& p, int tile, int g, int mt, int total_fr, int warp,
-                                           int n_warps, int lane) {
+// splits taken in index order (deterministic whoever runs it).  Every step is an L2 round trip, so the work is
+// laid out as two flat phases with many independent loads in flight: (1) one thread per row turns the per-split
+// (max, sum) pairs into weights in shared memory, (2) one thread per (row, 4 columns) accumulates the outputs.
+__device__ __forceinline__ void merge_rows(const TcParams& p, int tile, int g, int mt, int total_fr, float* wts) {
   const int rows = min(TM, total_fr - mt * TM);
-  for (int row = warp; row < rows; row += n_warps) {
-    // the merge is a chain of L2 latencies: read the per-split (max, sum) pairs lane-parallel, and keep four
-    // partial-output loads in flight at a time; the accumulation order stays s = 0, 1, 2, ...
+  const int S = p.n_splits;
+  float* inv_s = wts + TM * S;
+  for (int row = threadIdx.x; row < rows; row += NTHREADS) {
+    const float2* ml = reinterpret_cast<const float2*>(p.part_ml) + (size_t)tile * S * TM + row;
     float m = -INFINITY;
-    for (int s0 = 0; s0 < p.n_splits; s0 += 32) {
-      const int s = s0 + lane;
-      if (s < p.n_splits) {
-        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((size_t)(tile * p.n_splits + s) * TM + row) * 2));
-        if (ml.y > 0.f) m = fmaxf(m, ml.x);
-      }
+#pragma unroll 4
+    for (int s = 0; s < S; ++s) {
+      const float2 v = __ldcg(ml + (size_t)s * TM);
+      if (v.y > 0.f) m = fmaxf(m, v.x);
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     float tot = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s0 = 0; s0 < p.n_splits; s0 += 4) {
-      float2 ml[4];
-      float4 o[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int s = min(s0 + u, p.n_splits - 1);
-        const size_t base = (size_t)(tile * p.n_splits + s) * TM + row;
-        ml[u] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + base * 2));
-        o[u] = __ldcg(reinterpret_cast<const float4*>(p.part_O + base * HD + lane * 4));
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (s0 + u >= p.n_splits || !(ml[u].y > 0.f)) continue;
-        const float wgt = exp2f(ml[u].x - m);
-        tot += wgt * ml[u].y;
-        acc.x += wgt * o[u].x; acc.y += wgt * o[u].y; acc.z += wgt * o[u].z; acc.w += wgt * o[u].w;
-      }
+#pragma unroll 4
+    for (int s = 0; s < S; ++s) {
+      const float2 v = __ldcg(ml + (size_t)s * TM);
+      const float wgt = v.y > 0.f ? exp2f(v.x - m) : 0.f;
+      tot += wgt * v.y;
+      wts[row * S + s] = wgt;
     }
-    const float inv = tot > 0.f ? 1.f / tot : 0.f;
+    inv_s[row] = tot > 0.f ? 1.f / tot : 0.f;
+    if (p.lse) {
+      const int fr = mt * TM + row;
+      p.lse[(size_t)(g * p.hpg + fr % p.hpg) * p.lse_stride + fr / p.hpg] = (m + log2f(tot)) * 0.6931471805599453f;
+    }
+  }
+  __syncthreads();
+#pragma unroll 2
+  for (int item = threadIdx.x; item < rows * 32; item += NTHREADS) {
+    const int row = item >> 5, cg = item & 31;
+    const float4* po = reinterpret_cast<const float4*>(p.part_O) + ((size_t)tile * S * TM + row) * (HD / 4) + cg;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 4
+    for (int s = 0; s < S; ++s) {
+      const float wgt = wts[row * S + s];
+      const float4 o = __ldcg(po + (size_t)s * TM * (HD / 4));
+      if (wgt > 0.f) { acc.x += wgt * o.x; acc.y += wgt * o.y; acc.z += wgt * o.z; acc.w += wgt * o.w; }
+    }
+    const float inv = inv_s[row];
     const int fr = mt * TM + row;
-    const int qr = fr / p.hpg, hh = fr % p.hpg;
-    __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD + lane * 4;
+    __nv_bfloat16* orow = p.O + ((size_t)(fr / p.hpg) * p.H + (size_t)(g * p.hpg + fr % p.hpg)) * HD + cg * 4;
     uint2 v;
     v.x = pack_bf16(acc.x * inv, acc.y * inv);
     v.y = pack_bf16(acc.z * inv, acc.w * inv);
     *reinterpret_cast<uint2*>(orow) = v;
-    if (p.lse && lane == 0)
-      p.lse[(size_t)(g * p.hpg + hh) * p.lse_stride + qr] = (m + log2f(tot)) * 0.6931471805599453f;
   }
 }
 
 // Called by every thread of every split CTA once its partial is written: the CTA that arrives last at the
 // tile's counter merges all splits and re-arms the counter for the next launch.
-__device__ __forceinline__ void finish_split(const TcParams& p, int tile, int g, int mt, int total_fr, int* s_last) {
+__device__ __forceinline__ void finish_split(const TcParams& p, int tile, int g, int mt, int total_fr, int* s_last,
+                                             float* wts) {
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -162,7 +164,7 @@ __device__ __forceinline__ void finish_split(const TcParams& p, int tile, int g,
     __threadfence();
   }
   __syncthreads();
-  if (*s_last) merge_rows(p, tile, g, mt, total_fr, threadIdx.x >> 5, NTHREADS / 32, threadIdx.x & 31);
+  if (*s_last) merge_rows(p, tile, g, mt, total_fr, wts);
 }
 
 __global__ void __launch_bounds__(NTHREADS, 1)
@@ -172,11 +174,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
 
-  const int nrows = p.q_rows ? min(max(*p.n_rows, 0), p.rows_bound) : p.n_q;
+  // The prologue is a chain of global-memory latencies; everything that does not depend on another load is
+  // requested first: the row count, this group's block count, the positions of this thread's Q rows.
+  constexpr int QIT = (TM * 16 + NTHREADS - 1) / NTHREADS;      // 16-byte chunks of the Q tile per thread
+  const int nrows_raw = p.q_rows ? __ldg(p.n_rows) : p.n_q;
+  const int cnt_raw = p.dense ? 0 : __ldg(p.block_cnt + g * p.group_stride);
+  int qpos[QIT];
+#pragma unroll
+  for (int it = 0; it < QIT; ++it) {
+    const int idx = threadIdx.x + it * NTHREADS;
+    const int qr = (mt * TM + (idx >> 4)) / p.hpg;
+    qpos[it] = (idx < TM * 16 && qr < p.rows_bound) ? (p.q_rows ? __ldg(p.q_rows + qr) : p.q_base + qr) : -1;
+  }
+  const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
   const int total_fr = nrows * p.hpg;                    // stacked (row, head-of-group) rows of this KV head
   if (mt * TM >= total_fr) return;                       // uniform: nothing to compute for this tile
 
-  const TileEnum te = make_enum(p, g);
+  const TileEnum te = make_enum(p, g, cnt_raw);
   const int t0 = (int)(((long long)te.total * split) / p.n_splits);
   const int t1 = (int)(((long long)te.total * (split + 1)) / p.n_splits);
   const int nt = t1 - t0;
@@ -216,7 +230,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           p.part_ml[((size_t)cta_lin * TM + row) * 2 + 1] = 0.f;
         }
       }
-      if (p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p);
+      if (p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p, reinterpret_cast<float*>(sptr + Q_BYTES));
     }
     return;
   }
@@ -274,23 +288,34 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   }
   // Q tile -> shared memory in the 128-byte-swizzled K-major layout the MMA descriptor expects:
   // half h (columns 64h..64h+63) at h*16 KB, row r at r*128 bytes, 16-byte chunk c at ((c ^ (r & 7)) * 16).
-  for (int idx = threadIdx.x; idx < TM * 16; idx += NTHREADS) {
-    const int r = idx >> 4, c = idx & 15;
-    const int fr = mt * TM + r;
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (fr < total_fr) {
-      const int qr = fr / p.hpg, hh = fr % p.hpg;
-      const int pos = p.q_rows ? p.q_rows[qr] : p.q_base + qr;
-      if (pos >= p.q_base && pos < p.q_base + p.n_q) {
-        const __nv_bfloat16* src = p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
-                                   (long long)(g * p.hpg + hh) * p.q_stride_head + c * 8;
-        v = __ldg(reinterpret_cast<const uint4*>(src));
-      } else if (c == 0) {
-        set_status(p.status, FOCUS_ERR_INVALID_ARG);
+  {
+    uint4 qv[QIT];
+#pragma unroll
+    for (int it = 0; it < QIT; ++it) {
+      const int idx = threadIdx.x + it * NTHREADS;
+      const int r = idx >> 4, c = idx & 15;
+      const int fr = mt * TM + r;
+      qv[it] = make_uint4(0, 0, 0, 0);
+      if (idx < TM * 16 && fr < total_fr) {
+        const int pos = qpos[it];
+        if (pos >= p.q_base && pos < p.q_base + p.n_q) {
+          const __nv_bfloat16* src = p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
+                                     (long long)(g * p.hpg + fr % p.hpg) * p.q_stride_head + c * 8;
+          qv[it] = __ldg(reinterpret_cast<const uint4*>(src));
+        } else if (c == 0) {
+          set_status(p.status, FOCUS_ERR_INVALID_ARG);
+        }
       }
     }
-    const int half = c >> 3, cc = c & 7;
-    *reinterpret_cast<uint4*>(sptr + half * HALF_BYTES + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+#pragma unroll
+    for (int it = 0; it < QIT; ++it) {
+      const int idx = threadIdx.x + it * NTHREADS;
+      if (idx < TM * 16) {
+        const int r = idx >> 4, c = idx & 15;
+        const int half = c >> 3, cc = c & 7;
+        *reinterpret_cast<uint4*>(sptr + half * HALF_BYTES + r * 128 + ((cc ^ (r & 7)) << 4)) = qv[it];
+      }
+    }
   }
   fence_proxy_async();
   tc_fence_before();
@@ -510,7 +535,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     __syncwarp();
     tmem_dealloc(tmem, 512);
   }
-  if (p.n_splits > 1 && p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p);
+  if (p.n_splits > 1 && p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p, reinterpret_cast<float*>(sptr + Q_BYTES));
 }
 
 // Stand-alone merge (used when there are more query tiles than arrival counters): out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s, one warp per stacked row.
@@ -662,7 +687,8 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.Q = (const __nv_bfloat16*)a.Q; p.O = (__nv_bfloat16*)a.O; p.lse = a.lse;
   p.q_rows = a.q_rows; p.n_rows = a.n_rows; p.block_idx = a.block_idx; p.block_cnt = a.block_cnt;
   p.sink_mask = mask; p.part_O = part_O; p.part_ml = part_ml;
-  p.counters = (n_splits > 1 && base <= FOCUS_N_COUNTERS) ? ctx->d_counters : nullptr;
+  p.counters = (n_splits > 1 && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
+                   ? ctx->d_counters : nullptr;
   p.q_stride_row = sh.q_stride_row; p.q_stride_head = sh.q_stride_head;
   p.q_base = a.q_base; p.n_q = a.n_q; p.rows_bound = a.max_rows; p.L = sh.L; p.M = sh.M; p.H = sh.n_q_heads;
   p.Hkv = Hkv; p.hpg = hpg; p.B = sh.kv_block; p.nb = shape_nb(&sh); p.dense = a.dense;
