@@ -13,6 +13,8 @@
 //                 (aliasing S_b), lazy rescale of O, final normalisation and the epilogue
 // Split partials (unnormalised O, running max, running sum) go to scratch and are merged by a second kernel in
 // fixed split order, so results are deterministic.
+#include <stdlib.h>
+
 #include "tc_common.cuh"
 
 using namespace tc;
@@ -49,7 +51,16 @@ struct TcParams {
   int n_mtiles, n_splits, lse_stride;
   float scale_log2;            // softmax scale * log2(e)
   int32_t* status;
+#ifdef FOCUS_TIMELINE
+  unsigned long long* dbg;     // per-CTA timestamps (development builds only)
+#endif
 };
+
+#ifdef FOCUS_TIMELINE
+#define TL_STAMP(slot, tid) do { if (p.dbg && threadIdx.x == (tid)) p.dbg[(blockIdx.x * gridDim.y + blockIdx.y) * 8 + (slot)] = global_ns(); } while (0)
+#else
+#define TL_STAMP(slot, tid) do { } while (0)
+#endif
 
 struct TileInfo {
   int kind;     // 0: tile of the K/V tensors, 1: tile of the gathered sink rows
@@ -173,6 +184,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   extern __shared__ uint8_t smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
+  TL_STAMP(0, 0);
 
   // The prologue is a chain of global-memory latencies; everything that does not depend on another load is
   // requested first: the row count, this group's block count, the positions of this thread's Q rows.
@@ -281,10 +293,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     if (lane == 0)
       for (int q = 0; q < n_early; ++q) issue(q);
     __syncwarp();
+    TL_STAMP(6, 0);
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_holder), 512);
     tmem_relinquish();
+    TL_STAMP(7, 32);
   }
   // Q tile -> shared memory in the 128-byte-swizzled K-major layout the MMA descriptor expects:
   // half h (columns 64h..64h+63) at h*16 KB, row r at r*128 bytes, 16-byte chunk c at ((c ^ (r & 7)) * 16).
@@ -323,6 +337,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem = *tmem_holder;
   const uint32_t tmem_O = tmem + 256;
+  TL_STAMP(1, 0);
 
   if (warp == 0) {
     // ================================ TMA producer ================================================
@@ -401,6 +416,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       // votes keep the warp together: the TMEM loads and stores below are warp-collective
       if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(b), (uint32_t)(idx >> 1) & 1u, abort_flag, p.status))) { ok = false; break; }
       tc_fence_after();
+      if (idx == 0) TL_STAMP(5, 64);
       uint32_t sreg[128];
       const uint32_t ts = tmem + lane_off + b * 128;
       TC_LD32(ts, (sreg + 0));
@@ -528,6 +544,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
     }
   }
+  TL_STAMP(2, 64);
   // ---- teardown: every role converges here, also after a timed-out wait --------------------------
   tc_fence_before();
   __syncthreads();
@@ -535,7 +552,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     __syncwarp();
     tmem_dealloc(tmem, 512);
   }
+  TL_STAMP(3, 0);
   if (p.n_splits > 1 && p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p, reinterpret_cast<float*>(sptr + Q_BYTES));
+  TL_STAMP(4, 0);
 }
 
 // Stand-alone merge (used when there are more query tiles than arrival counters): out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s, one warp per stacked row.
@@ -696,6 +715,9 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.n_mtiles = n_mtiles; p.n_splits = n_splits; p.lse_stride = a.lse_stride;
   p.scale_log2 = a.scale * 1.4426950408889634f;
   p.status = ctx->d_status;
+#ifdef FOCUS_TIMELINE
+  p.dbg = getenv("FOCUS_TIMELINE") ? (unsigned long long*)(ctx->ws + ctx->ws_bytes - (1 << 20)) : nullptr;
+#endif
 
   static bool attr_set = false;
   if (!attr_set) {

@@ -187,3 +187,8 @@ extern "C" focus_status focus_find_sinks(focus_ctx* ctx, const focus_shape* shap
   if (s != FOCUS_OK) return s;
   return launch_sink_select(ctx, part, H, L, n_active, S, cand_lo, cand_hi, n_sink, sink_idx, stream);
 }
+
+#ifdef FOCUS_TIMELINE
+// Development builds only: where the attention kernel drops its per-CTA timestamps (last MiB of the workspace).
+extern "C" void* focus_debug_ptr(focus_ctx* ctx) { return ctx->ws + ctx->ws_bytes - (1 << 20); }
+#endif
