@@ -150,6 +150,25 @@ def test_planted_sinks_recovered_small_config(cfg):
     assert all(S[p] > 1.5 * tau for p in t["sink_pos"])
 
 
+def test_config0_literal_generator_sinks_sit_inside_the_band():
+    """With the literal recipe (keys x8, unshifted queries) a planted sink carries only a fraction of a percent
+    more attention mass than an ordinary key, i.e. less than the 1e-3 relative band around the selection
+    threshold can resolve; the shifted-query variant used everywhere else separates them by ~2x."""
+    w = wl.config(0)
+    s = w.shape
+    c_prev, _ = wl.gen_confidence(w.seed, s.N)
+    conf, masked = wl.full_conf(s, c_prev), wl.gen_masked(w)
+    _, active = fo.select_queries(conf, masked, w.blk_lo, w.blk_hi, w.k, w.w, s.M, s.L)
+    ratios = {}
+    for variant in ("lit", "fix"):
+        t = wl.gen_qkv(s, w.seed, variant=variant)
+        S = fo.sink_scores(wl.storage_to_f64(t["Q"], s.dtype)[active - s.M], wl.storage_to_f64(t["K"], s.dtype), 1.0 / math.sqrt(s.d))
+        tau = np.sort(S[:s.M])[::-1][w.n_sink - 1]
+        ratios[variant] = min(S[p] for p in t["sink_pos"]) / tau
+    assert ratios["fix"] > 1.5
+    assert ratios["lit"] < 1.05
+
+
 def test_find_sinks_brute_force():
     rng = np.random.default_rng(7)
     for _ in range(20):
