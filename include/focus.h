@@ -143,6 +143,32 @@ focus_status focus_score_blocks(focus_ctx* ctx, const focus_shape* shape, const 
                                 const void* K, const float* Kbar, int32_t head_reduce,
                                 float* R, focus_stream stream);
 
+/* focus_score_blocks for callers that cannot allocate device memory.  (The paper has no counterpart: this is a
+ * deployment variant of the Eq. 7 scorer above, computing the same R.)
+ *
+ * Who needs it: code that runs inside another component's memory budget (a serving process whose pool already
+ * owns the GPU), code for which cudaMalloc's implicit synchronisation is off limits, or a plug-in that is given a
+ * stream and buffers and nothing else.  Such callers cannot call focus_create, which allocates the workspace, so
+ * this entry point takes no context, and it calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * Its scratch (the mean focus query per KV head; in FOCUS_HEADS_ALL mode also the per-group scores) is a fixed
+ * 288.25 KiB array inside the library that every GPU loading the library holds until the process exits.  Limits,
+ * rejected with FOCUS_ERR_WORKSPACE_TOO_SMALL before anything is launched: n_kv_heads * head_dim <= 8192 and, in
+ * FOCUS_HEADS_ALL mode, n_kv_heads * nb <= 65536.
+ *
+ * The first call on each device looks up the array's device address (that device must be current); make that
+ * first call before any stream capture begins.  All calls share the one array and it keeps the previous call's
+ * contents; every element a call reads it has first rewritten, so nothing needs clearing, but two calls whose
+ * kernels overlap on the GPU (different streams, or several processes' worth of threads on one context) race on
+ * it: serialise them.
+ *
+ * Arguments as focus_score_blocks, minus the context; device_status (device int32, caller-owned) receives the
+ * code of a device-side anomaly (bad focus index, empty focus set) or may be NULL. */
+focus_status focus_score_blocks_static(const focus_shape* shape, const void* Q, int32_t q_base,
+                                       const int32_t* focus_idx, const int32_t* n_focus, int32_t max_focus,
+                                       const void* K, const float* Kbar, int32_t head_reduce,
+                                       float* R, int32_t* device_status, focus_stream stream);
+
 /* Per row g of R: the C highest-scoring blocks (ties: lower index), ascending, into
  * block_idx[g*max_blocks ...] (padded -1), count into block_cnt[g].
  * SINK_TOKENS: sink_keep[g*n_sink + s] = 1 iff sink token s lies outside every selected block of g.

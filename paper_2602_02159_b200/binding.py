@@ -47,6 +47,7 @@ _SIGS = {
     "focus_find_sinks": (_I, [_P, _SH, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _P, _P, _P]),
     "focus_pool_keys": (_I, [_P, _SH, _P, _P, _P]),
     "focus_score_blocks": (_I, [_P, _SH, _P, _I, _P, _P, _I, _P, _P, _I, _P, _P]),
+    "focus_score_blocks_static": (_I, [_SH, _P, _I, _P, _P, _I, _P, _P, _I, _P, _P, _P]),
     "focus_select_blocks": (_I, [_P, _SH, _P, _I, _I, _P, _I, _I, _P, _I, _P, _P, _P]),
     "focus_sparse_attn": (_I, [_P, _SH, _P, _I, _I, _P, _P, _I, _P, _P, _I, _P, _I, _P, _P, _P, _I, _P, _P, _P]),
     "focus_sparse_layer": (_I, [_P, _SH, _P, _I, _I, _P, _P, _I, _P, _P, _I, _P, _P, _P, _I, _P, _I, _P, _P, _P, _P, _P,
@@ -173,6 +174,17 @@ def focus_score_blocks(ctx, shape, Q, q_base, focus_idx, n_focus, max_focus, K, 
     _check(ctx._lib.focus_score_blocks(ctx.handle, C.byref(shape), _ptr(Q), q_base, _ptr(focus_idx), _ptr(n_focus),
                                        max_focus, _ptr(K), _ptr(Kbar), head_reduce, _ptr(R), _stream(stream)),
            "focus_score_blocks")
+
+
+def focus_score_blocks_static(shape, Q, q_base, focus_idx, n_focus, max_focus, K, Kbar, head_reduce, R,
+                              device_status=None, stream=None):
+    """Block relevance (Eq. 7) without a context and without any allocation: for callers that live inside someone
+    else's memory budget.  Scratch is a fixed array inside the library (limits in include/focus.h); calls that
+    overlap on the GPU race on it, and the first call on a device should precede any stream capture."""
+    _check(load_library().focus_score_blocks_static(C.byref(shape), _ptr(Q), q_base, _ptr(focus_idx), _ptr(n_focus),
+                                                    max_focus, _ptr(K), _ptr(Kbar), head_reduce, _ptr(R),
+                                                    _ptr(device_status), _stream(stream)),
+           "focus_score_blocks_static")
 
 
 def focus_select_blocks(ctx, shape, R, head_reduce, C_keep, sink_idx, n_sink, sink_mode, block_idx, max_blocks,

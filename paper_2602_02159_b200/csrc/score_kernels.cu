@@ -176,3 +176,83 @@ extern "C" focus_status focus_score_blocks(focus_ctx* ctx, const focus_shape* sh
   }
   return FOCUS_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant of focus_score_blocks.
+//
+// Written for callers that must never allocate device memory: code running inside someone else's memory
+// budget (an inference server whose pool already owns the whole GPU), code on a path where cudaMalloc's
+// implicit device synchronisation is unacceptable, or a plug-in that is handed a stream and nothing else.
+// Such callers cannot create a focus_ctx either (focus_create allocates the workspace), so this entry point
+// takes no context.  Its scratch -- the mean focus query of every KV head and, in all-heads mode, the
+// per-group scores before they are averaged -- lives in the fixed array below, which every GPU that loads the
+// library holds until the process exits.
+// ------------------------------------------------------------------------------------------------
+constexpr int STATIC_QBAR_FLOATS = 64 * 128;        // n_kv_heads * head_dim        <= 8192
+constexpr int STATIC_RG_FLOATS = 64 * 1024;         // n_kv_heads * nb (ALL mode)   <= 65536
+constexpr int STATIC_SCRATCH_FLOATS = STATIC_QBAR_FLOATS + STATIC_RG_FLOATS + 64;   // + status word; 288.25 KiB
+
+static __device__ __align__(256) float g_static_scratch[STATIC_SCRATCH_FLOATS];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel may use: the device
+// address is looked up once per device (with that device current) and cached here.
+constexpr int STATIC_MAX_DEVICES = 64;
+static float* g_static_scratch_dev[STATIC_MAX_DEVICES] = {nullptr};
+
+static focus_status static_scratch_ptr(float** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) return FOCUS_ERR_CUDA;
+  if (!g_static_scratch_dev[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return FOCUS_ERR_CUDA;
+    g_static_scratch_dev[dev] = static_cast<float*>(p);
+  }
+  *out = g_static_scratch_dev[dev];
+  return FOCUS_OK;
+}
+
+extern "C" focus_status focus_score_blocks_static(const focus_shape* shape, const void* Q, int32_t q_base,
+                                                  const int32_t* focus_idx, const int32_t* n_focus,
+                                                  int32_t max_focus, const void* K, const float* Kbar,
+                                                  int32_t head_reduce, float* R, int32_t* device_status,
+                                                  focus_stream stream) {
+  if (!shape_ok_basic(shape) || !Q || !focus_idx || !n_focus || !R) return FOCUS_ERR_INVALID_ARG;
+  if ((K == nullptr) == (Kbar == nullptr)) return FOCUS_ERR_INVALID_ARG;
+  if (max_focus <= 0 || q_base < 0 || q_base > shape->L) return FOCUS_ERR_INVALID_ARG;
+  if (head_reduce != FOCUS_HEADS_PER_KV_GROUP && head_reduce != FOCUS_HEADS_ALL) return FOCUS_ERR_INVALID_ARG;
+  if (!shape_supported(shape)) return FOCUS_ERR_UNSUPPORTED;
+  const int G = shape->n_kv_heads, d = shape->head_dim, nb = shape_nb(shape), hpg = shape->n_q_heads / G;
+  // the fixed scratch bounds the problem size: refuse anything that would not fit
+  if ((long long)G * d > STATIC_QBAR_FLOATS) return FOCUS_ERR_WORKSPACE_TOO_SMALL;
+  if (head_reduce == FOCUS_HEADS_ALL && (long long)G * nb > STATIC_RG_FLOATS) return FOCUS_ERR_WORKSPACE_TOO_SMALL;
+  float* scratch = nullptr;
+  focus_status st = static_scratch_ptr(&scratch);
+  if (st != FOCUS_OK) return st;
+  float* qbar = scratch;                                         // fully rewritten by every call
+  float* Rg = head_reduce == FOCUS_HEADS_ALL ? scratch + STATIC_QBAR_FLOATS : R;
+  int32_t* status = device_status ? device_status
+                                  : reinterpret_cast<int32_t*>(scratch + STATIC_QBAR_FLOATS + STATIC_RG_FLOATS);
+  if (shape->dtype == FOCUS_BF16)
+    qbar_kernel<__nv_bfloat16><<<G, 128, 0, stream>>>((const __nv_bfloat16*)Q, q_base, 0, shape->q_stride_row,
+                                                      shape->q_stride_head, focus_idx, n_focus, max_focus, hpg, d,
+                                                      shape->L, qbar, status);
+  else
+    qbar_kernel<float><<<G, 128, 0, stream>>>((const float*)Q, q_base, 0, shape->q_stride_row, shape->q_stride_head,
+                                              focus_idx, n_focus, max_focus, hpg, d, shape->L, qbar, status);
+  FOCUS_CHECK_LAUNCH();
+  if (nb == 0) return FOCUS_OK;
+  if (K) {
+    st = shape->dtype == FOCUS_BF16 ? pool_score_launch<__nv_bfloat16>(shape, K, nullptr, qbar, Rg, stream)
+                                    : pool_score_launch<float>(shape, K, nullptr, qbar, Rg, stream);
+    if (st != FOCUS_OK) return st;
+  } else {
+    const int warps = nb * G;
+    score_from_kbar_kernel<<<(warps * 32 + 255) / 256, 256, 0, stream>>>(Kbar, qbar, nb, d, G, Rg);
+    FOCUS_CHECK_LAUNCH();
+  }
+  if (head_reduce == FOCUS_HEADS_ALL) {
+    reduce_groups_kernel<<<(nb + 255) / 256, 256, 0, stream>>>(Rg, G, nb, R);
+    FOCUS_CHECK_LAUNCH();
+  }
+  return FOCUS_OK;
+}
