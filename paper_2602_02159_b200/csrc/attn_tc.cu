@@ -188,15 +188,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 
   // The prologue is a chain of global-memory latencies; everything that does not depend on another load is
   // requested first: the row count, this group's block count, the positions of this thread's Q rows.
-  constexpr int QIT = (TM * 16 + NTHREADS - 1) / NTHREADS;      // 16-byte chunks of the Q tile per thread
+  constexpr int QTHREADS = 128;                                  // the four softmax warps stage Q
+  constexpr int QIT = TM * 16 / QTHREADS;                        // 16-byte chunks of the Q tile per staging thread
+  const int qtid = (int)threadIdx.x - 64;
   const int nrows_raw = p.q_rows ? __ldg(p.n_rows) : p.n_q;
   const int cnt_raw = p.dense ? 0 : __ldg(p.block_cnt + g * p.group_stride);
   int qpos[QIT];
 #pragma unroll
   for (int it = 0; it < QIT; ++it) {
-    const int idx = threadIdx.x + it * NTHREADS;
+    const int idx = qtid + it * QTHREADS;
     const int qr = (mt * TM + (idx >> 4)) / p.hpg;
-    qpos[it] = (idx < TM * 16 && qr < p.rows_bound) ? (p.q_rows ? __ldg(p.q_rows + qr) : p.q_base + qr) : -1;
+    qpos[it] = (qtid >= 0 && qr < p.rows_bound) ? (p.q_rows ? __ldg(p.q_rows + qr) : p.q_base + qr) : -1;
   }
   const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
   const int total_fr = nrows * p.hpg;                    // stacked (row, head-of-group) rows of this KV head
@@ -302,15 +304,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   }
   // Q tile -> shared memory in the 128-byte-swizzled K-major layout the MMA descriptor expects:
   // half h (columns 64h..64h+63) at h*16 KB, row r at r*128 bytes, 16-byte chunk c at ((c ^ (r & 7)) * 16).
-  {
+  if (qtid >= 0) {
     uint4 qv[QIT];
 #pragma unroll
     for (int it = 0; it < QIT; ++it) {
-      const int idx = threadIdx.x + it * NTHREADS;
+      const int idx = qtid + it * QTHREADS;
       const int r = idx >> 4, c = idx & 15;
       const int fr = mt * TM + r;
       qv[it] = make_uint4(0, 0, 0, 0);
-      if (idx < TM * 16 && fr < total_fr) {
+      if (fr < total_fr) {
         const int pos = qpos[it];
         if (pos >= p.q_base && pos < p.q_base + p.n_q) {
           const __nv_bfloat16* src = p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
@@ -323,12 +325,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     }
 #pragma unroll
     for (int it = 0; it < QIT; ++it) {
-      const int idx = threadIdx.x + it * NTHREADS;
-      if (idx < TM * 16) {
-        const int r = idx >> 4, c = idx & 15;
-        const int half = c >> 3, cc = c & 7;
-        *reinterpret_cast<uint4*>(sptr + half * HALF_BYTES + r * 128 + ((cc ^ (r & 7)) << 4)) = qv[it];
-      }
+      const int idx = qtid + it * QTHREADS;
+      const int r = idx >> 4, c = idx & 15;
+      const int half = c >> 3, cc = c & 7;
+      *reinterpret_cast<uint4*>(sptr + half * HALF_BYTES + r * 128 + ((cc ^ (r & 7)) << 4)) = qv[it];
     }
   }
   fence_proxy_async();

@@ -162,16 +162,33 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
       tc_fence_after();
       const float* nl = neg_lse2 + hh * p.n_pad;
       float acc = 0.f;
-      for (int c0 = 0; c0 < n; c0 += 16) {
-        uint32_t r[16];
-        TC_LD16(tmem + lane_off + b * 256 + c0, r);
+      const uint32_t tsrc = tmem + lane_off + b * 256;
+      if (p.n_pad <= 64) {
+        // common case (at most 64 active rows per head): every column chunk is requested before the single wait,
+        // and the accumulator buffer goes back to the MMA warp before the exponentials are taken
+        uint32_t r[64];
+        TC_LD16(tsrc, (r + 0));
+        if (p.n_pad > 16) TC_LD16(tsrc + 16, (r + 16));
+        if (p.n_pad > 32) TC_LD16(tsrc + 32, (r + 32));
+        if (p.n_pad > 48) TC_LD16(tsrc + 48, (r + 48));
         tc_wait_ld();
+        tc_fence_before();
+        mbar_arrive(bar_sempty(b));
 #pragma unroll
-        for (int c = 0; c < 16; ++c)
-          if (c0 + c < n) acc += ex2(fmaf(__uint_as_float(r[c]), p.scale_log2, nl[c0 + c]));
+        for (int c = 0; c < 64; ++c)
+          if (c < n) acc += ex2(fmaf(__uint_as_float(r[c]), p.scale_log2, nl[c]));
+      } else {
+        for (int c0 = 0; c0 < n; c0 += 16) {
+          uint32_t r[16];
+          TC_LD16(tsrc + c0, r);
+          tc_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 16; ++c)
+            if (c0 + c < n) acc += ex2(fmaf(__uint_as_float(r[c]), p.scale_log2, nl[c0 + c]));
+        }
+        tc_fence_before();
+        mbar_arrive(bar_sempty(b));
       }
-      tc_fence_before();
-      mbar_arrive(bar_sempty(b));
       const int key = (t0 + i) * TK + krow;
       if (key < p.L) p.part[(size_t)(g * p.hpg + hh) * p.L + key] = acc;
     }
