@@ -20,6 +20,7 @@ constexpr int HALF_BYTES = SLOT_BYTES / 2;
 constexpr int NTHREADS = 192;
 constexpr int MAX_SLOTS = 6;
 constexpr int MAX_NPAD = 256;
+constexpr int MAX_BUF = 8;              // TMEM accumulator buffers (512 columns / buffer width)
 
 struct SinkParams {
   const __nv_bfloat16* Q;
@@ -29,6 +30,8 @@ struct SinkParams {
   float* part;                  // [H][L]
   long long q_stride_row, q_stride_head;
   int q_base, L, hpg, max_active, n_pad, n_slots, lse_stride, chunks;
+  int n_buf, buf_cols;           // accumulator ring in TMEM: n_buf buffers of buf_cols columns
+  int Hkv, n_ctas, groups_staged; // flat split of the Hkv*T key tiles over n_ctas CTAs; a CTA touches <= groups_staged heads
   float scale_log2;
   int32_t* status;
 };
@@ -45,14 +48,18 @@ __global__ void __launch_bounds__(NTHREADS, 1)
 sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams p) {
   extern __shared__ uint8_t smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = blockIdx.y, chunk = blockIdx.x;
+  // The Hkv * T key tiles (T per KV head) are cut into n_ctas contiguous ranges, one per CTA (one CTA per SM,
+  // every SM busy); a range may cross from one KV head into the next, so the queries of both are staged.
   const int T = (p.L + TK - 1) / TK;
-  const int t0 = (int)(((long long)T * chunk) / p.chunks), t1 = (int)(((long long)T * (chunk + 1)) / p.chunks);
-  const int nt = t1 - t0;
+  const long long U = (long long)p.Hkv * T;
+  const int u0 = (int)(U * blockIdx.x / p.n_ctas), u1 = (int)(U * (blockIdx.x + 1) / p.n_ctas);
+  const int nt = u1 - u0;
   if (nt <= 0) return;
+  const int g0 = u0 / T;
+  const int ngs = min((u1 - 1) / T - g0 + 1, p.groups_staged);
   const int n = min(max(*p.n_active, 0), p.max_active);
   const int q_head_bytes = p.n_pad * 256;              // two swizzled halves of n_pad rows x 128 bytes
-  const int q_bytes = p.hpg * q_head_bytes;
+  const int q_bytes = p.groups_staged * p.hpg * q_head_bytes;
 
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sptr = smem_raw + (sbase - smem_u32(smem_raw));
@@ -62,15 +69,15 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
   auto bar_full = [&](int s) { return sBar + 8u * s; };
   auto bar_empty = [&](int s) { return sBar + 8u * (MAX_SLOTS + s); };
   auto bar_sfull = [&](int b) { return sBar + 8u * (2 * MAX_SLOTS + b); };
-  auto bar_sempty = [&](int b) { return sBar + 8u * (2 * MAX_SLOTS + 2 + b); };
-  uint8_t* tail = sptr + q_bytes + p.n_slots * SLOT_BYTES + (2 * MAX_SLOTS + 4) * 8;
+  auto bar_sempty = [&](int b) { return sBar + 8u * (2 * MAX_SLOTS + MAX_BUF + b); };
+  uint8_t* tail = sptr + q_bytes + p.n_slots * SLOT_BYTES + (2 * MAX_SLOTS + 2 * MAX_BUF) * 8;
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 4);
-  float* neg_lse2 = reinterpret_cast<float*>(tail + 16);       // [hpg][n_pad]: -lse * log2(e)
+  float* neg_lse2 = reinterpret_cast<float*>(tail + 16);       // [staged heads][n_pad]: -lse * log2(e)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.n_slots; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_sempty(b), 128); }
+    for (int b = 0; b < p.n_buf; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_sempty(b), 128); }
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
@@ -80,25 +87,26 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
     tmem_alloc(smem_u32(tmem_holder), 512);
     tmem_relinquish();
   }
-  // query rows of every head of the group -> swizzled K-major B operand; rows >= n are zero
-  for (int idx = threadIdx.x; idx < p.hpg * p.n_pad * 16; idx += NTHREADS) {
-    const int c = idx & 15, r = (idx >> 4) % p.n_pad, hh = (idx >> 4) / p.n_pad;
+  // query rows of every head of the staged group(s) -> swizzled K-major B operand; rows >= n are zero
+  const int heads_staged = ngs * p.hpg;
+  for (int idx = threadIdx.x; idx < heads_staged * p.n_pad * 16; idx += NTHREADS) {
+    const int c = idx & 15, r = (idx >> 4) % p.n_pad, hs = (idx >> 4) / p.n_pad;     // hs = staged head slot
     uint4 v = make_uint4(0, 0, 0, 0);
     if (r < n) {
       const int pos = p.active_idx[r];
       if (pos >= p.q_base && pos < p.L) {
         v = __ldg(reinterpret_cast<const uint4*>(p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
-                                                 (long long)(g * p.hpg + hh) * p.q_stride_head + c * 8));
+                                                 (long long)(g0 * p.hpg + hs) * p.q_stride_head + c * 8));
       } else if (c == 0) {
         set_status(p.status, FOCUS_ERR_INVALID_ARG);
       }
     }
     const int half = c >> 3, cc = c & 7;
-    *reinterpret_cast<uint4*>(sptr + hh * q_head_bytes + half * (p.n_pad * 128) + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
+    *reinterpret_cast<uint4*>(sptr + hs * q_head_bytes + half * (p.n_pad * 128) + r * 128 + ((cc ^ (r & 7)) << 4)) = v;
   }
-  for (int idx = threadIdx.x; idx < p.hpg * p.n_pad; idx += NTHREADS) {
-    const int r = idx % p.n_pad, hh = idx / p.n_pad;
-    neg_lse2[idx] = r < n ? -p.lse[(size_t)(g * p.hpg + hh) * p.lse_stride + r] * 1.4426950408889634f : 0.f;
+  for (int idx = threadIdx.x; idx < heads_staged * p.n_pad; idx += NTHREADS) {
+    const int r = idx % p.n_pad, hs = idx / p.n_pad;
+    neg_lse2[idx] = r < n ? -p.lse[(size_t)(g0 * p.hpg + hs) * p.lse_stride + r] * 1.4426950408889634f : 0.f;
   }
   fence_proxy_async();
   tc_fence_before();
@@ -117,8 +125,9 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
         if (!mbar_wait(bar_empty(slot), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
         const uint32_t dst = sSlot + slot * SLOT_BYTES;
         mbar_expect_tx(bar_full(slot), SLOT_BYTES);
-        tma_load_3d(dst, &tmK, bar_full(slot), 0, (t0 + i) * TK, g);
-        tma_load_3d(dst + HALF_BYTES, &tmK, bar_full(slot), 64, (t0 + i) * TK, g);
+        const int u = u0 + i;
+        tma_load_3d(dst, &tmK, bar_full(slot), 0, (u % T) * TK, u / T);
+        tma_load_3d(dst + HALF_BYTES, &tmK, bar_full(slot), 64, (u % T) * TK, u / T);
         ++issued;
       }
       if (!ok) {
@@ -136,17 +145,18 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
       bool ok = true;
       for (int u = 0; u < units && ok; ++u) {
         const int i = u / p.hpg, hh = u % p.hpg;
-        const int slot = i % p.n_slots, b = u & 1;
-        if (!mbar_wait(bar_sempty(b), ((uint32_t)(u >> 1) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        const int slot = i % p.n_slots, b = u % p.n_buf;
+        if (!mbar_wait(bar_sempty(b), ((uint32_t)(u / p.n_buf) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
         if (hh == 0 && !mbar_wait(bar_full(slot), (uint32_t)(i / p.n_slots) & 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint64_t kdesc = make_sdesc(sSlot + slot * SLOT_BYTES, 16, 1024);
-        const uint64_t qdesc = make_sdesc(sQ + hh * q_head_bytes, 16, 1024);
+        const int hs = ((u0 + i) / T - g0) * p.hpg + hh;
+        const uint64_t qdesc = make_sdesc(sQ + hs * q_head_bytes, 16, 1024);
 #pragma unroll
         for (int half = 0; half < 2; ++half)
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks)
-            mma_ss(tmem + b * 256, kdesc + (uint64_t)((half * HALF_BYTES + ks * 32) >> 4),
+            mma_ss(tmem + b * p.buf_cols, kdesc + (uint64_t)((half * HALF_BYTES + ks * 32) >> 4),
                    qdesc + (uint64_t)((half * (p.n_pad * 128) + ks * 32) >> 4), idesc, (half | ks) ? 1u : 0u);
         tc_commit(bar_sfull(b));
         if (hh == p.hpg - 1) tc_commit(bar_empty(slot));
@@ -157,12 +167,13 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
     const int krow = rq * 32 + lane;                          // key of this thread inside the tile
     const uint32_t lane_off = (uint32_t)(rq * 32) << 16;
     for (int u = 0; u < units; ++u) {
-      const int i = u / p.hpg, hh = u % p.hpg, b = u & 1;
-      if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(b), (uint32_t)(u >> 1) & 1u, abort_flag, p.status))) break;
+      const int i = u / p.hpg, hh = u % p.hpg, b = u % p.n_buf;
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(b), (uint32_t)(u / p.n_buf) & 1u, abort_flag, p.status))) break;
       tc_fence_after();
-      const float* nl = neg_lse2 + hh * p.n_pad;
+      const int g = (u0 + i) / T;
+      const float* nl = neg_lse2 + ((g - g0) * p.hpg + hh) * p.n_pad;
       float acc = 0.f;
-      const uint32_t tsrc = tmem + lane_off + b * 256;
+      const uint32_t tsrc = tmem + lane_off + b * p.buf_cols;
       if (p.n_pad <= 64) {
         // common case (at most 64 active rows per head): every column chunk is requested before the single wait,
         // and the accumulator buffer goes back to the MMA warp before the exponentials are taken
@@ -189,7 +200,7 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
         tc_fence_before();
         mbar_arrive(bar_sempty(b));
       }
-      const int key = (t0 + i) * TK + krow;
+      const int key = ((u0 + i) % T) * TK + krow;
       if (key < p.L) p.part[(size_t)(g * p.hpg + hh) * p.L + key] = acc;
     }
   }
@@ -204,8 +215,8 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
 }  // namespace
 
 static int sink_npad(int max_active) { return (max_active + 15) / 16 * 16; }
-static int sink_slots(int hpg, int n_pad) {
-  const int fixed = 1024 + hpg * n_pad * 256 + (2 * MAX_SLOTS + 4) * 8 + 16 + hpg * n_pad * 4 + 64;
+static int sink_slots(int heads_staged, int n_pad) {
+  const int fixed = 1024 + heads_staged * n_pad * 256 + (2 * MAX_SLOTS + 2 * MAX_BUF) * 8 + 16 + heads_staged * n_pad * 4 + 64;
   int s = (232448 - fixed) / SLOT_BYTES;
   return s > MAX_SLOTS ? MAX_SLOTS : s;
 }
@@ -224,26 +235,43 @@ focus_status launch_sink_colsum_tc(focus_ctx* ctx, const focus_shape* s, const v
   p.Q = (const __nv_bfloat16*)Q; p.active_idx = active_idx; p.n_active = n_active; p.lse = lse; p.part = part;
   p.q_stride_row = s->q_stride_row; p.q_stride_head = s->q_stride_head;
   p.q_base = q_base; p.L = s->L; p.hpg = hpg; p.max_active = max_active; p.n_pad = sink_npad(max_active);
-  p.n_slots = sink_slots(hpg, p.n_pad); p.lse_stride = max_active;
+  p.lse_stride = max_active;
+  p.buf_cols = p.n_pad <= 64 ? 64 : (p.n_pad <= 128 ? 128 : 256);
+  p.n_buf = 512 / p.buf_cols;
   const int T = (s->L + TK - 1) / TK;
-  int chunks = ctx->sm_count / Hkv;
-  if (chunks < 1) chunks = 1;
-  if (chunks > T) chunks = T;
-  p.chunks = chunks;
+  // one CTA per SM over the flat tile range when the queries of two KV heads fit beside >= 4 ring slots and no
+  // range can span more than two heads; otherwise whole chunks of single heads
+  p.Hkv = Hkv;
+  const long long U = (long long)Hkv * T;
+  if (sink_slots(2 * hpg, p.n_pad) >= 4 && U / ctx->sm_count + 1 <= T && U >= ctx->sm_count) {
+    p.groups_staged = 2;
+    p.n_ctas = ctx->sm_count;
+  } else {
+    p.groups_staged = 1;
+    int chunks = ctx->sm_count / Hkv;
+    if (chunks < 1) chunks = 1;
+    if (chunks > T) chunks = T;
+    p.n_ctas = chunks * Hkv;            // ranges of T / chunks tiles never cross a head when chunks divides evenly...
+    while (T % chunks) --chunks;        // ...so take a divisor of T
+    p.n_ctas = chunks * Hkv;
+  }
+  p.chunks = 0;
+  p.n_slots = sink_slots(p.groups_staged * hpg, p.n_pad);
   p.scale_log2 = shape_scale(s) * 1.4426950408889634f;
   p.status = ctx->d_status;
   CUtensorMap tmK;
   if (!encode_kv_map(ctx->encode_tiled, &tmK, K, HD, s->L, Hkv, s->kv_stride_tok, s->kv_stride_head, 64, TK))
     return FOCUS_ERR_INVALID_ARG;
-  const int smem = 1024 + hpg * p.n_pad * 256 + p.n_slots * SLOT_BYTES + (2 * MAX_SLOTS + 4) * 8 + 16 +
-                   hpg * p.n_pad * 4 + 64;
+  const int hs = p.groups_staged * hpg;
+  const int smem = 1024 + hs * p.n_pad * 256 + p.n_slots * SLOT_BYTES + (2 * MAX_SLOTS + 2 * MAX_BUF) * 8 + 16 +
+                   hs * p.n_pad * 4 + 64;
   static int attr_smem = 0;
   if (smem > attr_smem) {
     if (cudaFuncSetAttribute(sink_colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return FOCUS_ERR_CUDA;
     attr_smem = smem;
   }
-  sink_colsum_tc_kernel<<<dim3(chunks, Hkv), NTHREADS, smem, st>>>(tmK, p);
+  sink_colsum_tc_kernel<<<p.n_ctas, NTHREADS, smem, st>>>(tmK, p);
   FOCUS_CHECK_LAUNCH();
   return FOCUS_OK;
 }
