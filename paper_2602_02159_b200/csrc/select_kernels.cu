@@ -194,27 +194,20 @@ __global__ void sink_reduce_heads_kernel(const float* __restrict__ part, int H, 
 constexpr int TN_THREADS = 1024;
 constexpr int TN_MAX_SMEM_KEYS = 56 * 1024;      // keys cached in shared memory (224 KB); beyond that they are re-read
 
-// Histogram increment with warp aggregation: lanes that hit the same bin elect one leader that adds their
-// count.  Sink scores are all close to 1/L, so without this nearly every add lands on one counter.
-__device__ __forceinline__ void hist_add(int* hist, uint32_t bin, bool active) {
-  const uint32_t amask = __ballot_sync(0xffffffffu, active);
-  if (!active) return;
-  const uint32_t peers = __match_any_sync(amask, bin);
-  if ((threadIdx.x & 31) == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
-}
-
-// One CTA.  Keys (order-preserving integers of the scores) are staged once in shared memory, then: 4-pass 8-bit
-// radix select of the want-th largest key T, and an ordered compaction in which warp w owns the w-th contiguous
-// segment of the candidates (ballot/popc keeps index order inside a warp, one block scan orders the warps).
+// One CTA.  Keys (order-preserving integers of the scores) are staged once in shared memory, then:
+// (1) the key T of the want-th largest element is found bit by bit, MSB first: T keeps a bit iff at least `want`
+//     keys are >= the candidate -- 32 counting sweeps with no atomics and one barrier each (sink scores are all
+//     close to 1/L, which makes histogram-based radix passes collide on one counter);
+// (2) an ordered compaction in which warp w owns the w-th contiguous segment of the candidates (ballot/popc
+//     keeps index order inside a warp, one block scan orders the warps); keys equal to T are taken in index
+//     order until the quota is filled.
 template <bool CACHED>
 __global__ void __launch_bounds__(TN_THREADS)
 sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const int32_t* n_active,
                  int32_t* __restrict__ sink_idx, int32_t* status) {
   extern __shared__ uint32_t skey[];
-  __shared__ int hist[256];
+  __shared__ int cnt[33];
   __shared__ int scan_s[33];
-  __shared__ uint32_t s_prefix;
-  __shared__ int s_remaining;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = hi - lo;
   const int want = min(n_sink, n);
@@ -227,60 +220,34 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
     for (int i = tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
     return;
   }
+  if (tid < 33) cnt[tid] = 0;
   if (CACHED) {
 #pragma unroll 8
     for (int i = tid; i < n; i += TN_THREADS) skey[i] = float_key(S[lo + i]);
-    __syncthreads();
   }
+  __syncthreads();
   auto key_at = [&](int i) -> uint32_t { return CACHED ? skey[i] : float_key(S[lo + i]); };
-  // radix select: find the key T of the want-th largest element, MSB first
-  uint32_t prefix = 0, pmask = 0;
-  int remaining = want;                       // rank (1-based) still to locate inside the current bucket
-  const int n_round = (n + TN_THREADS - 1) / TN_THREADS * TN_THREADS;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int b = tid; b < 256; b += TN_THREADS) hist[b] = 0;
+  uint32_t T = 0;
+  for (int bit = 31; bit >= 0; --bit) {
+    const uint32_t cand = T | (1u << bit);
+    int c = 0;
+#pragma unroll 8
+    for (int i = tid; i < n; i += TN_THREADS) c += key_at(i) >= cand ? 1 : 0;
+    c = __reduce_add_sync(0xffffffffu, c);
+    if (lane == 0 && c) atomicAdd(&cnt[bit], c);
     __syncthreads();
-    for (int i = tid; i < n_round; i += TN_THREADS) {
-      uint32_t k = 0;
-      if (i < n) k = key_at(i);
-      hist_add(hist, (k >> shift) & 255u, i < n && (k & pmask) == prefix);
-    }
-    __syncthreads();
-    if (tid < 32) {
-      // bucket b such that (count of keys in buckets above b) < remaining <= (that count + hist[b])
-      int above = 0, found = -1, found_above = 0;
-      for (int base = 224; base >= 0 && found < 0; base -= 32) {
-        const int b = base + 31 - tid;                       // lane 0 owns the highest bucket of the group
-        const int h = hist[b];
-        int incl = h;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int y = __shfl_up_sync(0xffffffffu, incl, o);
-          if (tid >= o) incl += y;
-        }
-        const bool hit = above + incl >= remaining;
-        const uint32_t bal = __ballot_sync(0xffffffffu, hit);
-        if (bal) {
-          const int l0 = __ffs(bal) - 1;
-          found = base + 31 - l0;
-          found_above = above + __shfl_sync(0xffffffffu, incl - h, l0);
-        } else {
-          above += __shfl_sync(0xffffffffu, incl, 31);
-        }
-      }
-      if (tid == 0) {
-        if (found < 0) { found = 0; found_above = above - hist[0]; }
-        s_prefix = prefix | ((uint32_t)found << shift);
-        s_remaining = remaining - found_above;
-      }
-    }
-    __syncthreads();
-    prefix = s_prefix;
-    remaining = s_remaining;
-    pmask |= 255u << shift;
+    if (cnt[bit] >= want) T = cand;
+  }
+  // T = key of the want-th largest element.  Count the strictly greater ones to know how many equal keys to take.
+  {
+    int c = 0;
+#pragma unroll 8
+    for (int i = tid; i < n; i += TN_THREADS) c += key_at(i) > T ? 1 : 0;
+    c = __reduce_add_sync(0xffffffffu, c);
+    if (lane == 0 && c) atomicAdd(&cnt[32], c);
     __syncthreads();
   }
-  const uint32_t T = prefix;                 // threshold key; `remaining` = how many == T to take (lowest index first)
+  const int remaining = want - cnt[32];          // how many keys == T to take (lowest index first)
   // ordered compaction: warp w owns candidates [w*seg, (w+1)*seg), seg a multiple of 32
   const int seg = ((n + 31) / 32 + 31) / 32 * 32;
   const int w_lo = min(warp * seg, n), w_hi = min(w_lo + seg, n);
