@@ -399,6 +399,95 @@ def run_focus(args):
     print(json.dumps(out))
 
 
+def run_sweep(args):
+    """Config 4: one attention layer, 32 heads, d 128, bf16, gen 256; context x keep ratio.  Per point: latency of
+    the sparse layer (selection + attention) and of the attention call alone, for the gen-region rows (256) and for
+    the paper's I_active rows, retained-FLOP TFLOP/s, HBM GB/s, and the ratio to the own dense attention."""
+    import torch
+
+    from paper_2602_02159_b200 import binding as fb
+    from paper_2602_02159_b200 import build as fbuild
+    from paper_2602_02159_b200 import step as fstep
+    from paper_2602_02159_b200 import workloads as wl
+    fbuild.build()
+    torch.cuda.set_device(0)
+    ctx = fb.Context(0, workspace_bytes=1 << 30)
+    P = peaks()
+    out = []
+    for L in wl.SWEEP_L:
+        w0 = wl.config(4, L=L, keep_den=1)
+        s = w0.shape
+        layer_bytes = 2 * s.Hkv * s.L * s.d * 2
+        NL = max(2, min(8, -(-400_000_000 // layer_bytes)))          # rotate layers: > 3x L2 in total
+        g = torch.Generator(device="cuda").manual_seed(L)
+        mk = lambda *sh: (torch.randn(*sh, device="cuda", generator=g) / s.d ** 0.5).to(torch.bfloat16)
+        Qs = [mk(s.N, s.H, s.d) for _ in range(NL)]
+        Ks = [mk(s.Hkv, s.L, s.d) for _ in range(NL)]
+        Vs = [mk(s.Hkv, s.L, s.d) for _ in range(NL)]
+        c_prev, _ = wl.gen_confidence(0, s.N)
+        conf = torch.from_numpy(wl.full_conf(s, c_prev)).cuda()
+        masked = torch.from_numpy(wl.gen_masked(w0)).cuda()
+
+        def graph_time(fn):
+            for l in range(NL):
+                fn(l)
+            torch.cuda.synchronize()
+            gr = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gr):
+                for l in range(NL):
+                    fn(l)
+            for _ in range(3):
+                gr.replay()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = max(3, min(20, int(2e-3 * 1e9 / layer_bytes) + 3))
+            e0.record()
+            for _ in range(reps):
+                gr.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps / NL * 1e3          # us per call
+
+        for rows in ("gen", "active"):
+            dense_us = None
+            for den in wl.SWEEP_KEEP_DEN:
+                w = wl.config(4, L=L, keep_den=den)
+                b = fstep.StepBuffers(w, rows=rows)
+                fstep.select_queries(ctx, b, conf, masked)
+                ba = fstep.StepBuffers(w, rows="active")
+                fstep.select_queries(ctx, ba, conf, masked)
+                fstep.dense_layer(ctx, ba, Qs[0], Ks[0], Vs[0])
+                fstep.find_sinks(ctx, ba, Qs[0], Ks[0], ba.lse)
+                b.sink_idx.copy_(ba.sink_idx)
+                Kb = []
+                for l in range(NL):
+                    kb = torch.zeros(s.Hkv, s.nb, s.d, dtype=torch.float32, device="cuda")
+                    fb.focus_pool_keys(ctx, b.shape, Ks[l], kb)
+                    Kb.append(kb)
+                if dense_us is None:
+                    dense_us = graph_time(lambda l: fstep.dense_layer(ctx, b, Qs[l], Ks[l], Vs[l]))
+                layer_us = graph_time(lambda l: fstep.sparse_layer(ctx, b, Qs[l], Ks[l], Vs[l], Kbar=Kb[l]))
+                q_rows, n_rows, max_rows = b._rows()
+                attn_us = graph_time(lambda l: fb.focus_sparse_attn(
+                    ctx, b.shape, Qs[l], s.M, s.N, q_rows, n_rows, max_rows, Ks[l], Vs[l], fb.HEADS_PER_KV_GROUP,
+                    b.block_idx, b.max_blocks, b.block_cnt, b.sink_idx, b.sink_keep, w.n_sink, b.O, b.lse))
+                n_q = s.N if rows == "gen" else int(b.n_active.item())
+                keys = w.C * s.B + w.n_sink + s.N
+                flops = 4.0 * n_q * keys * s.d * s.H
+                byts = 2.0 * s.Hkv * keys * s.d * 2 + 2.0 * n_q * s.H * s.d * 2
+                tf, gbs = flops / attn_us / 1e6, byts / attn_us / 1e3
+                out.append({"L": L, "rows": rows, "n_q": n_q, "keep": f"1/{den}", "blocks": w.C, "retained_keys": keys,
+                            "sparse_layer_us": round(layer_us, 2), "sparse_attn_us": round(attn_us, 2),
+                            "dense_attn_us": round(dense_us, 2), "attn_vs_dense": round(dense_us / attn_us, 2),
+                            "retained_TFLOPs": round(tf, 1), "frac_tensor_sustained": round(tf / P["tf_sust"], 3),
+                            "dense_equiv_TFLOPs": round(4.0 * n_q * s.L * s.d * s.H / attn_us / 1e6, 1),
+                            "GBps": round(gbs, 1), "frac_hbm": round(gbs / P["hbm"], 3)})
+                assert ctx.poll_status() == 0
+        del Qs, Ks, Vs
+        torch.cuda.empty_cache()
+    print(json.dumps({"sweep": out, "peaks": P}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -409,9 +498,12 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (quick runs)")
     ap.add_argument("--skip-gen", action="store_true", help="skip the gen-region-rows (tensor-bound) measurements")
     ap.add_argument("--no-graph", action="store_true", help="time eager C-ABI calls instead of a CUDA graph replay")
+    ap.add_argument("--sweep", action="store_true", help="run the context x keep-ratio sweep (config 4) instead")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle baseline leg")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_focus(args)
