@@ -49,6 +49,7 @@ struct TcParams {
   long long q_stride_row, q_stride_head;
   int q_base, n_q, rows_bound, L, M, H, Hkv, hpg, B, nb, dense, group_stride, max_blocks, n_sink, ns_pad;
   int n_mtiles, n_splits, lse_stride;
+  int cluster;                 // 1: the splits of a tile are one thread-block cluster and merge through shared memory
   float scale_log2;            // softmax scale * log2(e)
   int32_t* status;
 #ifdef FOCUS_TIMELINE
@@ -162,6 +163,80 @@ __device__ __forceinline__ void merge_rows(const TcParams& p, int tile, int g, i
   }
 }
 
+// ---- split merge inside a thread-block cluster ---------------------------------------------------------------
+// When the n_splits CTAs of one (KV head, query tile) are launched as a cluster, each leaves its unnormalised
+// partial (rows x 128 floats, row pitch PROW, plus (max, sum) per row) in its own shared memory; after a cluster
+// barrier CTA `rank` merges the rows r with r mod n_splits == rank, reading every CTA's copy through distributed
+// shared memory, splits in index order.  No global scratch, no fence, no atomic.
+constexpr int PROW = HD + 4;                                   // floats per partial row (padding spreads the banks)
+constexpr int PART_ML_OFF = TM * PROW;                         // float offset of the (max, sum) pairs
+
+__device__ __forceinline__ void cluster_sync_all() {
+  __syncwarp();
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 ld_dsmem_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float2 ld_dsmem_f2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
+
+__device__ __forceinline__ void cluster_merge(const TcParams& p, int g, int mt, int total_fr, int rank, uint32_t spart) {
+  __syncthreads();
+  cluster_sync_all();
+  const int rows = min(TM, total_fr - mt * TM);
+  const int S = p.n_splits;                                   // <= 8 in cluster mode
+  const int mine = rank < rows ? (rows - rank + S - 1) / S : 0;
+  for (int item = threadIdx.x; item < mine * 32; item += NTHREADS) {
+    const int row = rank + (item >> 5) * S, cg = item & 31;
+    float2 ml[8];
+    float4 o[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      if (s < S) {
+        const uint32_t base = map_to_rank(spart, (uint32_t)s);
+        ml[s] = ld_dsmem_f2(base + (uint32_t)(PART_ML_OFF + row * 2) * 4u);
+        o[s] = ld_dsmem_f4(base + (uint32_t)(row * PROW + cg * 4) * 4u);
+      }
+    }
+    float m = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < 8; ++s)
+      if (s < S && ml[s].y > 0.f) m = fmaxf(m, ml[s].x);
+    float tot = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      if (s < S && ml[s].y > 0.f) {
+        const float wgt = exp2f(ml[s].x - m);
+        tot += wgt * ml[s].y;
+        acc.x += wgt * o[s].x; acc.y += wgt * o[s].y; acc.z += wgt * o[s].z; acc.w += wgt * o[s].w;
+      }
+    }
+    const float inv = tot > 0.f ? 1.f / tot : 0.f;
+    const int fr = mt * TM + row;
+    const int qr = fr / p.hpg, hh = fr % p.hpg;
+    __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD + cg * 4;
+    uint2 v;
+    v.x = pack_bf16(acc.x * inv, acc.y * inv);
+    v.y = pack_bf16(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2*>(orow) = v;
+    if (p.lse && cg == 0)
+      p.lse[(size_t)(g * p.hpg + hh) * p.lse_stride + qr] = (m + log2f(tot)) * 0.6931471805599453f;
+  }
+  cluster_sync_all();                                          // nobody leaves while its partial may still be read
+}
+
 // Called by every thread of every split CTA once its partial is written: the CTA that arrives last at the
 // tile's counter merges all splits and re-arms the counter for the next launch.
 __device__ __forceinline__ void finish_split(const TcParams& p, int tile, int g, int mt, int total_fr, int* s_last,
@@ -235,6 +310,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     return tile_info(p, te, t0 + idx);
   };
 
+  if (nt <= 0 && p.cluster) {                             // empty split inside a cluster: neutral partial, then merge duty
+    float* ps = reinterpret_cast<float*>(sptr + Q_BYTES);
+    for (int r = threadIdx.x; r < TM; r += NTHREADS) { ps[PART_ML_OFF + 2 * r] = -INFINITY; ps[PART_ML_OFF + 2 * r + 1] = 0.f; }
+    cluster_merge(p, g, mt, total_fr, split, sSlot);
+    return;
+  }
   if (nt <= 0) {                                          // empty split: publish a neutral partial
     if (p.n_splits > 1) {
       if (warp >= 2) {
@@ -524,6 +605,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         }
         if (valid && p.lse)
           p.lse[(size_t)(g * p.hpg + hh) * p.lse_stride + qr] = (m_ref + log2f(l)) * 0.6931471805599453f;
+      } else if (p.cluster) {
+        if (__any_sync(0xffffffffu, valid)) {
+          float* ps = reinterpret_cast<float*>(sptr + Q_BYTES);
+          float* prow = ps + row * PROW;
+#pragma unroll
+          for (int cb = 0; cb < 4; ++cb) {
+            uint32_t oreg[32];
+            TC_LD32(tmem_O + lane_off + cb * 32, oreg);
+            tc_wait_ld();
+            if (valid) {
+#pragma unroll
+              for (int c = 0; c < 32; c += 4)
+                *reinterpret_cast<uint4*>(prow + cb * 32 + c) = make_uint4(oreg[c], oreg[c + 1], oreg[c + 2], oreg[c + 3]);
+            }
+          }
+          if (valid) { ps[PART_ML_OFF + 2 * row] = m_ref; ps[PART_ML_OFF + 2 * row + 1] = l; }
+        }
       } else if (__any_sync(0xffffffffu, valid)) {           // warps whose 32 rows are all padding have nothing to publish
         float* po = p.part_O + ((size_t)cta_lin * TM + row) * HD;
 #pragma unroll
@@ -553,7 +651,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     tmem_dealloc(tmem, 512);
   }
   TL_STAMP(3, 0);
-  if (p.n_splits > 1 && p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p, reinterpret_cast<float*>(sptr + Q_BYTES));
+  if (p.cluster) cluster_merge(p, g, mt, total_fr, split, sSlot);
+  else if (p.n_splits > 1 && p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p, reinterpret_cast<float*>(sptr + Q_BYTES));
   TL_STAMP(4, 0);
 }
 
@@ -629,7 +728,8 @@ int pick_splits(const focus_ctx* ctx, int base_ctas, int max_tiles) {
   int s = ctx->sm_count / (base_ctas > 0 ? base_ctas : 1);
   if (s < 1) s = 1;
   const int cap = max_tiles / 2 > 1 ? max_tiles / 2 : 1;
-  return s < cap ? s : cap;
+  if (s > cap) s = cap;
+  return s > 8 ? 8 : s;                      // at most 8 splits: they form one (portable-size) thread-block cluster
 }
 
 }  // namespace
@@ -676,8 +776,32 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
       mask = ws.get<uint8_t>((size_t)Hkv * ns_pad);
     }
   }
-  float* part_O = nullptr; float* part_ml = nullptr;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+      return FOCUS_ERR_CUDA;
+    attr_set = true;
+  }
+  // can the splits of a tile be co-scheduled as one cluster?  (asked once per cluster size)
+  static int cluster_ok[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};          // 0 unknown, 1 yes, -1 no
+  bool use_cluster = false;
   if (n_splits > 1) {
+    if (cluster_ok[n_splits] == 0) {
+      cudaLaunchConfig_t qc = {};
+      qc.gridDim = dim3(n_splits, n_splits, 1); qc.blockDim = dim3(NTHREADS, 1, 1); qc.dynamicSmemBytes = SMEM_BYTES;
+      cudaLaunchAttribute qa[1];
+      qa[0].id = cudaLaunchAttributeClusterDimension;
+      qa[0].val.clusterDim.x = 1; qa[0].val.clusterDim.y = n_splits; qa[0].val.clusterDim.z = 1;
+      qc.attrs = qa; qc.numAttrs = 1;
+      int n_clusters = 0;
+      const cudaError_t e = cudaOccupancyMaxActiveClusters(&n_clusters, attn_tc_kernel, &qc);
+      cluster_ok[n_splits] = (e == cudaSuccess && n_clusters >= 1) ? 1 : -1;
+      if (e != cudaSuccess) cudaGetLastError();
+    }
+    use_cluster = cluster_ok[n_splits] == 1;
+  }
+  float* part_O = nullptr; float* part_ml = nullptr;
+  if (n_splits > 1 && !use_cluster) {
     part_O = ws.get<float>((size_t)base * n_splits * TM * HD);
     part_ml = ws.get<float>((size_t)base * n_splits * TM * 2);
   }
@@ -706,7 +830,8 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.Q = (const __nv_bfloat16*)a.Q; p.O = (__nv_bfloat16*)a.O; p.lse = a.lse;
   p.q_rows = a.q_rows; p.n_rows = a.n_rows; p.block_idx = a.block_idx; p.block_cnt = a.block_cnt;
   p.sink_mask = mask; p.part_O = part_O; p.part_ml = part_ml;
-  p.counters = (n_splits > 1 && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
+  p.cluster = use_cluster ? 1 : 0;
+  p.counters = (n_splits > 1 && !use_cluster && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
                    ? ctx->d_counters : nullptr;
   p.q_stride_row = sh.q_stride_row; p.q_stride_head = sh.q_stride_head;
   p.q_base = a.q_base; p.n_q = a.n_q; p.rows_bound = a.max_rows; p.L = sh.L; p.M = sh.M; p.H = sh.n_q_heads;
@@ -719,15 +844,23 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.dbg = getenv("FOCUS_TIMELINE") ? (unsigned long long*)(ctx->ws + ctx->ws_bytes - (1 << 20)) : nullptr;
 #endif
 
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+  if (use_cluster) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(base, n_splits, 1); cfg.blockDim = dim3(NTHREADS, 1, 1);
+    cfg.dynamicSmemBytes = SMEM_BYTES; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = n_splits; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, attn_tc_kernel, tmK, tmV, tmSK, tmSV, p) != cudaSuccess) {
+      cudaGetLastError();
       return FOCUS_ERR_CUDA;
-    attr_set = true;
+    }
+  } else {
+    attn_tc_kernel<<<dim3(base, n_splits), NTHREADS, SMEM_BYTES, st>>>(tmK, tmV, tmSK, tmSV, p);
   }
-  attn_tc_kernel<<<dim3(base, n_splits), NTHREADS, SMEM_BYTES, st>>>(tmK, tmV, tmSK, tmSV, p);
   FOCUS_CHECK_LAUNCH();
-  if (n_splits > 1 && !p.counters) {
+  if (n_splits > 1 && !p.counters && !use_cluster) {
     const int rows_total = base * TM;
     attn_combine_kernel<<<rows_total / 8, 256, 0, st>>>(part_O, part_ml, n_splits, n_mtiles, hpg, sh.n_q_heads,
                                                         a.q_rows, a.n_rows, a.max_rows, a.n_q,
