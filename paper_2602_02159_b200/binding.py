@@ -10,7 +10,7 @@ import os
 from typing import Optional
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libfocus.so")
+LIB_PATH = os.environ.get("FOCUS_LIB_PATH") or os.path.join(HERE, "libfocus.so")   # override: an alternative build
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIMEOUT = range(6)
 F32, BF16 = 0, 1
