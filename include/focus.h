@@ -89,6 +89,11 @@ const char* focus_status_string(focus_status s);
 /* Number of kernels this library has launched in this process so far (all contexts). */
 uint64_t focus_launch_count(void);
 
+/* Which attention kernel the last focus_dense_attn / focus_sparse_attn / focus_sparse_layer call on this context
+ * used: 1 = generic SIMT, 2 = tensor-core kernel with one 128-row query tile per CTA, 3 = tensor-core kernel with
+ * two query tiles per CTA (taken for >= 256 stacked rows per KV head on long key streams); 0 = none yet. */
+int32_t focus_last_attn_variant(focus_ctx* ctx);
+
 /* Selects the attention implementation for bf16 / head_dim 128 inputs: 0 = automatic (tensor-core
  * kernel where supported), 1 = force the generic SIMT kernels.  Returns the previous value. */
 int32_t focus_set_force_simt(focus_ctx* ctx, int32_t force);

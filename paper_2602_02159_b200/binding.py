@@ -43,6 +43,7 @@ _SIGS = {
     "focus_status_string": (C.c_char_p, [_I]),
     "focus_set_force_simt": (_I, [_P, _I]),
     "focus_launch_count": (C.c_uint64, []),
+    "focus_last_attn_variant": (_I, [_P]),
     "focus_select_queries": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P, _P, _P, _P, _P]),
     "focus_find_sinks": (_I, [_P, _SH, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _P, _P, _P]),
     "focus_pool_keys": (_I, [_P, _SH, _P, _P, _P]),
@@ -135,6 +136,9 @@ class Context:
         v = _I(0)
         _check(self._lib.focus_poll_status(self.handle, _stream(stream), C.byref(v)), "focus_poll_status")
         return v.value
+
+    def last_attn_variant(self) -> int:
+        return self._lib.focus_last_attn_variant(self.handle)
 
     def set_force_simt(self, force: bool) -> int:
         return self._lib.focus_set_force_simt(self.handle, 1 if force else 0)

@@ -169,7 +169,6 @@ __device__ __forceinline__ void merge_rows(const TcParams& p, int tile, int g, i
 // barrier CTA `rank` merges the rows r with r mod n_splits == rank, reading every CTA's copy through distributed
 // shared memory, splits in index order.  No global scratch, no fence, no atomic.
 constexpr int PROW = HD + 4;                                   // floats per partial row (padding spreads the banks)
-constexpr int PART_ML_OFF = TM * PROW;                         // float offset of the (max, sum) pairs
 
 __device__ __forceinline__ void cluster_sync_all() {
   __syncwarp();
@@ -191,13 +190,15 @@ __device__ __forceinline__ float2 ld_dsmem_f2(uint32_t addr) {
   return v;
 }
 
+template <int ROWS, int NTH>
 __device__ __forceinline__ void cluster_merge(const TcParams& p, int g, int mt, int total_fr, int rank, uint32_t spart) {
+  constexpr int PART_ML_OFF = ROWS * PROW;                     // float offset of the (max, sum) pairs
   __syncthreads();
   cluster_sync_all();
-  const int rows = min(TM, total_fr - mt * TM);
+  const int rows = min(ROWS, total_fr - mt * ROWS);
   const int S = p.n_splits;                                   // <= 8 in cluster mode
   const int mine = rank < rows ? (rows - rank + S - 1) / S : 0;
-  for (int item = threadIdx.x; item < mine * 32; item += NTHREADS) {
+  for (int item = threadIdx.x; item < mine * 32; item += NTH) {
     const int row = rank + (item >> 5) * S, cg = item & 31;
     float2 ml[8];
     float4 o[8];
@@ -224,7 +225,7 @@ __device__ __forceinline__ void cluster_merge(const TcParams& p, int g, int mt, 
       }
     }
     const float inv = tot > 0.f ? 1.f / tot : 0.f;
-    const int fr = mt * TM + row;
+    const int fr = mt * ROWS + row;
     const int qr = fr / p.hpg, hh = fr % p.hpg;
     __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD + cg * 4;
     uint2 v;
@@ -312,8 +313,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 
   if (nt <= 0 && p.cluster) {                             // empty split inside a cluster: neutral partial, then merge duty
     float* ps = reinterpret_cast<float*>(sptr + Q_BYTES);
-    for (int r = threadIdx.x; r < TM; r += NTHREADS) { ps[PART_ML_OFF + 2 * r] = -INFINITY; ps[PART_ML_OFF + 2 * r + 1] = 0.f; }
-    cluster_merge(p, g, mt, total_fr, split, sSlot);
+    for (int r = threadIdx.x; r < TM; r += NTHREADS) { ps[TM * PROW + 2 * r] = -INFINITY; ps[TM * PROW + 2 * r + 1] = 0.f; }
+    cluster_merge<TM, NTHREADS>(p, g, mt, total_fr, split, sSlot);
     return;
   }
   if (nt <= 0) {                                          // empty split: publish a neutral partial
@@ -508,8 +509,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       const TileInfo ti = get_tile(idx);
       float tmax = -INFINITY;
       if (ti.kind == 0 && ti.nvalid == TN) {
+        float t4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains instead of one of 128
 #pragma unroll
-        for (int c = 0; c < 128; ++c) tmax = fmaxf(tmax, __uint_as_float(sreg[c]));
+        for (int c = 0; c < 128; c += 4) {
+          t4[0] = fmaxf(t4[0], __uint_as_float(sreg[c]));     t4[1] = fmaxf(t4[1], __uint_as_float(sreg[c + 1]));
+          t4[2] = fmaxf(t4[2], __uint_as_float(sreg[c + 2])); t4[3] = fmaxf(t4[3], __uint_as_float(sreg[c + 3]));
+        }
+        tmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
       } else if (ti.kind == 0) {
 #pragma unroll
         for (int c = 0; c < 128; ++c) {
@@ -544,15 +550,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       // p = 2^(s*scale_log2 - m_ref); a fully masked row so far (m_ref = -inf) contributes zeros
       const float mneg = m_ref == -INFINITY ? 0.f : -m_ref;
       uint32_t preg[64];
-      float lsum = 0.f;
+      float ls4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int c = 0; c < 64; ++c) {
         const float p0 = ex2(fmaf(__uint_as_float(sreg[2 * c]), p.scale_log2, mneg));
         const float p1 = ex2(fmaf(__uint_as_float(sreg[2 * c + 1]), p.scale_log2, mneg));
-        lsum += p0 + p1;
+        ls4[c & 3] += p0 + p1;
         preg[c] = pack_bf16(p0, p1);
       }
-      l = l * alpha + lsum;
+      l = l * alpha + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
       if (idx > 0) {
         // P_{idx-1} V_{idx-1} must have left the tensor core before O is touched; waiting for every phase in
         // order also keeps the parity of this barrier unambiguous
@@ -620,7 +626,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
                 *reinterpret_cast<uint4*>(prow + cb * 32 + c) = make_uint4(oreg[c], oreg[c + 1], oreg[c + 2], oreg[c + 3]);
             }
           }
-          if (valid) { ps[PART_ML_OFF + 2 * row] = m_ref; ps[PART_ML_OFF + 2 * row + 1] = l; }
+          if (valid) { ps[TM * PROW + 2 * row] = m_ref; ps[TM * PROW + 2 * row + 1] = l; }
         }
       } else if (__any_sync(0xffffffffu, valid)) {           // warps whose 32 rows are all padding have nothing to publish
         float* po = p.part_O + ((size_t)cta_lin * TM + row) * HD;
@@ -651,9 +657,380 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     tmem_dealloc(tmem, 512);
   }
   TL_STAMP(3, 0);
-  if (p.cluster) cluster_merge(p, g, mt, total_fr, split, sSlot);
+  if (p.cluster) cluster_merge<TM, NTHREADS>(p, g, mt, total_fr, split, sSlot);
   else if (p.n_splits > 1 && p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p, reinterpret_cast<float*>(sptr + Q_BYTES));
   TL_STAMP(4, 0);
+}
+
+// ================================================================================================================
+// Wide variant: one CTA = TWO 128-row query tiles (A, B) of one KV head.  Used when a KV head has at least 256
+// stacked query rows (the gen-region query set), where the kernel is bound by the tensor pipe and by the
+// exponentials rather than by HBM.  Every K/V tile is staged once and serves 256 rows; the two tiles take turns
+// on the tensor core: while the softmax warps of A work on S_A(j), the tensor pipe runs S_B(j) = Q_B K_j^T and
+// O_B += P_B(j-1) V_(j-1), and vice versa.  TMEM: S_A | S_B | O_A | O_B (4 x 128 columns), P aliases S.
+// Warps (320 threads): 0 TMA producer, 1 MMA issuer + TMEM owner, 2..5 softmax of tile A, 6..9 softmax of tile B.
+// ================================================================================================================
+constexpr int TMW = 256;
+constexpr int NSLOT_W = 5;
+constexpr int Q_BYTES_W = TMW * HD * 2;
+constexpr int NBAR_W = 2 * NSLOT_W + 7;
+constexpr int MAXT_W = 96;
+constexpr int NTHREADS_W = 320;
+constexpr int SMEM_BYTES_W = 1024 + Q_BYTES_W + NSLOT_W * SLOT_BYTES + NBAR_W * 8 + 64 + MAXT_W * 8;
+
+__global__ void __launch_bounds__(NTHREADS_W, 1)
+attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                    const __grid_constant__ CUtensorMap tmSK, const __grid_constant__ CUtensorMap tmSV, const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
+
+  constexpr int QTHREADS = 256;                                  // the eight softmax warps stage Q
+  constexpr int QIT = TMW * 16 / QTHREADS;
+  const int qtid = (int)threadIdx.x - 64;
+  const int nrows_raw = p.q_rows ? __ldg(p.n_rows) : p.n_q;
+  const int cnt_raw = p.dense ? 0 : __ldg(p.block_cnt + g * p.group_stride);
+  int qpos[QIT];
+#pragma unroll
+  for (int it = 0; it < QIT; ++it) {
+    const int idx = qtid + it * QTHREADS;
+    const int qr = (mt * TMW + (idx >> 4)) / p.hpg;
+    qpos[it] = (qtid >= 0 && qr < p.rows_bound) ? (p.q_rows ? __ldg(p.q_rows + qr) : p.q_base + qr) : -1;
+  }
+  const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
+  const int total_fr = nrows * p.hpg;
+  if (mt * TMW >= total_fr) return;
+
+  const TileEnum te = make_enum(p, g, cnt_raw);
+  const int t0 = (int)(((long long)te.total * split) / p.n_splits);
+  const int t1 = (int)(((long long)te.total * (split + 1)) / p.n_splits);
+  const int nt = t1 - t0;
+
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sptr = smem_raw + (sbase - smem_u32(smem_raw));
+  const uint32_t sQ = sbase;
+  const uint32_t sSlot = sbase + Q_BYTES_W;
+  const uint32_t sBar = sSlot + NSLOT_W * SLOT_BYTES;
+  auto bar_full = [&](int s) { return sBar + 8u * s; };
+  auto bar_empty = [&](int s) { return sBar + 8u * (NSLOT_W + s); };
+  auto bar_sfull = [&](int x) { return sBar + 8u * (2 * NSLOT_W + x); };
+  auto bar_pready = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 2 + x); };
+  auto bar_pvdone = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 4 + x); };
+  const uint32_t bar_alldone = sBar + 8u * (2 * NSLOT_W + 6);   // every MMA of this CTA has completed
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(sptr + Q_BYTES_W + NSLOT_W * SLOT_BYTES + NBAR_W * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  int2* tlist = reinterpret_cast<int2*>(tmem_holder + 16);
+  const bool use_list = !p.dense && nt <= MAXT_W;
+  auto get_tile = [&](int idx) -> TileInfo {
+    if (use_list) {
+      const int2 e = tlist[idx];
+      TileInfo ti; ti.kind = e.x >> 30; ti.start = e.x & 0x3FFFFFFF; ti.nvalid = e.y;
+      return ti;
+    }
+    return tile_info(p, te, t0 + idx);
+  };
+  float* ps = reinterpret_cast<float*>(sptr + Q_BYTES_W);        // split partial (cluster mode), over the K/V ring
+
+  if (nt <= 0) {                                                 // empty split (cluster mode only: see the launcher)
+    for (int r = threadIdx.x; r < TMW; r += NTHREADS_W) { ps[TMW * PROW + 2 * r] = -INFINITY; ps[TMW * PROW + 2 * r + 1] = 0.f; }
+    cluster_merge<TMW, NTHREADS_W>(p, g, mt, total_fr, split, sSlot);
+    return;
+  }
+
+  // load sequence: q even -> K_(q/2), q odd -> V_(q/2); the MMA warp consumes K0, V0, K1, V1, ... in this order
+  auto issue = [&](int q) {
+    const bool isV = q & 1;
+    const TileInfo ti = get_tile(q >> 1);
+    const int slot = q % NSLOT_W;
+    const CUtensorMap* map = ti.kind ? (isV ? &tmSV : &tmSK) : (isV ? &tmV : &tmK);
+    const uint32_t dst = sSlot + slot * SLOT_BYTES;
+    mbar_expect_tx(bar_full(slot), SLOT_BYTES);
+    tma_load_3d(dst, map, bar_full(slot), 0, ti.start, g);
+    tma_load_3d(dst + HALF_BYTES, map, bar_full(slot), 64, ti.start, g);
+  };
+  const int n_loads = 2 * nt;
+  const int n_early = n_loads < NSLOT_W ? n_loads : NSLOT_W;
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int s = 0; s < NSLOT_W; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+      for (int x = 0; x < 2; ++x) { mbar_init(bar_sfull(x), 1); mbar_init(bar_pready(x), 128); mbar_init(bar_pvdone(x), 1); }
+      mbar_init(bar_alldone, 1);
+      *abort_flag = 0;
+      fence_barrier_init();
+      fence_proxy_async();
+    }
+    if (use_list) {
+      for (int t = lane; t < nt; t += 32) {
+        const TileInfo ti = tile_info(p, te, t0 + t);
+        if (t0 + t < te.n_blk) {
+          const int b = te.blocks[t0 + t];
+          if (b < 0 || b >= p.nb) set_status(p.status, FOCUS_ERR_INVALID_ARG);
+        }
+        tlist[t] = make_int2(ti.start | (ti.kind << 30), ti.nvalid);
+      }
+    }
+    __syncwarp();
+    if (lane == 0)
+      for (int q = 0; q < n_early; ++q) issue(q);
+    __syncwarp();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_holder), 512);
+    tmem_relinquish();
+  }
+  if (qtid >= 0) {                                               // both Q tiles: tile X at X * 32 KB, swizzled K-major
+    uint4 qv[QIT];
+#pragma unroll
+    for (int it = 0; it < QIT; ++it) {
+      const int idx = qtid + it * QTHREADS;
+      const int r = idx >> 4, c = idx & 15;
+      const int fr = mt * TMW + r;
+      qv[it] = make_uint4(0, 0, 0, 0);
+      if (fr < total_fr) {
+        const int pos = qpos[it];
+        if (pos >= p.q_base && pos < p.q_base + p.n_q) {
+          const __nv_bfloat16* src = p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
+                                     (long long)(g * p.hpg + fr % p.hpg) * p.q_stride_head + c * 8;
+          qv[it] = __ldg(reinterpret_cast<const uint4*>(src));
+        } else if (c == 0) {
+          set_status(p.status, FOCUS_ERR_INVALID_ARG);
+        }
+      }
+    }
+#pragma unroll
+    for (int it = 0; it < QIT; ++it) {
+      const int idx = qtid + it * QTHREADS;
+      const int r = idx >> 4, c = idx & 15;
+      const int x = r >> 7, rr = r & 127, half = c >> 3, cc = c & 7;
+      *reinterpret_cast<uint4*>(sptr + x * Q_BYTES + half * HALF_BYTES + rr * 128 + ((cc ^ (rr & 7)) << 4)) = qv[it];
+    }
+  }
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_holder;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int issued = n_early;
+      bool ok = true;
+      for (int q = n_early; q < n_loads; ++q) {
+        if (!mbar_wait(bar_empty(q % NSLOT_W), (uint32_t)((q / NSLOT_W) & 1) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        issue(q);
+        ++issued;
+      }
+      if (!ok) {
+        const uint32_t first = issued > NSLOT_W ? (uint32_t)(issued - NSLOT_W) : 0u;
+        for (uint32_t i = first; i < (uint32_t)issued; ++i) {
+          const uint64_t t_start = global_ns();
+          while (!mbar_try_wait(bar_full(i % NSLOT_W), (i / NSLOT_W) & 1u))
+            if (global_ns() - t_start > WAIT_LIMIT_NS) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t IDESC_QK = make_idesc(TM, TN, 0);
+      constexpr uint32_t IDESC_PV = make_idesc(TM, HD, 1);
+      bool ok = true;
+      auto wait_load = [&](int q) { return mbar_wait(bar_full(q % NSLOT_W), (uint32_t)(q / NSLOT_W) & 1u, abort_flag, p.status); };
+      auto do_qk = [&](int x, int j) {                              // S_x = Q_x K_j^T
+        const uint64_t qdesc = make_sdesc(sQ + x * Q_BYTES, 16, 1024);
+        const uint64_t kdesc = make_sdesc(sSlot + ((2 * j) % NSLOT_W) * SLOT_BYTES, 16, 1024);
+#pragma unroll
+        for (int half = 0; half < 2; ++half)
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            const uint64_t off = (uint64_t)((half * HALF_BYTES + ks * 32) >> 4);
+            mma_ss(tmem + x * 128, qdesc + off, kdesc + off, IDESC_QK, (half | ks) ? 1u : 0u);
+          }
+        tc_commit(bar_sfull(x));
+      };
+      auto do_pv = [&](int x, int j) {                              // O_x += P_x(j) V_j
+        const uint64_t vdesc = make_sdesc(sSlot + ((2 * j + 1) % NSLOT_W) * SLOT_BYTES, HALF_BYTES, 1024);
+#pragma unroll
+        for (int ks = 0; ks < TN / 16; ++ks)
+          mma_ts(tmem + 256 + x * 128, tmem + x * 128 + ks * 8, vdesc + (uint64_t)(ks * (2048 >> 4)), IDESC_PV,
+                 (j > 0 || ks > 0) ? 1u : 0u);
+        tc_commit(bar_pvdone(x));
+      };
+      ok = wait_load(0);
+      if (ok) {
+        tc_fence_after();
+        do_qk(0, 0);
+        do_qk(1, 0);
+        tc_commit(bar_empty(0));                                     // K_0's slot: free once both products have read it
+      }
+      for (int j = 0; j < nt && ok; ++j) {
+        const uint32_t par = (uint32_t)j & 1u;
+        if (!wait_load(2 * j + 1)) { ok = false; break; }            // V_j
+        if (!mbar_wait(bar_pready(0), par, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        do_pv(0, j);
+        if (j + 1 < nt) {
+          if (!wait_load(2 * j + 2)) { ok = false; break; }          // K_(j+1)
+          tc_fence_after();
+          do_qk(0, j + 1);
+        }
+        if (!mbar_wait(bar_pready(1), par, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        do_pv(1, j);
+        tc_commit(bar_empty((2 * j + 1) % NSLOT_W));                 // V_j
+        if (j + 1 < nt) {
+          do_qk(1, j + 1);
+          tc_commit(bar_empty((2 * j + 2) % NSLOT_W));               // K_(j+1)
+        }
+      }
+      tc_commit(bar_alldone);
+    }
+  } else {
+    const int x = (warp - 2) >> 2;                                   // query tile of this softmax warp
+    const int rq = warp & 3;
+    const int row = rq * 32 + lane;                                  // row inside the 128-row tile
+    const uint32_t lane_off = (uint32_t)(rq * 32) << 16;
+    const uint32_t ts = tmem + lane_off + x * 128;
+    const uint32_t to = tmem + lane_off + 256 + x * 128;
+    float m_ref = -INFINITY, l = 0.f;
+    bool ok = true;
+    for (int idx = 0; idx < nt; ++idx) {
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(x), (uint32_t)idx & 1u, abort_flag, p.status))) { ok = false; break; }
+      tc_fence_after();
+      uint32_t sreg[128];
+      TC_LD32(ts, (sreg + 0));
+      TC_LD32(ts + 32, (sreg + 32));
+      TC_LD32(ts + 64, (sreg + 64));
+      TC_LD32(ts + 96, (sreg + 96));
+      tc_wait_ld();
+      const TileInfo ti = get_tile(idx);
+      float tmax = -INFINITY;
+      if (ti.kind == 0 && ti.nvalid == TN) {
+        float t4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains instead of one of 128
+#pragma unroll
+        for (int c = 0; c < 128; c += 4) {
+          t4[0] = fmaxf(t4[0], __uint_as_float(sreg[c]));     t4[1] = fmaxf(t4[1], __uint_as_float(sreg[c + 1]));
+          t4[2] = fmaxf(t4[2], __uint_as_float(sreg[c + 2])); t4[3] = fmaxf(t4[3], __uint_as_float(sreg[c + 3]));
+        }
+        tmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
+      } else if (ti.kind == 0) {
+#pragma unroll
+        for (int c = 0; c < 128; ++c) {
+          const float v = c < ti.nvalid ? __uint_as_float(sreg[c]) : -INFINITY;
+          sreg[c] = __float_as_uint(v);
+          tmax = fmaxf(tmax, v);
+        }
+      } else {
+        const uint32_t* mk = reinterpret_cast<const uint32_t*>(p.sink_mask + (size_t)g * p.ns_pad + ti.start);
+#pragma unroll
+        for (int c4 = 0; c4 < 32; ++c4) {
+          const uint32_t mword = __ldg(mk + c4);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const int c = c4 * 4 + e;
+            const float v = ((mword >> (8 * e)) & 0xffu) ? __uint_as_float(sreg[c]) : -INFINITY;
+            sreg[c] = __float_as_uint(v);
+            tmax = fmaxf(tmax, v);
+          }
+        }
+      }
+      tmax *= p.scale_log2;
+      float alpha = 1.f;
+      bool rescale = false;
+      if (tmax > m_ref + RESCALE_THRESHOLD) {
+        if (m_ref != -INFINITY) {
+          alpha = ex2(m_ref - tmax);
+          rescale = true;
+        }
+        m_ref = tmax;
+      }
+      const float mneg = m_ref == -INFINITY ? 0.f : -m_ref;
+      uint32_t preg[64];
+      float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c = 0; c < 64; ++c) {
+        const float p0 = ex2(fmaf(__uint_as_float(sreg[2 * c]), p.scale_log2, mneg));
+        const float p1 = ex2(fmaf(__uint_as_float(sreg[2 * c + 1]), p.scale_log2, mneg));
+        ls4[c & 3] += p0 + p1;
+        preg[c] = pack_bf16(p0, p1);
+      }
+      l = l * alpha + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
+      if (idx > 0) {
+        if (!__all_sync(0xffffffffu, mbar_wait(bar_pvdone(x), (uint32_t)(idx - 1) & 1u, abort_flag, p.status))) { ok = false; break; }
+        if (__any_sync(0xffffffffu, rescale)) {
+          tc_fence_after();
+#pragma unroll
+          for (int cb = 0; cb < 4; ++cb) {
+            uint32_t oreg[32];
+            TC_LD32(to + cb * 32, oreg);
+            tc_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * alpha);
+            TC_ST32(to + cb * 32, oreg);
+          }
+        }
+      }
+      TC_ST32(ts, (preg + 0));
+      TC_ST32(ts + 32, (preg + 32));
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar_pready(x));
+    }
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_pvdone(x), (uint32_t)(nt - 1) & 1u, abort_flag, p.status));
+    if (ok) {
+      tc_fence_after();
+      const int trow = x * 128 + row;                                // row inside the 256-row CTA tile
+      const int fr = mt * TMW + trow;
+      const bool valid = fr < total_fr;
+      if (p.n_splits == 1) {
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        const int qr = valid ? fr / p.hpg : 0, hh = valid ? fr % p.hpg : 0;
+        __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD;
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t oreg[32];
+          TC_LD32(to + cb * 32, oreg);
+          tc_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int c = 0; c < 32; c += 8) {
+              uint4 v;
+              v.x = pack_bf16(__uint_as_float(oreg[c + 0]) * inv, __uint_as_float(oreg[c + 1]) * inv);
+              v.y = pack_bf16(__uint_as_float(oreg[c + 2]) * inv, __uint_as_float(oreg[c + 3]) * inv);
+              v.z = pack_bf16(__uint_as_float(oreg[c + 4]) * inv, __uint_as_float(oreg[c + 5]) * inv);
+              v.w = pack_bf16(__uint_as_float(oreg[c + 6]) * inv, __uint_as_float(oreg[c + 7]) * inv);
+              *reinterpret_cast<uint4*>(orow + cb * 32 + c) = v;
+            }
+          }
+        }
+        if (valid && p.lse)
+          p.lse[(size_t)(g * p.hpg + hh) * p.lse_stride + qr] = (m_ref + log2f(l)) * 0.6931471805599453f;
+      } else if (__all_sync(0xffffffffu, mbar_wait(bar_alldone, 0u, abort_flag, p.status)) &&
+                 __any_sync(0xffffffffu, valid)) {
+        // cluster mode: partial into own shared memory, which overlays the K/V ring -- the other query tile's last
+        // P V product may still be reading its V tile there, hence the wait for every MMA of the CTA
+        float* prow = ps + trow * PROW;
+#pragma unroll
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t oreg[32];
+          TC_LD32(to + cb * 32, oreg);
+          tc_wait_ld();
+          if (valid) {
+#pragma unroll
+            for (int c = 0; c < 32; c += 4)
+              *reinterpret_cast<uint4*>(prow + cb * 32 + c) = make_uint4(oreg[c], oreg[c + 1], oreg[c + 2], oreg[c + 3]);
+          }
+        }
+        if (valid) { ps[TMW * PROW + 2 * trow] = m_ref; ps[TMW * PROW + 2 * trow + 1] = l; }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem, 512);
+  }
+  if (p.n_splits > 1) cluster_merge<TMW, NTHREADS_W>(p, g, mt, total_fr, split, sSlot);
 }
 
 // Stand-alone merge (used when there are more query tiles than arrival counters): out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s, one warp per stacked row.
@@ -732,6 +1109,38 @@ int pick_splits(const focus_ctx* ctx, int base_ctas, int max_tiles) {
   return s > 8 ? 8 : s;                      // at most 8 splits: they form one (portable-size) thread-block cluster
 }
 
+// Can `n` CTAs of this kernel (one per SM, maximum shared memory) be co-scheduled as one thread-block cluster?
+template <typename K>
+static bool cluster_fits(K kernel, int n, int threads, int smem) {
+  cudaLaunchConfig_t qc = {};
+  qc.gridDim = dim3(n, n, 1); qc.blockDim = dim3(threads, 1, 1); qc.dynamicSmemBytes = smem;
+  cudaLaunchAttribute qa[1];
+  qa[0].id = cudaLaunchAttributeClusterDimension;
+  qa[0].val.clusterDim.x = 1; qa[0].val.clusterDim.y = n; qa[0].val.clusterDim.z = 1;
+  qc.attrs = qa; qc.numAttrs = 1;
+  int n_clusters = 0;
+  const cudaError_t e = cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &qc);
+  if (e != cudaSuccess) cudaGetLastError();
+  return e == cudaSuccess && n_clusters >= 1;
+}
+
+template <typename K>
+static focus_status launch_clustered(K kernel, dim3 grid, int threads, int smem, int cluster_y, cudaStream_t st,
+                                     const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
+                                     const CUtensorMap& d, const TcParams& p) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = dim3(threads, 1, 1); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = cluster_y; at[0].val.clusterDim.z = 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kernel, a, b, c, d, p) != cudaSuccess) {
+    cudaGetLastError();
+    return FOCUS_ERR_CUDA;
+  }
+  return FOCUS_OK;
+}
+
 }  // namespace
 
 bool attn_tc_supported(const focus_ctx* ctx, const AttnArgs& a) {
@@ -758,13 +1167,41 @@ focus_status launch_attn_tc(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st) 
 focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, const SinkGather* pre, cudaStream_t st) {
   const focus_shape& sh = a.sh;
   const int Hkv = sh.n_kv_heads, hpg = sh.n_q_heads / Hkv;
-  const int n_mtiles = (int)(((long long)a.max_rows * hpg + TM - 1) / TM);
-  if (n_mtiles == 0) return FOCUS_OK;
-  const int base = n_mtiles * Hkv;
+  const long long stacked = (long long)a.max_rows * hpg;            // stacked query rows per KV head (host bound)
+  if (stacked == 0) return FOCUS_OK;
   const int ns_pad = a.dense ? 0 : (a.n_sink + TN - 1) / TN * TN;
   const int n_resp = a.dense ? (sh.L + TN - 1) / TN : (sh.L - sh.M + TN - 1) / TN;
   const int max_tiles = a.dense ? n_resp : a.max_blocks + ns_pad / TN + n_resp;
-  const int n_splits = pick_splits(ctx, base, max_tiles);
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_tc_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES_W) != cudaSuccess)
+      return FOCUS_ERR_CUDA;
+    attr_set = true;
+  }
+  static int cluster_ok[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};            // per cluster size: 0 unknown, 1 yes, -1 no
+  static int cluster_ok_w[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+  // two query tiles per CTA when a KV head has at least 256 stacked rows (tensor-bound regime)
+  bool wide = stacked >= TMW && !ctx->no_wide;
+  int n_mtiles = 0, base = 0, n_splits = 1;
+  if (wide) {
+    n_mtiles = (int)((stacked + TMW - 1) / TMW);
+    base = n_mtiles * Hkv;
+    n_splits = pick_splits(ctx, base, max_tiles);
+    if (n_splits > 1) {
+      if (cluster_ok_w[n_splits] == 0)
+        cluster_ok_w[n_splits] = cluster_fits(attn_tc_wide_kernel, n_splits, NTHREADS_W, SMEM_BYTES_W) ? 1 : -1;
+      if (cluster_ok_w[n_splits] != 1) wide = false;                  // its splits merge through a cluster only
+    }
+    // it pays on long key streams (measured: +6 % on dense 32K); with a few dozen tiles per CTA the one-tile kernel
+    // without a key split is faster
+    if (max_tiles / n_splits < 32) wide = false;
+  }
+  if (!wide) {
+    n_mtiles = (int)((stacked + TM - 1) / TM);
+    base = n_mtiles * Hkv;
+    n_splits = pick_splits(ctx, base, max_tiles);
+  }
 
   __nv_bfloat16* gK = nullptr; __nv_bfloat16* gV = nullptr; uint8_t* mask = nullptr;
   if (ns_pad > 0) {
@@ -776,32 +1213,15 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
       mask = ws.get<uint8_t>((size_t)Hkv * ns_pad);
     }
   }
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
-      return FOCUS_ERR_CUDA;
-    attr_set = true;
-  }
-  // can the splits of a tile be co-scheduled as one cluster?  (asked once per cluster size)
-  static int cluster_ok[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};          // 0 unknown, 1 yes, -1 no
   bool use_cluster = false;
-  if (n_splits > 1) {
-    if (cluster_ok[n_splits] == 0) {
-      cudaLaunchConfig_t qc = {};
-      qc.gridDim = dim3(n_splits, n_splits, 1); qc.blockDim = dim3(NTHREADS, 1, 1); qc.dynamicSmemBytes = SMEM_BYTES;
-      cudaLaunchAttribute qa[1];
-      qa[0].id = cudaLaunchAttributeClusterDimension;
-      qa[0].val.clusterDim.x = 1; qa[0].val.clusterDim.y = n_splits; qa[0].val.clusterDim.z = 1;
-      qc.attrs = qa; qc.numAttrs = 1;
-      int n_clusters = 0;
-      const cudaError_t e = cudaOccupancyMaxActiveClusters(&n_clusters, attn_tc_kernel, &qc);
-      cluster_ok[n_splits] = (e == cudaSuccess && n_clusters >= 1) ? 1 : -1;
-      if (e != cudaSuccess) cudaGetLastError();
-    }
+  if (n_splits > 1 && !wide) {
+    if (cluster_ok[n_splits] == 0)
+      cluster_ok[n_splits] = cluster_fits(attn_tc_kernel, n_splits, NTHREADS, SMEM_BYTES) ? 1 : -1;
     use_cluster = cluster_ok[n_splits] == 1;
   }
+  if (wide) use_cluster = n_splits > 1;
   float* part_O = nullptr; float* part_ml = nullptr;
-  if (n_splits > 1 && !use_cluster) {
+  if (n_splits > 1 && !use_cluster && !wide) {
     part_O = ws.get<float>((size_t)base * n_splits * TM * HD);
     part_ml = ws.get<float>((size_t)base * n_splits * TM * 2);
   }
@@ -831,7 +1251,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.q_rows = a.q_rows; p.n_rows = a.n_rows; p.block_idx = a.block_idx; p.block_cnt = a.block_cnt;
   p.sink_mask = mask; p.part_O = part_O; p.part_ml = part_ml;
   p.cluster = use_cluster ? 1 : 0;
-  p.counters = (n_splits > 1 && !use_cluster && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
+  p.counters = (n_splits > 1 && !use_cluster && !wide && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
                    ? ctx->d_counters : nullptr;
   p.q_stride_row = sh.q_stride_row; p.q_stride_head = sh.q_stride_head;
   p.q_base = a.q_base; p.n_q = a.n_q; p.rows_bound = a.max_rows; p.L = sh.L; p.M = sh.M; p.H = sh.n_q_heads;
@@ -844,23 +1264,24 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.dbg = getenv("FOCUS_TIMELINE") ? (unsigned long long*)(ctx->ws + ctx->ws_bytes - (1 << 20)) : nullptr;
 #endif
 
-  if (use_cluster) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(base, n_splits, 1); cfg.blockDim = dim3(NTHREADS, 1, 1);
-    cfg.dynamicSmemBytes = SMEM_BYTES; cfg.stream = st;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = n_splits; at[0].val.clusterDim.z = 1;
-    cfg.attrs = at; cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, attn_tc_kernel, tmK, tmV, tmSK, tmSV, p) != cudaSuccess) {
-      cudaGetLastError();
-      return FOCUS_ERR_CUDA;
+  ctx->last_attn_variant = wide ? 3 : 2;
+  if (wide) {
+    if (n_splits > 1) {
+      focus_status ls = launch_clustered(attn_tc_wide_kernel, dim3(base, n_splits, 1), NTHREADS_W, SMEM_BYTES_W, n_splits, st,
+                                         tmK, tmV, tmSK, tmSV, p);
+      if (ls != FOCUS_OK) return ls;
+    } else {
+      attn_tc_wide_kernel<<<dim3(base, 1), NTHREADS_W, SMEM_BYTES_W, st>>>(tmK, tmV, tmSK, tmSV, p);
     }
+  } else if (use_cluster) {
+    focus_status ls = launch_clustered(attn_tc_kernel, dim3(base, n_splits, 1), NTHREADS, SMEM_BYTES, n_splits, st, tmK, tmV,
+                                       tmSK, tmSV, p);
+    if (ls != FOCUS_OK) return ls;
   } else {
     attn_tc_kernel<<<dim3(base, n_splits), NTHREADS, SMEM_BYTES, st>>>(tmK, tmV, tmSK, tmSV, p);
   }
   FOCUS_CHECK_LAUNCH();
-  if (n_splits > 1 && !p.counters && !use_cluster) {
+  if (n_splits > 1 && !p.counters && !use_cluster && !wide) {
     const int rows_total = base * TM;
     attn_combine_kernel<<<rows_total / 8, 256, 0, st>>>(part_O, part_ml, n_splits, n_mtiles, hpg, sh.n_q_heads,
                                                         a.q_rows, a.n_rows, a.max_rows, a.n_q,

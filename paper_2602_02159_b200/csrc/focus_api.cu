@@ -46,6 +46,8 @@ extern "C" focus_status focus_create(focus_ctx** out, int device, size_t workspa
   c->sm_count = prop.multiProcessorCount;
   c->ws_bytes = workspace_bytes ? workspace_bytes : (size_t)256 << 20;
   c->force_simt = 0;
+  c->last_attn_variant = 0;
+  c->no_wide = getenv("FOCUS_NO_WIDE") != nullptr;
   c->encode_tiled = nullptr;
   if (prop.major == 10) {   // tensor-core kernels are built for sm_100a only
     cudaDriverEntryPointQueryResult q;
@@ -81,6 +83,8 @@ extern "C" int32_t focus_set_force_simt(focus_ctx* ctx, int32_t force) {
   ctx->force_simt = force ? 1 : 0;
   return prev;
 }
+
+extern "C" int32_t focus_last_attn_variant(focus_ctx* ctx) { return ctx ? ctx->last_attn_variant : -1; }
 
 extern "C" focus_status focus_poll_status(focus_ctx* ctx, focus_stream stream, int32_t* device_status) {
   if (!ctx || !device_status) return FOCUS_ERR_INVALID_ARG;
@@ -123,6 +127,7 @@ static focus_status attn_common(focus_ctx* ctx, const focus_shape* shape, const 
 static focus_status attn_dispatch(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st) {
   if (a.max_rows == 0) return FOCUS_OK;
   if (!ctx->force_simt && attn_tc_supported(ctx, a)) return launch_attn_tc(ctx, a, st);
+  ctx->last_attn_variant = 1;
   return launch_attn_simt(ctx, a, st);
 }
 
