@@ -327,7 +327,7 @@ def run_focus(args):
                "sparse_layer_ms": gs, "sparse_retained_tflops": fl_sparse / gs / 1e9,
                "sparse_dense_equiv_tflops": fl_dense / gs / 1e9,
                "roofline": {"bound": "tensor", "achieved": fl_dense / gd / 1e9, "peak": P["tf_sust"], "unit": "TFLOP/s",
-                            "frac": fl_dense / gd / 1e9 / P["tf_sust"], "kernel": "attn_tc_kernel (dense layer, 512 rows)",
+                            "frac": fl_dense / gd / 1e9 / P["tf_sust"], "kernel": "attn_tc_wide_kernel (dense layer, 512 gen rows)",
                             "peak_source": f"{P['src']} sustained bf16"}}
     assert ctx.poll_status() == 0
 
@@ -386,7 +386,7 @@ def run_focus(args):
                    "sparse_layer_frac_of_hbm": sparse_bytes / (sparse_ms * 1e-3) / 1e9 / P["hbm"],
                    "per_layer_sparse_vs_dense": dense_ms / sparse_ms},
         "roofline": {"bound": "hbm", "achieved": dense_gbs, "peak": P["hbm"], "unit": "GB/s", "frac": dense_gbs / P["hbm"],
-                     "traffic": traffic, "kernel": "attn_tc_kernel + attn_combine_kernel (dense layer, I_active rows)",
+                     "traffic": traffic, "kernel": "attn_tc_kernel incl. its in-cluster split merge (dense layer, I_active rows)",
                      "bytes_per_launch": kv_bytes + qo_bytes, "peak_source": f"{P['src']} copy bandwidth"},
         "gen_mode": gen,
         "e2e": {"value": ms_e2e, "unit": "ms", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
@@ -488,6 +488,94 @@ def run_sweep(args):
     print(json.dumps({"sweep": out, "peaks": P}))
 
 
+def run_stages(args):
+    """Per-stage latency of one configuration (graph replay over a few rotating layer copies so that inputs do not
+    sit in L2), for the paper's I_active rows and for the gen-region rows."""
+    import torch
+
+    from paper_2602_02159_b200 import binding as fb
+    from paper_2602_02159_b200 import build as fbuild
+    from paper_2602_02159_b200 import step as fstep
+    from paper_2602_02159_b200 import workloads as wl
+    fbuild.build()
+    torch.cuda.set_device(0)
+    ctx = fb.Context(0, workspace_bytes=512 << 20)
+    P = peaks()
+    w = wl.config(args.config)
+    s = w.shape
+    eb = 4 if s.dtype == "f32" else 2
+    layer_bytes = 2 * s.Hkv * s.L * s.d * eb
+    NL = max(2, min(8, -(-400_000_000 // layer_bytes)))
+    Qs, Ks, Vs, Kb = [], [], [], []
+    for l in range(NL):
+        t = wl.gen_qkv(s, l)
+        Qs.append(fstep.to_device(t["Q"], s.dtype)); Ks.append(fstep.to_device(t["K"], s.dtype))
+        Vs.append(fstep.to_device(t["V"], s.dtype))
+    c_prev, _ = wl.gen_confidence(w.seed, s.N)
+    conf = torch.from_numpy(wl.full_conf(s, c_prev)).cuda()
+    masked = torch.from_numpy(wl.gen_masked(w)).cuda()
+    ba = fstep.StepBuffers(w, rows="active")
+    bg = fstep.StepBuffers(w, rows="gen")
+    for b in (ba, bg):
+        fstep.select_queries(ctx, b, conf, masked)
+    for l in range(NL):
+        kb = torch.zeros(s.Hkv, s.nb, s.d, dtype=torch.float32, device="cuda")
+        fb.focus_pool_keys(ctx, ba.shape, Ks[l], kb)
+        Kb.append(kb)
+    fstep.dense_layer(ctx, ba, Qs[0], Ks[0], Vs[0])
+    fstep.find_sinks(ctx, ba, Qs[0], Ks[0], ba.lse)
+    bg.sink_idx.copy_(ba.sink_idx)
+    lse_keep = ba.lse.clone()
+    torch.cuda.synchronize()
+
+    def graph_time(fn):
+        for l in range(NL):
+            fn(l)
+        torch.cuda.synchronize()
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            for l in range(NL):
+                fn(l)
+        for _ in range(3):
+            gr.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            gr.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return round(e0.elapsed_time(e1) / 20 / NL * 1e3, 2)
+
+    na = int(ba.n_active.item())
+    keys = w.C * s.B + w.n_sink + s.N
+    out = {"workload": w.name, "n_active": na, "retained_keys_per_head": keys, "layers_rotated": NL, "us": {}}
+    u = out["us"]
+    u["select_queries"] = graph_time(lambda l: fstep.select_queries(ctx, ba, conf, masked))
+    u["find_sinks (with LSE of the dense pass)"] = graph_time(lambda l: fstep.find_sinks(ctx, ba, Qs[l], Ks[l], lse_keep))
+    u["pool_keys"] = graph_time(lambda l: fb.focus_pool_keys(ctx, ba.shape, Ks[l], Kb[l]))
+    u["score_blocks cold (streams K)"] = graph_time(lambda l: fb.focus_score_blocks(
+        ctx, ba.shape, Qs[l], s.M, ba.focus_idx, ba.n_focus, max(1, w.k), Ks[l], None, 0, ba.R))
+    for name, b in (("I_active rows", ba), ("gen rows", bg)):
+        q_rows, n_rows, max_rows = b._rows()
+        n_q = na if b is ba else s.N
+        d_us = graph_time(lambda l: fstep.dense_layer(ctx, b, Qs[l], Ks[l], Vs[l]))
+        l_us = graph_time(lambda l: fstep.sparse_layer(ctx, b, Qs[l], Ks[l], Vs[l], Kbar=Kb[l]))
+        a_us = graph_time(lambda l: fb.focus_sparse_attn(
+            ctx, b.shape, Qs[l], s.M, s.N, q_rows, n_rows, max_rows, Ks[l], Vs[l], fb.HEADS_PER_KV_GROUP, b.block_idx,
+            b.max_blocks, b.block_cnt, b.sink_idx, b.sink_keep, w.n_sink, b.O, b.lse))
+        fl_d, fl_s = 4.0 * n_q * s.L * s.d * s.H, 4.0 * n_q * keys * s.d * s.H
+        by_d = 2.0 * s.Hkv * s.L * s.d * eb
+        by_s = 2.0 * s.Hkv * keys * s.d * eb
+        u[name] = {"n_q": n_q, "dense_attn": d_us, "sparse_layer (score+select+attn)": l_us, "sparse_attn": a_us,
+                   "dense_TFLOPs": round(fl_d / d_us / 1e6, 1), "dense_GBps": round(by_d / d_us / 1e3, 1),
+                   "sparse_retained_TFLOPs": round(fl_s / a_us / 1e6, 1), "sparse_GBps": round(by_s / a_us / 1e3, 1),
+                   "sparse_attn_vs_dense": round(d_us / a_us, 2)}
+    assert ctx.poll_status() == 0
+    out["peaks"] = P
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -498,10 +586,13 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (quick runs)")
     ap.add_argument("--skip-gen", action="store_true", help="skip the gen-region-rows (tensor-bound) measurements")
     ap.add_argument("--no-graph", action="store_true", help="time eager C-ABI calls instead of a CUDA graph replay")
+    ap.add_argument("--stages", action="store_true", help="per-stage latencies of --config (0..3) instead of the step")
     ap.add_argument("--sweep", action="store_true", help="run the context x keep-ratio sweep (config 4) instead")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle baseline leg")
     args = ap.parse_args()
-    if args.sweep:
+    if args.stages:
+        run_stages(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args)
