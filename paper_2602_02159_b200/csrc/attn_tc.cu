@@ -15,6 +15,9 @@
 // fixed split order, so results are deterministic.
 #include <stdlib.h>
 
+#include <stdio.h>
+#include <stdlib.h>
+
 #include "tc_common.cuh"
 
 using namespace tc;
@@ -1109,9 +1112,10 @@ int pick_splits(const focus_ctx* ctx, int base_ctas, int max_tiles) {
   return s > 8 ? 8 : s;                      // at most 8 splits: they form one (portable-size) thread-block cluster
 }
 
-// Can `n` CTAs of this kernel (one per SM, maximum shared memory) be co-scheduled as one thread-block cluster?
+// How many clusters of `n` CTAs of this kernel (one CTA per SM, maximum shared memory) can be resident at once on
+// this device.  It depends on how the enabled SMs are spread over the GPCs, which differs from chip to chip.
 template <typename K>
-static bool cluster_fits(K kernel, int n, int threads, int smem) {
+static int cluster_capacity(K kernel, int n, int threads, int smem) {
   cudaLaunchConfig_t qc = {};
   qc.gridDim = dim3(n, n, 1); qc.blockDim = dim3(threads, 1, 1); qc.dynamicSmemBytes = smem;
   cudaLaunchAttribute qa[1];
@@ -1120,8 +1124,8 @@ static bool cluster_fits(K kernel, int n, int threads, int smem) {
   qc.attrs = qa; qc.numAttrs = 1;
   int n_clusters = 0;
   const cudaError_t e = cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &qc);
-  if (e != cudaSuccess) cudaGetLastError();
-  return e == cudaSuccess && n_clusters >= 1;
+  if (e != cudaSuccess) { cudaGetLastError(); return 0; }
+  return n_clusters;
 }
 
 template <typename K>
@@ -1179,8 +1183,11 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
       return FOCUS_ERR_CUDA;
     attr_set = true;
   }
-  static int cluster_ok[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};            // per cluster size: 0 unknown, 1 yes, -1 no
-  static int cluster_ok_w[9] = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+  // resident-cluster capacity per cluster size (-1 = not asked yet): a launch whose clusters do not all fit at once
+  // would run in two waves, so such launches fall back to the merge through global memory (narrow kernel) or to
+  // the narrow kernel (wide kernel)
+  static int cluster_cap[9] = {-1, -1, -1, -1, -1, -1, -1, -1, -1};
+  static int cluster_cap_w[9] = {-1, -1, -1, -1, -1, -1, -1, -1, -1};
   // two query tiles per CTA when a KV head has at least 256 stacked rows (tensor-bound regime)
   bool wide = stacked >= TMW && !ctx->no_wide;
   int n_mtiles = 0, base = 0, n_splits = 1;
@@ -1189,9 +1196,9 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     base = n_mtiles * Hkv;
     n_splits = pick_splits(ctx, base, max_tiles);
     if (n_splits > 1) {
-      if (cluster_ok_w[n_splits] == 0)
-        cluster_ok_w[n_splits] = cluster_fits(attn_tc_wide_kernel, n_splits, NTHREADS_W, SMEM_BYTES_W) ? 1 : -1;
-      if (cluster_ok_w[n_splits] != 1) wide = false;                  // its splits merge through a cluster only
+      if (cluster_cap_w[n_splits] < 0)
+        cluster_cap_w[n_splits] = cluster_capacity(attn_tc_wide_kernel, n_splits, NTHREADS_W, SMEM_BYTES_W);
+      if (cluster_cap_w[n_splits] < base) wide = false;               // its splits merge through a cluster only
     }
     // it pays on long key streams (measured: +6 % on dense 32K); with a few dozen tiles per CTA the one-tile kernel
     // without a key split is faster
@@ -1215,9 +1222,13 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   }
   bool use_cluster = false;
   if (n_splits > 1 && !wide) {
-    if (cluster_ok[n_splits] == 0)
-      cluster_ok[n_splits] = cluster_fits(attn_tc_kernel, n_splits, NTHREADS, SMEM_BYTES) ? 1 : -1;
-    use_cluster = cluster_ok[n_splits] == 1;
+    // the largest split count (not above the one wanted) whose clusters are all resident at once; if even two-CTA
+    // clusters do not fit, keep the wanted count and merge through global memory
+    for (int sp = n_splits; sp >= 2; --sp) {
+      if (cluster_cap[sp] < 0) cluster_cap[sp] = cluster_capacity(attn_tc_kernel, sp, NTHREADS, SMEM_BYTES);
+      if (cluster_cap[sp] >= base) { n_splits = sp; use_cluster = true; break; }
+    }
+    if (getenv("FOCUS_LOG")) fprintf(stderr, "[focus] attn: base %d splits %d cluster %d\n", base, n_splits, (int)use_cluster);
   }
   if (wide) use_cluster = n_splits > 1;
   float* part_O = nullptr; float* part_ml = nullptr;

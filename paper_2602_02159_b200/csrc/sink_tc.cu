@@ -32,6 +32,7 @@ struct SinkParams {
   int q_base, L, hpg, max_active, n_pad, n_slots, lse_stride, chunks;
   int n_buf, buf_cols;           // accumulator ring in TMEM: n_buf buffers of buf_cols columns
   int Hkv, n_ctas, groups_staged; // flat split of the Hkv*T key tiles over n_ctas CTAs; a CTA touches <= groups_staged heads
+  int kv_div;                     // the kernel walks QUERY heads (Hkv = H, hpg = 1); query head h reads KV head h / kv_div
   float scale_log2;
   int32_t* status;
 };
@@ -126,8 +127,8 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
         const uint32_t dst = sSlot + slot * SLOT_BYTES;
         mbar_expect_tx(bar_full(slot), SLOT_BYTES);
         const int u = u0 + i;
-        tma_load_3d(dst, &tmK, bar_full(slot), 0, (u % T) * TK, u / T);
-        tma_load_3d(dst + HALF_BYTES, &tmK, bar_full(slot), 64, (u % T) * TK, u / T);
+        tma_load_3d(dst, &tmK, bar_full(slot), 0, (u % T) * TK, u / T / p.kv_div);
+        tma_load_3d(dst + HALF_BYTES, &tmK, bar_full(slot), 64, (u % T) * TK, u / T / p.kv_div);
         ++issued;
       }
       if (!ok) {
@@ -223,15 +224,20 @@ static int sink_slots(int heads_staged, int n_pad) {
 
 bool sink_tc_supported(const focus_ctx* ctx, const focus_shape* s, int max_active) {
   if (!ctx->encode_tiled || s->dtype != FOCUS_BF16 || s->head_dim != HD) return false;
-  const int n_pad = sink_npad(max_active), hpg = s->n_q_heads / s->n_kv_heads;
-  return n_pad <= MAX_NPAD && sink_slots(hpg, n_pad) >= 2;
+  const int n_pad = sink_npad(max_active);
+  return n_pad <= MAX_NPAD && sink_slots(1, n_pad) >= 2;
 }
 
 focus_status launch_sink_colsum_tc(focus_ctx* ctx, const focus_shape* s, const void* Q, int q_base,
                                    const int32_t* active_idx, const int32_t* n_active, int max_active, const void* K,
                                    const float* lse, float* part, WsAlloc&, cudaStream_t st) {
-  const int Hkv = s->n_kv_heads, hpg = s->n_q_heads / Hkv;
+  // Every query head is walked on its own (its key tiles come from KV head h / (H / Hkv)): with GQA the K tiles of
+  // a KV head are then read once per query head of the group, from L2 after the first, but a CTA stages the
+  // queries of at most two heads instead of two whole groups.
+  const int kvh = s->n_kv_heads, H = s->n_q_heads;
+  const int Hkv = H, hpg = 1;
   SinkParams p;
+  p.kv_div = H / kvh;
   p.Q = (const __nv_bfloat16*)Q; p.active_idx = active_idx; p.n_active = n_active; p.lse = lse; p.part = part;
   p.q_stride_row = s->q_stride_row; p.q_stride_head = s->q_stride_head;
   p.q_base = q_base; p.L = s->L; p.hpg = hpg; p.max_active = max_active; p.n_pad = sink_npad(max_active);
@@ -260,7 +266,7 @@ focus_status launch_sink_colsum_tc(focus_ctx* ctx, const focus_shape* s, const v
   p.scale_log2 = shape_scale(s) * 1.4426950408889634f;
   p.status = ctx->d_status;
   CUtensorMap tmK;
-  if (!encode_kv_map(ctx->encode_tiled, &tmK, K, HD, s->L, Hkv, s->kv_stride_tok, s->kv_stride_head, 64, TK))
+  if (!encode_kv_map(ctx->encode_tiled, &tmK, K, HD, s->L, kvh, s->kv_stride_tok, s->kv_stride_head, 64, TK))
     return FOCUS_ERR_INVALID_ARG;
   const int hs = p.groups_staged * hpg;
   const int smem = 1024 + hs * p.n_pad * 256 + p.n_slots * SLOT_BYTES + (2 * MAX_SLOTS + 2 * MAX_BUF) * 8 + 16 +
