@@ -192,22 +192,31 @@ __global__ void sink_reduce_heads_kernel(const float* __restrict__ part, int H, 
 }
 
 constexpr int TN_THREADS = 1024;
-constexpr int TN_MAX_SMEM_KEYS = 56 * 1024;      // keys cached in shared memory (224 KB); beyond that they are re-read
+constexpr int TN_MAX_SMEM_KEYS = 50 * 1024;      // keys cached in shared memory (200 KB); beyond that they are re-read
 
 // One CTA.  Keys (order-preserving integers of the scores) are staged once in shared memory, then:
-// (1) the key T of the want-th largest element is found bit by bit, MSB first: T keeps a bit iff at least `want`
-//     keys are >= the candidate -- 32 counting sweeps with no atomics and one barrier each (sink scores are all
-//     close to 1/L, which makes histogram-based radix passes collide on one counter);
-// (2) an ordered compaction in which warp w owns the w-th contiguous segment of the candidates (ballot/popc
-//     keeps index order inside a warp, one block scan orders the warps); keys equal to T are taken in index
-//     order until the quota is filled.
+// (1) the key T of the want-th largest element is found bit by bit, MSB first (T keeps a bit iff at least `want`
+//     keys are >= the candidate): counting sweeps with no atomics per element.  Sink scores are all close to 1/L,
+//     so (a) the bits on which all keys agree are found first (one AND/OR sweep) and skipped, and (b) as soon as
+//     at most LIST_MAX keys are still undecided (same prefix as T) they are copied to a short list and the
+//     remaining bits only look at the list;
+// (2) the selected positions are written ascending.  If every key equal to T is taken (no tie is cut) they are
+//     collected in any order and ranked by position; otherwise warp w walks the w-th contiguous segment of the
+//     candidates (ballot/popc keeps index order, one block scan orders the warps) and keys equal to T are taken in
+//     index order until the quota is filled.
+constexpr int LIST_MAX = TN_THREADS;
+constexpr int SEL_MAX = 4096;
+
 template <bool CACHED>
 __global__ void __launch_bounds__(TN_THREADS)
 sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const int32_t* n_active,
                  int32_t* __restrict__ sink_idx, int32_t* status) {
   extern __shared__ uint32_t skey[];
-  __shared__ int cnt[33];
+  __shared__ int cnt[40];
   __shared__ int scan_s[33];
+  __shared__ uint32_t s_and, s_or;
+  __shared__ uint32_t list[LIST_MAX];
+  __shared__ int sel[SEL_MAX];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = hi - lo;
   const int want = min(n_sink, n);
@@ -220,34 +229,83 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
     for (int i = tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
     return;
   }
-  if (tid < 33) cnt[tid] = 0;
+  if (tid < 40) cnt[tid] = 0;
+  if (tid == 0) { s_and = 0xFFFFFFFFu; s_or = 0u; }
   if (CACHED) {
 #pragma unroll 8
     for (int i = tid; i < n; i += TN_THREADS) skey[i] = float_key(S[lo + i]);
   }
   __syncthreads();
   auto key_at = [&](int i) -> uint32_t { return CACHED ? skey[i] : float_key(S[lo + i]); };
-  uint32_t T = 0;
-  for (int bit = 31; bit >= 0; --bit) {
-    const uint32_t cand = T | (1u << bit);
+  auto count_ge = [&](uint32_t cand, int slot) -> int {          // block-wide count of keys >= cand (one barrier)
     int c = 0;
 #pragma unroll 8
     for (int i = tid; i < n; i += TN_THREADS) c += key_at(i) >= cand ? 1 : 0;
     c = __reduce_add_sync(0xffffffffu, c);
-    if (lane == 0 && c) atomicAdd(&cnt[bit], c);
+    if (lane == 0 && c) atomicAdd(&cnt[slot], c);
     __syncthreads();
-    if (cnt[bit] >= want) T = cand;
-  }
-  // T = key of the want-th largest element.  Count the strictly greater ones to know how many equal keys to take.
+    return cnt[slot];
+  };
+  // bits shared by all keys
   {
-    int c = 0;
+    uint32_t a = 0xFFFFFFFFu, o = 0u;
 #pragma unroll 8
-    for (int i = tid; i < n; i += TN_THREADS) c += key_at(i) > T ? 1 : 0;
-    c = __reduce_add_sync(0xffffffffu, c);
-    if (lane == 0 && c) atomicAdd(&cnt[32], c);
+    for (int i = tid; i < n; i += TN_THREADS) { const uint32_t k = key_at(i); a &= k; o |= k; }
+    a = __reduce_and_sync(0xffffffffu, a);
+    o = __reduce_or_sync(0xffffffffu, o);
+    if (lane == 0) { atomicAnd(&s_and, a); atomicOr(&s_or, o); }
     __syncthreads();
   }
-  const int remaining = want - cnt[32];          // how many keys == T to take (lowest index first)
+  const uint32_t diff = s_and ^ s_or;
+  const int hb = diff ? 31 - __clz(diff) : -1;                    // highest bit on which two keys differ
+  uint32_t T = hb >= 0 ? (s_or & ~((2u << hb) - 1u)) : s_or;      // common prefix, lower bits still open
+  if (hb == 31) T = 0u;
+  int lo_cnt = n, hi_cnt = 0;                                     // keys >= T; keys >= T + 2^(bit+1)
+  int bit = hb;
+  for (; bit >= 0 && lo_cnt - hi_cnt > LIST_MAX; --bit) {
+    const uint32_t cand = T | (1u << bit);
+    const int c = count_ge(cand, bit);
+    if (c >= want) { T = cand; lo_cnt = c; } else { hi_cnt = c; }
+  }
+  if (bit >= 0) {
+    // undecided keys (prefix above `bit` equal to T's) -> list; the remaining bits only look at the list
+    const uint32_t top = bit == 31 ? 0u : (T >> (bit + 1));
+#pragma unroll 4
+    for (int i = tid; i < n; i += TN_THREADS) {
+      const uint32_t k = key_at(i);
+      if ((bit == 31 ? 0u : (k >> (bit + 1))) == top) list[atomicAdd(&cnt[32], 1)] = k;
+    }
+    __syncthreads();
+    const int nl = cnt[32];
+    const uint32_t mine = tid < nl ? list[tid] : 0u;
+    const int above = hi_cnt;                    // keys above the listed range: they are >= every further candidate
+    for (; bit >= 0; --bit) {
+      const uint32_t cand = T | (1u << bit);
+      int c = (tid < nl && mine >= cand) ? 1 : 0;
+      c = __reduce_add_sync(0xffffffffu, c);
+      if (lane == 0 && c) atomicAdd(&cnt[bit], c);
+      __syncthreads();
+      const int tot = above + cnt[bit];
+      if (tot >= want) { T = cand; lo_cnt = tot; } else { hi_cnt = tot; }
+    }
+  }
+  // T = key of the want-th largest element; hi_cnt = keys > T; lo_cnt - hi_cnt = keys == T
+  const int remaining = want - hi_cnt;           // how many keys == T to take (lowest index first)
+  if (remaining == lo_cnt - hi_cnt && want <= SEL_MAX) {
+    // no tie is cut: the selected set is {key >= T}; collect in any order, then rank by position
+#pragma unroll 4
+    for (int i = tid; i < n; i += TN_THREADS)
+      if (key_at(i) >= T) sel[atomicAdd(&cnt[33], 1)] = lo + i;
+    __syncthreads();
+    for (int t = tid; t < want; t += TN_THREADS) {
+      const int mine = sel[t];
+      int rank = 0;
+      for (int j = 0; j < want; ++j) rank += sel[j] < mine ? 1 : 0;
+      sink_idx[rank] = mine;
+    }
+    for (int i = want + tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
+    return;
+  }
   // ordered compaction: warp w owns candidates [w*seg, (w+1)*seg), seg a multiple of 32
   const int seg = ((n + 31) / 32 + 31) / 32 * 32;
   const int w_lo = min(warp * seg, n), w_hi = min(w_lo + seg, n);
