@@ -20,6 +20,8 @@ Functions and the passages they follow
   select_blocks    B_relevant = Top-C(R_b) and Eq. 8 (I_p).
   sparse_attn      K_attn = concat(K_Ip, K_resp) and Eq. 9.
   dense_attn       "FullAttn" of Algorithm 1: plain bidirectional softmax attention.
+  confidence       Section "Diffusion LLM inference", Eq. 2: predicted token and confidence of a position.
+  update_kv        "Approximate KV cache in dLLMs", Eq. 3: refreshed rows replace the cached ones.
 
 Readings where the paper leaves a choice (parity unpinned by the paper for these):
   * Eq. 6 writes one softmax over an "aggregated query representation"; here every
@@ -218,3 +220,33 @@ def dense_attn(Q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float,
     for h in (range(H) if heads is None else heads):
         O[:, h, :], lse[h] = _attend(Q[:, h, :], K[h // hpg], V[h // hpg], None, scale)
     return O, lse
+
+
+# ----------------------------------------------------------------------------- Eq. 2
+def confidence(logits: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Eq. 2 for each row of `logits` [n, V]: the predicted token argmax_v p(v) (lowest v on ties) and its
+    confidence c = max_v p(v), with p = softmax(logits) over the vocabulary.  NaN logits count as -inf."""
+    x = np.asarray(logits, dtype=np.float64).copy()
+    x[np.isnan(x)] = -np.inf
+    tok = np.zeros(x.shape[0], dtype=np.int64)
+    conf = np.zeros(x.shape[0], dtype=np.float64)
+    for r in range(x.shape[0]):
+        row = x[r]
+        m = row.max()
+        p = np.exp(row - m)
+        p = p / p.sum()
+        tok[r] = int(np.argmax(p))          # first occurrence = lowest index
+        conf[r] = p[tok[r]]
+    return conf, tok
+
+
+# ----------------------------------------------------------------------------- Eq. 3
+def update_kv(K_cache: np.ndarray, V_cache: np.ndarray, K_new: np.ndarray, V_new: np.ndarray,
+              rows: Sequence[int]) -> Tuple[np.ndarray, np.ndarray]:
+    """Eq. 3: K_i = f_K(x)_i for i in the refreshed set U (here `rows`, with the new states K_new[r] for rows[r]),
+    the cached state otherwise; same for V.  Caches are [Hkv, L, d], new states [n, Hkv, d].  Returns new arrays."""
+    K, V = np.array(K_cache, copy=True), np.array(V_cache, copy=True)
+    for r, pos in enumerate(rows):
+        K[:, int(pos), :] = K_new[r]
+        V[:, int(pos), :] = V_new[r]
+    return K, V

@@ -352,6 +352,52 @@ def test_sparse_output_approaches_dense_when_dropped_keys_carry_no_mass():
     assert np.allclose(Os, Od, atol=1e-12)
 
 
+# ------------------------------------------------------------------ confidence (Eq. 2), cache update (Eq. 3)
+def test_confidence_closed_forms_library_and_ties():
+    from scipy.special import softmax
+    rng = np.random.default_rng(43)
+    x = rng.standard_normal((5, 300)) * 3
+    conf, tok = fo.confidence(x)
+    p = softmax(x, axis=1)
+    assert np.array_equal(tok, p.argmax(axis=1)) and np.allclose(conf, p.max(axis=1), atol=1e-15)
+    # uniform logits: every token has probability 1/V, the lowest index wins the tie
+    c, t = fo.confidence(np.full((1, 64), 2.5))
+    assert t[0] == 0 and abs(c[0] - 1 / 64) < 1e-15
+    # logits ln(6), ln(3), ln(1): probabilities 0.6, 0.3, 0.1
+    c, t = fo.confidence(np.log(np.array([[1.0, 6.0, 3.0]])))
+    assert t[0] == 1 and abs(c[0] - 0.6) < 1e-15
+    # a tie between positions 2 and 5, and a NaN that must not win
+    row = np.array([[0.0, -1.0, 4.0, np.nan, 1.0, 4.0]])
+    c, t = fo.confidence(row)
+    z = 2 * math.exp(4) + math.exp(0) + math.exp(-1) + math.exp(1)
+    assert t[0] == 2 and abs(c[0] - math.exp(4) / z) < 1e-15
+    # shifting a row by a constant changes nothing (softmax invariance)
+    c2, t2 = fo.confidence(x + 1000.0)
+    assert np.array_equal(t2, tok) and np.allclose(c2, conf, atol=1e-12)
+
+
+def test_update_kv_replaces_exactly_the_listed_rows():
+    rng = np.random.default_rng(47)
+    K, V = rng.standard_normal((2, 10, 4)), rng.standard_normal((2, 10, 4))
+    Kn, Vn = rng.standard_normal((3, 2, 4)), rng.standard_normal((3, 2, 4))
+    K2, V2 = fo.update_kv(K, V, Kn, Vn, [7, 2, 9])
+    untouched = [0, 1, 3, 4, 5, 6, 8]
+    assert np.array_equal(K2[:, untouched], K[:, untouched]) and np.array_equal(V2[:, untouched], V[:, untouched])
+    for r, pos in enumerate([7, 2, 9]):
+        assert np.array_equal(K2[:, pos], Kn[r]) and np.array_equal(V2[:, pos], Vn[r])
+    assert not np.shares_memory(K2, K)
+    # an empty refresh set leaves the cache as it is
+    K3, V3 = fo.update_kv(K, V, Kn[:0], Vn[:0], [])
+    assert np.array_equal(K3, K) and np.array_equal(V3, V)
+    # refreshed attention equals attention over the refreshed cache (the two stages compose)
+    Q = rng.standard_normal((2, 2, 4))
+    O1, _ = fo.dense_attn(Q, K2, V2, 0.5)
+    Kc, Vc = K.copy(), V.copy()
+    Kc[:, [7, 2, 9]] = np.transpose(Kn, (1, 0, 2)); Vc[:, [7, 2, 9]] = np.transpose(Vn, (1, 0, 2))
+    O2, _ = fo.dense_attn(Q, Kc, Vc, 0.5)
+    assert np.array_equal(O1, O2)
+
+
 # ------------------------------------------------------------------ generators (inputs only)
 def test_bf16_round_trip_and_rne():
     x = np.array([1.0, 1.00390625, 1.01171875, -2.5, 3.140625], dtype=np.float32)   # 1+2^-8 ties to even
