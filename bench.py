@@ -556,6 +556,19 @@ def run_stages(args):
     u["pool_keys"] = graph_time(lambda l: fb.focus_pool_keys(ctx, ba.shape, Ks[l], Kb[l]))
     u["score_blocks cold (streams K)"] = graph_time(lambda l: fb.focus_score_blocks(
         ctx, ba.shape, Qs[l], s.M, ba.focus_idx, ba.n_focus, max(1, w.k), Ks[l], None, 0, ba.R))
+    # loop-closing stages: confidence from logits (LLaDA vocabulary, bf16) for the I_active rows, KV refresh of those rows
+    V = 126464
+    logits = (torch.randn(s.N, V, device="cuda") * 2).to(torch.bfloat16)
+    cconf = torch.zeros(ba.max_active, dtype=torch.float32, device="cuda")
+    ctok = torch.zeros(ba.max_active, dtype=torch.int32, device="cuda")
+    t_conf = graph_time(lambda l: fb.focus_confidence(ctx, logits, fb.BF16, V, V, s.M, s.N, ba.active_idx, ba.n_active,
+                                                      ba.max_active, cconf, ctok))
+    u["confidence (Eq. 2), I_active rows x 126464 vocab"] = {"us": t_conf, "GBps": round(na * V * 2 / t_conf / 1e3, 1)}
+    del logits
+    if s.dtype == "bf16":
+        Kn = torch.randn(ba.max_active, s.Hkv, s.d, device="cuda").to(torch.bfloat16)
+        u["update_kv (Eq. 3), I_active rows"] = graph_time(lambda l: fb.focus_update_kv(
+            ctx, ba.shape, Ks[l], Vs[l], Kn, Kn, ba.active_idx, ba.n_active, ba.max_active))
     for name, b in (("I_active rows", ba), ("gen rows", bg)):
         q_rows, n_rows, max_rows = b._rows()
         n_q = na if b is ba else s.N

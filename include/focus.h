@@ -221,6 +221,32 @@ focus_status focus_dense_attn(focus_ctx* ctx, const focus_shape* shape, const vo
                               const int32_t* q_rows, const int32_t* n_rows, int32_t max_rows,
                               const void* K, const void* V, void* O, float* lse, focus_stream stream);
 
+/* ---- closing the decoding loop around the attention path ------------------------------------------ */
+
+/* Eq. 2: for each listed position, the predicted token argmax_v p(v) (lowest v on ties; NaN logits count as
+ * -inf) and its confidence c = max_v p(v), p = softmax over the vocabulary of that position's logits row.
+ * The confidences are the conf_prev of the next step's focus_select_queries; the same selection call with
+ * k = n^(t) and w = 0 picks the positions to unmask ("unmasks the highest-confidence positions").
+ *   logits    [n_pos rows, vocab] for positions [pos_base, pos_base + n_pos), dtype FOCUS_F32 or FOCUS_BF16;
+ *             row_stride in elements, a multiple of 8 (bf16) / 4 (f32); base 16-byte aligned
+ *   rows      int32[max_rows] positions (device) with n_rows int32[1] (device), or both NULL: the first max_rows
+ *             positions
+ *   conf      float[max_rows], token int32[max_rows]; entries beyond n_rows are 0 and -1. */
+focus_status focus_confidence(focus_ctx* ctx, const void* logits, int32_t dtype, int64_t row_stride, int32_t vocab,
+                              int32_t pos_base, int32_t n_pos, const int32_t* rows, const int32_t* n_rows,
+                              int32_t max_rows, float* conf, int32_t* token, focus_stream stream);
+
+/* Eq. 3 / Algorithm 1 ("Update KV Cache for indices in I_active"): the key and value states computed this
+ * step for the listed positions replace the cached rows; every other row keeps its cached state.
+ *   K_cache, V_cache  [Hkv, L, d] by the shape's strides (updated in place)
+ *   K_new, V_new      [max_rows, Hkv, d] contiguous; row r belongs to position rows[r]
+ *   rows int32[max_rows], n_rows int32[1] (device).  Positions outside [0, L) are skipped and reported through
+ * the status word.  Pooled keys are not touched: the listed positions of a non-block-entry step lie in the
+ * response region; after a block-entry refresh of prompt rows call focus_pool_keys again. */
+focus_status focus_update_kv(focus_ctx* ctx, const focus_shape* shape, void* K_cache, void* V_cache,
+                             const void* K_new, const void* V_new, const int32_t* rows, const int32_t* n_rows,
+                             int32_t max_rows, focus_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -53,6 +53,8 @@ _SIGS = {
     "focus_sparse_attn": (_I, [_P, _SH, _P, _I, _I, _P, _P, _I, _P, _P, _I, _P, _I, _P, _P, _P, _I, _P, _P, _P]),
     "focus_sparse_layer": (_I, [_P, _SH, _P, _I, _I, _P, _P, _I, _P, _P, _I, _P, _P, _P, _I, _P, _I, _P, _P, _P, _P, _P,
                                 _P, _P]),
+    "focus_confidence": (_I, [_P, _P, _I, C.c_int64, _I, _I, _I, _P, _P, _I, _P, _P, _P]),
+    "focus_update_kv": (_I, [_P, _SH, _P, _P, _P, _P, _P, _P, _I, _P]),
     "focus_dense_attn": (_I, [_P, _SH, _P, _I, _I, _P, _P, _I, _P, _P, _P, _P, _P]),
 }
 
@@ -219,3 +221,15 @@ def focus_dense_attn(ctx, shape, Q, q_base, n_q, q_rows, n_rows, max_rows, K, V,
     _check(ctx._lib.focus_dense_attn(ctx.handle, C.byref(shape), _ptr(Q), q_base, n_q, _ptr(q_rows), _ptr(n_rows),
                                      max_rows, _ptr(K), _ptr(V), _ptr(O), _ptr(lse), _stream(stream)),
            "focus_dense_attn")
+
+
+def focus_confidence(ctx, logits, dtype, row_stride, vocab, pos_base, n_pos, rows, n_rows, max_rows, conf, token,
+                     stream=None):
+    _check(ctx._lib.focus_confidence(ctx.handle, _ptr(logits), dtype, row_stride, vocab, pos_base, n_pos, _ptr(rows),
+                                     _ptr(n_rows), max_rows, _ptr(conf), _ptr(token), _stream(stream)),
+           "focus_confidence")
+
+
+def focus_update_kv(ctx, shape, K_cache, V_cache, K_new, V_new, rows, n_rows, max_rows, stream=None):
+    _check(ctx._lib.focus_update_kv(ctx.handle, C.byref(shape), _ptr(K_cache), _ptr(V_cache), _ptr(K_new), _ptr(V_new),
+                                    _ptr(rows), _ptr(n_rows), max_rows, _stream(stream)), "focus_update_kv")

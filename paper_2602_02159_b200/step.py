@@ -112,3 +112,16 @@ def sparse_layer(ctx, b: StepBuffers, Q, K, V, Kbar: Optional[torch.Tensor] = No
     fb.focus_sparse_attn(ctx, b.shape, Q, s.M, s.N, q_rows, n_rows, max_rows, K, V, b.head_reduce, b.block_idx,
                          b.max_blocks, b.block_cnt, b.sink_idx, b.sink_keep, w.n_sink, b.O if O is None else O,
                          b.lse if lse is None else lse, stream)
+
+
+def layer_schedule(n_layers: int, probe_layer: int, final_dense: int = 0):
+    """Which attention each layer of a non-block-entry step runs: 'dense' for layers 0..probe_layer (the probe layer
+    also identifies the sinks), 'sparse' after it, except that the last `final_dense` layers stay dense (the paper
+    keeps the final four layers of Dream-7B dense; 0 for UltraLLaDA)."""
+    out = []
+    for l in range(n_layers):
+        if l <= probe_layer or l >= n_layers - final_dense:
+            out.append("probe" if l == probe_layer else "dense")
+        else:
+            out.append("sparse")
+    return out

@@ -74,3 +74,14 @@ def test_product_does_not_import_the_oracle():
                 assert "focus_oracle" not in src, f"{f} names the oracle module"
     src = open(os.path.join(ROOT, "oracle", "focus_oracle.py")).read()
     assert "import paper_2602_02159_b200" not in src and "from paper_2602_02159_b200" not in src
+
+
+def test_layer_schedule_matches_the_paper():
+    """Sparse layers start after the cut-off layer; Dream keeps its final four layers dense (appendix
+    'Details of Focus-dLLM')."""
+    from paper_2602_02159_b200.step import layer_schedule
+    s = layer_schedule(32, 16)
+    assert s[:16] == ["dense"] * 16 and s[16] == "probe" and s[17:] == ["sparse"] * 15
+    d = layer_schedule(28, 5, final_dense=4)                 # paper: l_dense = 6 (1-indexed) -> probe layer 5
+    assert d[:5] == ["dense"] * 5 and d[5] == "probe" and d[6:24] == ["sparse"] * 18 and d[24:] == ["dense"] * 4
+    assert layer_schedule(4, 3, final_dense=4) == ["dense", "dense", "dense", "probe"]
