@@ -182,7 +182,17 @@ extern "C" focus_status focus_find_sinks(focus_ctx* ctx, const focus_shape* shap
     a.sh = *shape; a.scale = shape_scale(shape);
     a.Q = Q; a.q_base = q_base; a.n_q = L - q_base; a.q_rows = active_idx; a.n_rows = n_active;
     a.max_rows = max_active; a.K = K; a.V = K; a.O = nullptr; a.lse = lse_buf; a.lse_stride = max_active; a.dense = 1;
-    focus_status s = launch_attn_simt(ctx, a, stream);
+    focus_status s;
+    if (tc) {
+      // the tensor-core attention kernel yields the LSE as a by-product; its output rows (with K standing in for V)
+      // go to scratch and are dropped
+      a.O = ws.get<__nv_bfloat16>((size_t)max_active * H * shape->head_dim);
+      if (!ws.ok) return FOCUS_ERR_WORKSPACE_TOO_SMALL;
+      s = attn_tc_supported(ctx, a) ? launch_attn_tc_ws(ctx, a, ws, nullptr, stream) : FOCUS_ERR_UNSUPPORTED;
+      if (s == FOCUS_ERR_UNSUPPORTED) { a.O = nullptr; s = launch_attn_simt(ctx, a, stream); }
+    } else {
+      s = launch_attn_simt(ctx, a, stream);
+    }
     if (s != FOCUS_OK) return s;
     lse = lse_buf;
   }
