@@ -53,6 +53,7 @@ struct TcParams {
   int q_base, n_q, rows_bound, L, M, H, Hkv, hpg, B, nb, dense, group_stride, max_blocks, n_sink, ns_pad;
   int n_mtiles, n_splits, lse_stride;
   int cluster;                 // 1: the splits of a tile are one thread-block cluster and merge through shared memory
+  int pdl;                     // 1: launched as a programmatic dependent of the selection kernel (see the wait below)
   float scale_log2;            // softmax scale * log2(e)
   int32_t* status;
 #ifdef FOCUS_TIMELINE
@@ -265,30 +266,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
   TL_STAMP(0, 0);
 
-  // The prologue is a chain of global-memory latencies; everything that does not depend on another load is
-  // requested first: the row count, this group's block count, the positions of this thread's Q rows.
-  constexpr int QTHREADS = 128;                                  // the four softmax warps stage Q
-  constexpr int QIT = TM * 16 / QTHREADS;                        // 16-byte chunks of the Q tile per staging thread
-  const int qtid = (int)threadIdx.x - 64;
-  const int nrows_raw = p.q_rows ? __ldg(p.n_rows) : p.n_q;
-  const int cnt_raw = p.dense ? 0 : __ldg(p.block_cnt + g * p.group_stride);
-  int qpos[QIT];
-#pragma unroll
-  for (int it = 0; it < QIT; ++it) {
-    const int idx = qtid + it * QTHREADS;
-    const int qr = (mt * TM + (idx >> 4)) / p.hpg;
-    qpos[it] = (qtid >= 0 && qr < p.rows_bound) ? (p.q_rows ? __ldg(p.q_rows + qr) : p.q_base + qr) : -1;
-  }
-  const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
-  const int total_fr = nrows * p.hpg;                    // stacked (row, head-of-group) rows of this KV head
-  if (mt * TM >= total_fr) return;                       // uniform: nothing to compute for this tile
-
-  const TileEnum te = make_enum(p, g, cnt_raw);
-  const int t0 = (int)(((long long)te.total * split) / p.n_splits);
-  const int t1 = (int)(((long long)te.total * (split + 1)) / p.n_splits);
-  const int nt = t1 - t0;
-  const int cta_lin = blockIdx.x * p.n_splits + split;
-
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sptr = smem_raw + (sbase - smem_u32(smem_raw));
   const uint32_t sQ = sbase;
@@ -303,6 +280,84 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   int* s_last_p = reinterpret_cast<int*>(tmem_holder + 2);
   int2* tlist = reinterpret_cast<int2*>(tmem_holder + 16);      // (start | kind << 30, nvalid) per tile of this split
+
+  // The prologue is a chain of global-memory latencies; everything that does not depend on another load is
+  // requested first: the row count, this group's block count, the positions of this thread's Q rows.
+  constexpr int QTHREADS = 128;                                  // the four softmax warps stage Q
+  constexpr int QIT = TM * 16 / QTHREADS;                        // 16-byte chunks of the Q tile per staging thread
+  const int qtid = (int)threadIdx.x - 64;
+  const int nrows_raw = p.q_rows ? __ldg(p.n_rows) : p.n_q;
+  int qpos[QIT];
+#pragma unroll
+  for (int it = 0; it < QIT; ++it) {
+    const int idx = qtid + it * QTHREADS;
+    const int qr = (mt * TM + (idx >> 4)) / p.hpg;
+    qpos[it] = (qtid >= 0 && qr < p.rows_bound) ? (p.q_rows ? __ldg(p.q_rows + qr) : p.q_base + qr) : -1;
+  }
+  const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
+  const int total_fr = nrows * p.hpg;                    // stacked (row, head-of-group) rows of this KV head
+  if (mt * TM >= total_fr) return;                       // uniform: nothing to compute for this tile
+
+  // query rows of this thread (softmax warps only): requested now, stored to shared memory further down
+  uint4 qv[QIT];
+#pragma unroll
+  for (int it = 0; it < QIT; ++it) {
+    qv[it] = make_uint4(0, 0, 0, 0);
+    if (qtid >= 0) {
+      const int idx = qtid + it * QTHREADS;
+      const int r = idx >> 4, c = idx & 15;
+      const int fr = mt * TM + r;
+      if (fr < total_fr) {
+        const int pos = qpos[it];
+        if (pos >= p.q_base && pos < p.q_base + p.n_q) {
+          const __nv_bfloat16* src = p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
+                                     (long long)(g * p.hpg + fr % p.hpg) * p.q_stride_head + c * 8;
+          qv[it] = __ldg(reinterpret_cast<const uint4*>(src));
+        } else if (c == 0) {
+          set_status(p.status, FOCUS_ERR_INVALID_ARG);
+        }
+      }
+    }
+  }
+  // Launched as a programmatic dependent of the selection kernel of the same sparse layer: everything above
+  // (row list, query rows) does not come from that kernel and overlaps with it; the block lists, the gathered
+  // sink rows and their mask do, so nothing below may start before it has completed.
+  auto arm_barriers = [&]() {                        // warp 0, lane 0
+    for (int sl = 0; sl < NSLOT; ++sl) { mbar_init(bar_full(sl), 1); mbar_init(bar_empty(sl), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pready(b), 128); }
+    mbar_init(bar_pvdone, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  };
+  auto alloc_tmem = [&]() {                          // warp 1, all lanes
+    tmem_alloc(smem_u32(tmem_holder), 512);
+    tmem_relinquish();
+  };
+  auto store_q = [&]() {                             // softmax warps
+#pragma unroll
+    for (int it = 0; it < QIT; ++it) {
+      const int idx = qtid + it * QTHREADS;
+      const int r = idx >> 4, c = idx & 15;
+      const int half = c >> 3, cc = c & 7;
+      *reinterpret_cast<uint4*>(sptr + half * HALF_BYTES + r * 128 + ((cc ^ (r & 7)) << 4)) = qv[it];
+    }
+  };
+  if (p.pdl) {
+    // as a programmatic dependent the whole private set-up runs while the selection kernel is still at work
+    if (warp == 0 && lane == 0) arm_barriers();
+    if (warp == 1) alloc_tmem();
+    if (qtid >= 0) store_q();
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+  }
+  const int cnt_raw = p.dense ? 0 : __ldg(p.block_cnt + g * p.group_stride);
+
+  const TileEnum te = make_enum(p, g, cnt_raw);
+  const int t0 = (int)(((long long)te.total * split) / p.n_splits);
+  const int t1 = (int)(((long long)te.total * (split + 1)) / p.n_splits);
+  const int nt = t1 - t0;
+  const int cta_lin = blockIdx.x * p.n_splits + split;
+
   const bool use_list = !p.dense && nt <= MAXT;
   // tile descriptor: from the staged list (sparse) or by arithmetic (dense; splits longer than the list)
   auto get_tile = [&](int idx) -> TileInfo {
@@ -314,6 +369,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     return tile_info(p, te, t0 + idx);
   };
 
+  if (nt <= 0 && p.pdl) {                                 // TMEM was allocated before the split turned out empty
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) {
+      __syncwarp();
+      tmem_dealloc(*tmem_holder, 512);
+    }
+  }
   if (nt <= 0 && p.cluster) {                             // empty split inside a cluster: neutral partial, then merge duty
     float* ps = reinterpret_cast<float*>(sptr + Q_BYTES);
     for (int r = threadIdx.x; r < TM; r += NTHREADS) { ps[TM * PROW + 2 * r] = -INFINITY; ps[TM * PROW + 2 * r + 1] = 0.f; }
@@ -358,14 +422,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   const int n_loads = 2 * nt;
   const int n_early = n_loads < NSLOT ? n_loads : NSLOT;
   if (warp == 0) {
-    if (lane == 0) {
-      for (int s = 0; s < NSLOT; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
-      for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pready(b), 128); }
-      mbar_init(bar_pvdone, 1);
-      *abort_flag = 0;
-      fence_barrier_init();
-      fence_proxy_async();
-    }
+    if (lane == 0 && !p.pdl) arm_barriers();
     if (use_list) {
       for (int t = lane; t < nt; t += 32) {
         const TileInfo ti = tile_info(p, te, t0 + t);
@@ -382,40 +439,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     __syncwarp();
     TL_STAMP(6, 0);
   }
-  if (warp == 1) {
-    tmem_alloc(smem_u32(tmem_holder), 512);
-    tmem_relinquish();
-    TL_STAMP(7, 32);
-  }
+  if (warp == 1 && !p.pdl) alloc_tmem();
   // Q tile -> shared memory in the 128-byte-swizzled K-major layout the MMA descriptor expects:
   // half h (columns 64h..64h+63) at h*16 KB, row r at r*128 bytes, 16-byte chunk c at ((c ^ (r & 7)) * 16).
-  if (qtid >= 0) {
-    uint4 qv[QIT];
-#pragma unroll
-    for (int it = 0; it < QIT; ++it) {
-      const int idx = qtid + it * QTHREADS;
-      const int r = idx >> 4, c = idx & 15;
-      const int fr = mt * TM + r;
-      qv[it] = make_uint4(0, 0, 0, 0);
-      if (fr < total_fr) {
-        const int pos = qpos[it];
-        if (pos >= p.q_base && pos < p.q_base + p.n_q) {
-          const __nv_bfloat16* src = p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
-                                     (long long)(g * p.hpg + fr % p.hpg) * p.q_stride_head + c * 8;
-          qv[it] = __ldg(reinterpret_cast<const uint4*>(src));
-        } else if (c == 0) {
-          set_status(p.status, FOCUS_ERR_INVALID_ARG);
-        }
-      }
-    }
-#pragma unroll
-    for (int it = 0; it < QIT; ++it) {
-      const int idx = qtid + it * QTHREADS;
-      const int r = idx >> 4, c = idx & 15;
-      const int half = c >> 3, cc = c & 7;
-      *reinterpret_cast<uint4*>(sptr + half * HALF_BYTES + r * 128 + ((cc ^ (r & 7)) << 4)) = qv[it];
-    }
-  }
+  if (qtid >= 0 && !p.pdl) store_q();
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();
@@ -1129,15 +1156,24 @@ static int cluster_capacity(K kernel, int n, int threads, int smem) {
 }
 
 template <typename K>
-static focus_status launch_clustered(K kernel, dim3 grid, int threads, int smem, int cluster_y, cudaStream_t st,
-                                     const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c,
-                                     const CUtensorMap& d, const TcParams& p) {
+static focus_status launch_ex(K kernel, dim3 grid, int threads, int smem, int cluster_y, bool pdl, cudaStream_t st,
+                              const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& c, const CUtensorMap& d,
+                              const TcParams& p) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid; cfg.blockDim = dim3(threads, 1, 1); cfg.dynamicSmemBytes = smem; cfg.stream = st;
-  cudaLaunchAttribute at[1];
-  at[0].id = cudaLaunchAttributeClusterDimension;
-  at[0].val.clusterDim.x = 1; at[0].val.clusterDim.y = cluster_y; at[0].val.clusterDim.z = 1;
-  cfg.attrs = at; cfg.numAttrs = 1;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  if (cluster_y > 1) {
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = 1; at[na].val.clusterDim.y = cluster_y; at[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  if (pdl) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = at; cfg.numAttrs = na;
   if (cudaLaunchKernelEx(&cfg, kernel, a, b, c, d, p) != cudaSuccess) {
     cudaGetLastError();
     return FOCUS_ERR_CUDA;
@@ -1262,6 +1298,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.q_rows = a.q_rows; p.n_rows = a.n_rows; p.block_idx = a.block_idx; p.block_cnt = a.block_cnt;
   p.sink_mask = mask; p.part_O = part_O; p.part_ml = part_ml;
   p.cluster = use_cluster ? 1 : 0;
+  p.pdl = (pre != nullptr && !wide && !ctx->no_pdl) ? 1 : 0;   // pre-gathered sinks: called right after the selection kernel
   p.counters = (n_splits > 1 && !use_cluster && !wide && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
                    ? ctx->d_counters : nullptr;
   p.q_stride_row = sh.q_stride_row; p.q_stride_head = sh.q_stride_head;
@@ -1277,19 +1314,13 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
 
   ctx->last_attn_variant = wide ? 3 : 2;
   if (wide) {
-    if (n_splits > 1) {
-      focus_status ls = launch_clustered(attn_tc_wide_kernel, dim3(base, n_splits, 1), NTHREADS_W, SMEM_BYTES_W, n_splits, st,
-                                         tmK, tmV, tmSK, tmSV, p);
-      if (ls != FOCUS_OK) return ls;
-    } else {
-      attn_tc_wide_kernel<<<dim3(base, 1), NTHREADS_W, SMEM_BYTES_W, st>>>(tmK, tmV, tmSK, tmSV, p);
-    }
-  } else if (use_cluster) {
-    focus_status ls = launch_clustered(attn_tc_kernel, dim3(base, n_splits, 1), NTHREADS, SMEM_BYTES, n_splits, st, tmK, tmV,
-                                       tmSK, tmSV, p);
+    focus_status ls = launch_ex(attn_tc_wide_kernel, dim3(base, n_splits, 1), NTHREADS_W, SMEM_BYTES_W, n_splits, false, st,
+                                tmK, tmV, tmSK, tmSV, p);
     if (ls != FOCUS_OK) return ls;
   } else {
-    attn_tc_kernel<<<dim3(base, n_splits), NTHREADS, SMEM_BYTES, st>>>(tmK, tmV, tmSK, tmSV, p);
+    focus_status ls = launch_ex(attn_tc_kernel, dim3(base, n_splits, 1), NTHREADS, SMEM_BYTES, use_cluster ? n_splits : 1,
+                                p.pdl != 0, st, tmK, tmV, tmSK, tmSV, p);
+    if (ls != FOCUS_OK) return ls;
   }
   FOCUS_CHECK_LAUNCH();
   if (n_splits > 1 && !p.counters && !use_cluster && !wide) {

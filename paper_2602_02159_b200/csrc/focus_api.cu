@@ -48,6 +48,7 @@ extern "C" focus_status focus_create(focus_ctx** out, int device, size_t workspa
   c->force_simt = 0;
   c->last_attn_variant = 0;
   c->no_wide = getenv("FOCUS_NO_WIDE") != nullptr;
+  c->no_pdl = getenv("FOCUS_NO_PDL") != nullptr;
   c->encode_tiled = nullptr;
   if (prop.major == 10) {   // tensor-core kernels are built for sm_100a only
     cudaDriverEntryPointQueryResult q;

@@ -16,6 +16,7 @@ struct focus_ctx {
   int32_t* d_counters; // FOCUS_N_COUNTERS arrival counters for split merges; zero between launches
   int force_simt;
   int last_attn_variant;   // 0 none yet, 1 SIMT, 2 tensor-core 128-row tiles, 3 tensor-core 256-row tiles
+  int no_pdl;          // 1: never launch the attention kernel as a programmatic dependent (A/B comparisons)
   int no_wide;         // 1: never use the two-query-tile attention kernel (A/B comparisons)
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime (no libcuda link)
 };

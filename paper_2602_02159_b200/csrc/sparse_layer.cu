@@ -18,6 +18,9 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
                     int32_t* __restrict__ block_cnt, uint8_t* __restrict__ sink_keep, __nv_bfloat16* __restrict__ gK,
                     __nv_bfloat16* __restrict__ gV, uint8_t* __restrict__ mask, int32_t* status) {
   const int tid = threadIdx.x;
+  // the attention kernel of this layer is launched as a programmatic dependent: let its CTAs start their own
+  // set-up now; it waits for this grid to complete before it reads anything written here
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if ((int)blockIdx.x >= Hkv) {
     // ---- gather: 64 sink rows of one KV head per CTA, one 16-byte chunk of K and of V per thread ---------
     const int gi = (int)blockIdx.x - Hkv;
