@@ -46,6 +46,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         flags += ["-Xptxas", "-v"]
     if os.environ.get("FOCUS_TIMELINE"):          # development: per-CTA timestamps in the attention kernel
         flags += ["-DFOCUS_TIMELINE"]
+    flags += os.environ.get("FOCUS_EXTRA_NVCC_FLAGS", "").split()     # development: experiment switches
 
     def compile_one(src):
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")

@@ -63,8 +63,12 @@ struct TcParams {
 
 #ifdef FOCUS_TIMELINE
 #define TL_STAMP(slot, tid) do { if (p.dbg && threadIdx.x == (tid)) p.dbg[(blockIdx.x * gridDim.y + blockIdx.y) * 8 + (slot)] = global_ns(); } while (0)
+// per-iteration trace of CTA (0,0): who 0 = MMA thread, 1 = first softmax thread of tile A, 2 = of tile B
+__device__ __forceinline__ unsigned long long tl_clock() { unsigned long long c; asm volatile("mov.u64 %0, %%clock64;" : "=l"(c) :: "memory"); return c; }
+#define TL_ITER(who, tid, it, ev) do { if (p.dbg && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == (tid) && (it) < 64) p.dbg[65536 + (who) * 512 + (it) * 8 + (ev)] = tl_clock(); } while (0)
 #else
 #define TL_STAMP(slot, tid) do { } while (0)
+#define TL_ITER(who, tid, it, ev) do { } while (0)
 #endif
 
 struct TileInfo {
@@ -183,6 +187,16 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t saddr, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
   return r;
 }
+__device__ __forceinline__ float4 ld_smem_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float2 ld_smem_f2(uint32_t addr) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+  return v;
+}
 __device__ __forceinline__ float4 ld_dsmem_f4(uint32_t addr) {
   float4 v;
   asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
@@ -194,51 +208,98 @@ __device__ __forceinline__ float2 ld_dsmem_f2(uint32_t addr) {
   return v;
 }
 
-template <int ROWS, int NTH>
-__device__ __forceinline__ void cluster_merge(const TcParams& p, int g, int mt, int total_fr, int rank, uint32_t spart) {
+// In-cluster merge for split counts up to SMAX.  One work item = one row x the 4-column groups c8, c8 + 8, c8 + 16,
+// c8 + 24 (c8 = 0..7): the per-row work (weights, normaliser, addressing) is paid once per 16 output columns, and a
+// quarter-warp reads 128 contiguous bytes of a partial.  The CTA's own partial is read with plain shared-memory
+// loads, the others through the cluster window.
+template <int ROWS, int NTH, int SMAX>
+__device__ __forceinline__ void cluster_merge_items(const TcParams& p, int g, int mt, int rank, uint32_t spart, int mine, int tid) {
   constexpr int PART_ML_OFF = ROWS * PROW;                     // float offset of the (max, sum) pairs
-  __syncthreads();
-  cluster_sync_all();
-  const int rows = min(ROWS, total_fr - mt * ROWS);
-  const int S = p.n_splits;                                   // <= 8 in cluster mode
-  const int mine = rank < rows ? (rows - rank + S - 1) / S : 0;
-  for (int item = threadIdx.x; item < mine * 32; item += NTH) {
-    const int row = rank + (item >> 5) * S, cg = item & 31;
-    float2 ml[8];
-    float4 o[8];
+  constexpr int KB = SMAX <= 4 ? 4 : 2;                        // column groups in flight per batch (register budget)
+  const int S = p.n_splits;
+  const int n_items = mine * 8;
+  for (int item = tid; item < n_items; item += NTH) {
+    const int row = rank + (item >> 3) * S, c8 = item & 7;
+    float2 ml[SMAX];
 #pragma unroll
-    for (int s = 0; s < 8; ++s) {
+    for (int s = 0; s < SMAX; ++s) {
+      ml[s] = make_float2(0.f, 0.f);
       if (s < S) {
-        const uint32_t base = map_to_rank(spart, (uint32_t)s);
-        ml[s] = ld_dsmem_f2(base + (uint32_t)(PART_ML_OFF + row * 2) * 4u);
-        o[s] = ld_dsmem_f4(base + (uint32_t)(row * PROW + cg * 4) * 4u);
+        const uint32_t off = (uint32_t)(PART_ML_OFF + row * 2) * 4u;
+#ifdef MERGE_LOCAL_ONLY
+        ml[s] = ld_smem_f2(spart + off);
+#else
+        ml[s] = s == rank ? ld_smem_f2(spart + off) : ld_dsmem_f2(map_to_rank(spart, (uint32_t)s) + off);
+#endif
       }
     }
     float m = -INFINITY;
 #pragma unroll
-    for (int s = 0; s < 8; ++s)
-      if (s < S && ml[s].y > 0.f) m = fmaxf(m, ml[s].x);
+    for (int s = 0; s < SMAX; ++s)
+      if (ml[s].y > 0.f) m = fmaxf(m, ml[s].x);
+    float wgt[SMAX];
     float tot = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-    for (int s = 0; s < 8; ++s) {
-      if (s < S && ml[s].y > 0.f) {
-        const float wgt = exp2f(ml[s].x - m);
-        tot += wgt * ml[s].y;
-        acc.x += wgt * o[s].x; acc.y += wgt * o[s].y; acc.z += wgt * o[s].z; acc.w += wgt * o[s].w;
-      }
+    for (int s = 0; s < SMAX; ++s) {
+      wgt[s] = ml[s].y > 0.f ? exp2f(ml[s].x - m) : 0.f;
+      tot += wgt[s] * ml[s].y;
     }
     const float inv = tot > 0.f ? 1.f / tot : 0.f;
+#pragma unroll
+    for (int s = 0; s < SMAX; ++s) wgt[s] *= inv;
     const int fr = mt * ROWS + row;
     const int qr = fr / p.hpg, hh = fr % p.hpg;
-    __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD + cg * 4;
-    uint2 v;
-    v.x = pack_bf16(acc.x * inv, acc.y * inv);
-    v.y = pack_bf16(acc.z * inv, acc.w * inv);
-    *reinterpret_cast<uint2*>(orow) = v;
-    if (p.lse && cg == 0)
+    __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD;
+#pragma unroll
+    for (int k0 = 0; k0 < 4; k0 += KB) {
+      float4 o[KB][SMAX];
+#pragma unroll
+      for (int k = 0; k < KB; ++k)
+#pragma unroll
+        for (int s = 0; s < SMAX; ++s)
+          if (s < S) {
+            const uint32_t off = (uint32_t)(row * PROW + (c8 + 8 * (k0 + k)) * 4) * 4u;
+#ifdef MERGE_LOCAL_ONLY
+            o[k][s] = ld_smem_f4(spart + off);
+#else
+            o[k][s] = s == rank ? ld_smem_f4(spart + off) : ld_dsmem_f4(map_to_rank(spart, (uint32_t)s) + off);
+#endif
+          }
+#pragma unroll
+      for (int k = 0; k < KB; ++k) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int s = 0; s < SMAX; ++s)
+          if (s < S && wgt[s] > 0.f) {                           // an empty partial's accumulator is never read
+            acc.x += wgt[s] * o[k][s].x; acc.y += wgt[s] * o[k][s].y;
+            acc.z += wgt[s] * o[k][s].z; acc.w += wgt[s] * o[k][s].w;
+          }
+        uint2 v;
+        v.x = pack_bf16(acc.x, acc.y);
+        v.y = pack_bf16(acc.z, acc.w);
+        *reinterpret_cast<uint2*>(orow + (c8 + 8 * (k0 + k)) * 4) = v;
+      }
+    }
+    if (p.lse && c8 == 0)
       p.lse[(size_t)(g * p.hpg + hh) * p.lse_stride + qr] = (m + log2f(tot)) * 0.6931471805599453f;
   }
+}
+
+// All threads of all CTAs of the cluster call this; the threads with 0 <= tid < NTH share the merge work.
+template <int ROWS, int NTH>
+__device__ __forceinline__ void cluster_merge(const TcParams& p, int g, int mt, int total_fr, int rank, uint32_t spart, int tid) {
+  asm volatile("bar.sync 0;" ::: "memory");
+  cluster_sync_all();
+  const int rows = min(ROWS, total_fr - mt * ROWS);
+  const int S = p.n_splits;                                   // <= 8 in cluster mode
+  const int mine = rank < rows ? (rows - rank + S - 1) / S : 0;
+  TL_STAMP(5, 0);
+  if (tid >= 0) {
+    if (S <= 2) cluster_merge_items<ROWS, NTH, 2>(p, g, mt, rank, spart, mine, tid);
+    else if (S <= 4) cluster_merge_items<ROWS, NTH, 4>(p, g, mt, rank, spart, mine, tid);
+    else cluster_merge_items<ROWS, NTH, 8>(p, g, mt, rank, spart, mine, tid);
+  }
+  TL_STAMP(6, 128);
   cluster_sync_all();                                          // nobody leaves while its partial may still be read
 }
 
@@ -381,7 +442,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   if (nt <= 0 && p.cluster) {                             // empty split inside a cluster: neutral partial, then merge duty
     float* ps = reinterpret_cast<float*>(sptr + Q_BYTES);
     for (int r = threadIdx.x; r < TM; r += NTHREADS) { ps[TM * PROW + 2 * r] = -INFINITY; ps[TM * PROW + 2 * r + 1] = 0.f; }
-    cluster_merge<TM, NTHREADS>(p, g, mt, total_fr, split, sSlot);
+    cluster_merge<TM, NTHREADS>(p, g, mt, total_fr, split, sSlot, (int)threadIdx.x);
     return;
   }
   if (nt <= 0) {                                          // empty split: publish a neutral partial
@@ -687,7 +748,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     tmem_dealloc(tmem, 512);
   }
   TL_STAMP(3, 0);
-  if (p.cluster) cluster_merge<TM, NTHREADS>(p, g, mt, total_fr, split, sSlot);
+  if (p.cluster) cluster_merge<TM, NTHREADS>(p, g, mt, total_fr, split, sSlot, (int)threadIdx.x);
   else if (p.n_splits > 1 && p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p, reinterpret_cast<float*>(sptr + Q_BYTES));
   TL_STAMP(4, 0);
 }
@@ -698,14 +759,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 // exponentials rather than by HBM.  Every K/V tile is staged once and serves 256 rows; the two tiles take turns
 // on the tensor core: while the softmax warps of A work on S_A(j), the tensor pipe runs S_B(j) = Q_B K_j^T and
 // O_B += P_B(j-1) V_(j-1), and vice versa.  TMEM: S_A | S_B | O_A | O_B (4 x 128 columns), P aliases S.
-// Warps (320 threads): 0 TMA producer, 1 MMA issuer + TMEM owner, 2..5 softmax of tile A, 6..9 softmax of tile B.
+// Warps (384 threads): 0 TMA producer, 1 MMA issuer + TMEM owner, 2..3 idle, 4..7 softmax of tile A, 8..11 softmax of
+// tile B.  After set-up the first warpgroup hands most of its registers to the softmax warpgroups (setmaxnreg), which
+// keep a whole 128-column score row per thread in registers.
 // ================================================================================================================
 constexpr int TMW = 256;
 constexpr int NSLOT_W = 5;
 constexpr int Q_BYTES_W = TMW * HD * 2;
-constexpr int NBAR_W = 2 * NSLOT_W + 7;
+constexpr int NBAR_W = 2 * NSLOT_W + 9;
 constexpr int MAXT_W = 96;
-constexpr int NTHREADS_W = 320;
+constexpr int NTHREADS_W = 384;                 // three warpgroups: {producer, MMA, two idle warps}, softmax A, softmax B
 constexpr int SMEM_BYTES_W = 1024 + Q_BYTES_W + NSLOT_W * SLOT_BYTES + NBAR_W * 8 + 64 + MAXT_W * 8;
 
 __global__ void __launch_bounds__(NTHREADS_W, 1)
@@ -713,11 +776,12 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     const __grid_constant__ CUtensorMap tmSK, const __grid_constant__ CUtensorMap tmSV, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  TL_STAMP(0, 0);
   const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
 
   constexpr int QTHREADS = 256;                                  // the eight softmax warps stage Q
   constexpr int QIT = TMW * 16 / QTHREADS;
-  const int qtid = (int)threadIdx.x - 64;
+  const int qtid = (int)threadIdx.x - 128;
   const int nrows_raw = p.q_rows ? __ldg(p.n_rows) : p.n_q;
   const int cnt_raw = p.dense ? 0 : __ldg(p.block_cnt + g * p.group_stride);
   int qpos[QIT];
@@ -744,7 +808,8 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   auto bar_full = [&](int s) { return sBar + 8u * s; };
   auto bar_empty = [&](int s) { return sBar + 8u * (NSLOT_W + s); };
   auto bar_sfull = [&](int x) { return sBar + 8u * (2 * NSLOT_W + x); };
-  auto bar_pready = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 2 + x); };
+  auto bar_pready = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 2 + x); };    // P_x columns of keys 0..63 stored
+  auto bar_pready2 = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 7 + x); };   // ... of keys 64..127
   auto bar_pvdone = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 4 + x); };
   const uint32_t bar_alldone = sBar + 8u * (2 * NSLOT_W + 6);   // every MMA of this CTA has completed
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(sptr + Q_BYTES_W + NSLOT_W * SLOT_BYTES + NBAR_W * 8);
@@ -763,7 +828,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 
   if (nt <= 0) {                                                 // empty split (cluster mode only: see the launcher)
     for (int r = threadIdx.x; r < TMW; r += NTHREADS_W) { ps[TMW * PROW + 2 * r] = -INFINITY; ps[TMW * PROW + 2 * r + 1] = 0.f; }
-    cluster_merge<TMW, NTHREADS_W>(p, g, mt, total_fr, split, sSlot);
+    cluster_merge<TMW, 256>(p, g, mt, total_fr, split, sSlot, (int)threadIdx.x - 128);
     return;
   }
 
@@ -783,7 +848,9 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   if (warp == 0) {
     if (lane == 0) {
       for (int s = 0; s < NSLOT_W; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
-      for (int x = 0; x < 2; ++x) { mbar_init(bar_sfull(x), 1); mbar_init(bar_pready(x), 128); mbar_init(bar_pvdone(x), 1); }
+      for (int x = 0; x < 2; ++x) {
+        mbar_init(bar_sfull(x), 1); mbar_init(bar_pready(x), 128); mbar_init(bar_pready2(x), 128); mbar_init(bar_pvdone(x), 1);
+      }
       mbar_init(bar_alldone, 1);
       *abort_flag = 0;
       fence_barrier_init();
@@ -840,7 +907,9 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_holder;
-
+  TL_STAMP(1, 0);
+  if (warp < 4) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
   if (warp == 0) {
     if (lane == 0) {
       int issued = n_early;
@@ -877,13 +946,22 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           }
         tc_commit(bar_sfull(x));
       };
-      auto do_pv = [&](int x, int j) {                              // O_x += P_x(j) V_j
+      // O_x += P_x(j) V_j in two halves of 64 keys: the first starts while the softmax warps still work on the second
+      auto do_pv = [&](int x, int j, uint32_t par) -> bool {
         const uint64_t vdesc = make_sdesc(sSlot + ((2 * j + 1) % NSLOT_W) * SLOT_BYTES, HALF_BYTES, 1024);
+        if (!mbar_wait(bar_pready(x), par, abort_flag, p.status)) return false;
+        tc_fence_after();
 #pragma unroll
-        for (int ks = 0; ks < TN / 16; ++ks)
+        for (int ks = 0; ks < TN / 32; ++ks)
           mma_ts(tmem + 256 + x * 128, tmem + x * 128 + ks * 8, vdesc + (uint64_t)(ks * (2048 >> 4)), IDESC_PV,
                  (j > 0 || ks > 0) ? 1u : 0u);
+        if (!mbar_wait(bar_pready2(x), par, abort_flag, p.status)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = TN / 32; ks < TN / 16; ++ks)
+          mma_ts(tmem + 256 + x * 128, tmem + x * 128 + ks * 8, vdesc + (uint64_t)(ks * (2048 >> 4)), IDESC_PV, 1u);
         tc_commit(bar_pvdone(x));
+        return true;
       };
       ok = wait_load(0);
       if (ok) {
@@ -895,27 +973,42 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       for (int j = 0; j < nt && ok; ++j) {
         const uint32_t par = (uint32_t)j & 1u;
         if (!wait_load(2 * j + 1)) { ok = false; break; }            // V_j
-        if (!mbar_wait(bar_pready(0), par, abort_flag, p.status)) { ok = false; break; }
-        tc_fence_after();
-        do_pv(0, j);
+        TL_ITER(0, 32, j, 0);
+        if (!do_pv(0, j, par)) { ok = false; break; }
+        TL_ITER(0, 32, j, 4);
         if (j + 1 < nt) {
           if (!wait_load(2 * j + 2)) { ok = false; break; }          // K_(j+1)
           tc_fence_after();
           do_qk(0, j + 1);
         }
-        if (!mbar_wait(bar_pready(1), par, abort_flag, p.status)) { ok = false; break; }
-        tc_fence_after();
-        do_pv(1, j);
+        TL_ITER(0, 32, j, 5);
+        TL_ITER(0, 32, j, 2);
+        if (!do_pv(1, j, par)) { ok = false; break; }
         tc_commit(bar_empty((2 * j + 1) % NSLOT_W));                 // V_j
+        TL_ITER(0, 32, j, 6);
         if (j + 1 < nt) {
           do_qk(1, j + 1);
           tc_commit(bar_empty((2 * j + 2) % NSLOT_W));               // K_(j+1)
         }
+        TL_ITER(0, 32, j, 7);
       }
       tc_commit(bar_alldone);
     }
+  }
+    // tail of the first warpgroup, inside its own register-budget region: release TMEM, take part in the barriers of
+    // the merge (registers given away above are not asked back: a late setmaxnreg.inc never returned on this part)
+    tc_fence_before();
+    asm volatile("bar.sync 0;" ::: "memory");
+    if (warp == 1) {
+      __syncwarp();
+      tmem_dealloc(tmem, 512);
+    }
+    TL_STAMP(3, 0);
+    if (p.n_splits > 1) cluster_merge<TMW, 256>(p, g, mt, total_fr, split, sSlot, -1);
+    TL_STAMP(4, 0);
   } else {
-    const int x = (warp - 2) >> 2;                                   // query tile of this softmax warp
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+    const int x = (warp - 4) >> 2;                                   // query tile of this softmax warp
     const int rq = warp & 3;
     const int row = rq * 32 + lane;                                  // row inside the 128-row tile
     const uint32_t lane_off = (uint32_t)(rq * 32) << 16;
@@ -924,7 +1017,9 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
     for (int idx = 0; idx < nt; ++idx) {
+      TL_ITER(warp - 3, warp * 32, idx, 0);
       if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(x), (uint32_t)idx & 1u, abort_flag, p.status))) { ok = false; break; }
+      TL_ITER(warp - 3, warp * 32, idx, 1);
       tc_fence_after();
       uint32_t sreg[128];
       TC_LD32(ts, (sreg + 0));
@@ -932,14 +1027,17 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       TC_LD32(ts + 64, (sreg + 64));
       TC_LD32(ts + 96, (sreg + 96));
       tc_wait_ld();
+      TL_ITER(warp - 3, warp * 32, idx, 2);
       const TileInfo ti = get_tile(idx);
       float tmax = -INFINITY;
       if (ti.kind == 0 && ti.nvalid == TN) {
         float t4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains instead of one of 128
 #pragma unroll
-        for (int c = 0; c < 128; c += 4) {
-          t4[0] = fmaxf(t4[0], __uint_as_float(sreg[c]));     t4[1] = fmaxf(t4[1], __uint_as_float(sreg[c + 1]));
-          t4[2] = fmaxf(t4[2], __uint_as_float(sreg[c + 2])); t4[3] = fmaxf(t4[3], __uint_as_float(sreg[c + 3]));
+        for (int c = 0; c < 128; c += 8) {
+          t4[0] = fmax3(t4[0], __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]));
+          t4[1] = fmax3(t4[1], __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
+          t4[2] = fmax3(t4[2], __uint_as_float(sreg[c + 4]), __uint_as_float(sreg[c + 5]));
+          t4[3] = fmax3(t4[3], __uint_as_float(sreg[c + 6]), __uint_as_float(sreg[c + 7]));
         }
         tmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
       } else if (ti.kind == 0) {
@@ -974,38 +1072,48 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         m_ref = tmax;
       }
       const float mneg = m_ref == -INFINITY ? 0.f : -m_ref;
-      uint32_t preg[64];
-      float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+      // sfull(idx) implies that every earlier product of this tile, P V of key tile idx-1 included, has completed
+      if (idx > 0 && __any_sync(0xffffffffu, rescale)) {
 #pragma unroll
-      for (int c = 0; c < 64; ++c) {
-        const float p0 = ex2(fmaf(__uint_as_float(sreg[2 * c]), p.scale_log2, mneg));
-        const float p1 = ex2(fmaf(__uint_as_float(sreg[2 * c + 1]), p.scale_log2, mneg));
-        ls4[c & 3] += p0 + p1;
-        preg[c] = pack_bf16(p0, p1);
-      }
-      l = l * alpha + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
-      if (idx > 0) {
-        if (!__all_sync(0xffffffffu, mbar_wait(bar_pvdone(x), (uint32_t)(idx - 1) & 1u, abort_flag, p.status))) { ok = false; break; }
-        if (__any_sync(0xffffffffu, rescale)) {
-          tc_fence_after();
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t oreg[32];
+          TC_LD32(to + cb * 32, oreg);
+          tc_wait_ld();
 #pragma unroll
-          for (int cb = 0; cb < 4; ++cb) {
-            uint32_t oreg[32];
-            TC_LD32(to + cb * 32, oreg);
-            tc_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * alpha);
-            TC_ST32(to + cb * 32, oreg);
-          }
+          for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * alpha);
+          TC_ST32(to + cb * 32, oreg);
         }
       }
-      TC_ST32(ts, (preg + 0));
-      TC_ST32(ts + 32, (preg + 32));
+      TL_ITER(warp - 3, warp * 32, idx, 3);
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) {                               // 32 keys at a time: exponentials, bf16 P, row sum
+        uint32_t preg[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int c = ch * 32 + 2 * i;
+          float x0, x1;
+          ffma2(x0, x1, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]), p.scale_log2, p.scale_log2, mneg, mneg);
+          const float p0 = ex2(x0), p1 = ex2(x1);
+          preg[i] = pack_bf16(p0, p1);
+          fadd2(acc[(i & 1) * 2], acc[(i & 1) * 2 + 1], acc[(i & 1) * 2], acc[(i & 1) * 2 + 1], p0, p1);
+        }
+        TC_ST16(ts + ch * 16, preg);
+        if (ch == 1) {
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar_pready(x));
+          TL_ITER(warp - 3, warp * 32, idx, 4);
+        }
+      }
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_pready(x));
+      mbar_arrive(bar_pready2(x));
+      l = l * alpha + ((acc[0] + acc[1]) + (acc[2] + acc[3]));
+      TL_ITER(warp - 3, warp * 32, idx, 5);
     }
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_pvdone(x), (uint32_t)(nt - 1) & 1u, abort_flag, p.status));
+    TL_STAMP(2, 128);
     if (ok) {
       tc_fence_after();
       const int trow = x * 128 + row;                                // row inside the 256-row CTA tile
@@ -1053,14 +1161,11 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         if (valid) { ps[TMW * PROW + 2 * trow] = m_ref; ps[TMW * PROW + 2 * trow + 1] = l; }
       }
     }
+    // tail of the softmax warpgroups (kept inside their register-budget region): they do the split merge
+    tc_fence_before();
+    asm volatile("bar.sync 0;" ::: "memory");
+    if (p.n_splits > 1) cluster_merge<TMW, 256>(p, g, mt, total_fr, split, sSlot, (int)threadIdx.x - 128);
   }
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 1) {
-    __syncwarp();
-    tmem_dealloc(tmem, 512);
-  }
-  if (p.n_splits > 1) cluster_merge<TMW, NTHREADS_W>(p, g, mt, total_fr, split, sSlot);
 }
 
 // Stand-alone merge (used when there are more query tiles than arrival counters): out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s, one warp per stacked row.
@@ -1238,7 +1343,8 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     }
     // it pays on long key streams (measured: +6 % on dense 32K); with a few dozen tiles per CTA the one-tile kernel
     // without a key split is faster
-    if (max_tiles / n_splits < 32) wide = false;
+    static const int wide_min = getenv("FOCUS_WIDE_MIN") ? atoi(getenv("FOCUS_WIDE_MIN")) : 32;
+    if (max_tiles / n_splits < wide_min) wide = false;
   }
   if (!wide) {
     n_mtiles = (int)((stacked + TM - 1) / TM);
