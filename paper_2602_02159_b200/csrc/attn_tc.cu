@@ -31,7 +31,7 @@ constexpr int NSLOT = 6;           // K/V ring slots
 constexpr int SLOT_BYTES = TN * HD * 2;
 constexpr int HALF_BYTES = SLOT_BYTES / 2;     // one 64-wide half of a tile: 128 rows x 128 bytes
 constexpr int Q_BYTES = TM * HD * 2;
-constexpr int NBAR = 2 * NSLOT + 5;
+constexpr int NBAR = 2 * NSLOT + 7;
 constexpr int MAXT = 128;            // key tiles of a split whose descriptors are staged in shared memory
 constexpr int SMEM_BYTES = 1024 + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8 + 64 + MAXT * 8;
 constexpr int NTHREADS = 192;
@@ -337,6 +337,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   auto bar_sfull = [&](int b) { return sBar + 8u * (2 * NSLOT + b); };
   auto bar_pready = [&](int b) { return sBar + 8u * (2 * NSLOT + 2 + b); };
   const uint32_t bar_pvdone = sBar + 8u * (2 * NSLOT + 4);
+  auto bar_pready2 = [&](int b) { return sBar + 8u * (2 * NSLOT + 5 + b); };   // second half (keys 64..127) of P_b stored
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(sptr + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   int* s_last_p = reinterpret_cast<int*>(tmem_holder + 2);
@@ -385,7 +386,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   // sink rows and their mask do, so nothing below may start before it has completed.
   auto arm_barriers = [&]() {                        // warp 0, lane 0
     for (int sl = 0; sl < NSLOT; ++sl) { mbar_init(bar_full(sl), 1); mbar_init(bar_empty(sl), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pready(b), 128); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pready(b), 128); mbar_init(bar_pready2(b), 128); }
     mbar_init(bar_pvdone, 1);
     *abort_flag = 0;
     fence_barrier_init();
@@ -550,8 +551,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         const uint64_t vdesc = make_sdesc(sSlot + slot * SLOT_BYTES, HALF_BYTES, 1024);
         const uint32_t pt = tmem + b * 128;
 #pragma unroll
-        for (int ks = 0; ks < TN / 16; ++ks)
+        for (int ks = 0; ks < TN / 32; ++ks)
           mma_ts(tmem_O, pt + ks * 8, vdesc + (uint64_t)(ks * (2048 >> 4)), IDESC_PV, (idx > 0 || ks > 0) ? 1u : 0u);
+        if (!mbar_wait(bar_pready2(b), (uint32_t)(idx >> 1) & 1u, abort_flag, p.status)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int ks = TN / 32; ks < TN / 16; ++ks)
+          mma_ts(tmem_O, pt + ks * 8, vdesc + (uint64_t)(ks * (2048 >> 4)), IDESC_PV, 1u);
         tc_commit(bar_empty(slot));
         tc_commit(bar_pvdone);
         ++q;
@@ -640,40 +646,51 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
       // p = 2^(s*scale_log2 - m_ref); a fully masked row so far (m_ref = -inf) contributes zeros
       const float mneg = m_ref == -INFINITY ? 0.f : -m_ref;
-      uint32_t preg[64];
-      float ls4[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int c = 0; c < 64; ++c) {
-        const float p0 = ex2(fmaf(__uint_as_float(sreg[2 * c]), p.scale_log2, mneg));
-        const float p1 = ex2(fmaf(__uint_as_float(sreg[2 * c + 1]), p.scale_log2, mneg));
-        ls4[c & 3] += p0 + p1;
-        preg[c] = pack_bf16(p0, p1);
-      }
-      l = l * alpha + ((ls4[0] + ls4[1]) + (ls4[2] + ls4[3]));
-      if (idx > 0) {
-        // P_{idx-1} V_{idx-1} must have left the tensor core before O is touched; waiting for every phase in
-        // order also keeps the parity of this barrier unambiguous
+      if (idx > 0 && __any_sync(0xffffffffu, rescale)) {   // tcgen05.ld/st are warp-collective: the whole warp takes the branch
+        // P_{idx-1} V_{idx-1} must have left the tensor core before O is touched.  Phases that were not waited for
+        // cannot alias: phase idx of this barrier needs this thread's own arrival below.
         if (!__all_sync(0xffffffffu, mbar_wait(bar_pvdone, (uint32_t)(idx - 1) & 1u, abort_flag, p.status))) { ok = false; break; }
-        if (__any_sync(0xffffffffu, rescale)) {   // tcgen05.ld/st are warp-collective: the whole warp takes the branch
-          tc_fence_after();
+        tc_fence_after();
 #pragma unroll
-          for (int cb = 0; cb < 4; ++cb) {
-            uint32_t oreg[32];
-            TC_LD32(tmem_O + lane_off + cb * 32, oreg);
-            tc_wait_ld();
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t oreg[32];
+          TC_LD32(tmem_O + lane_off + cb * 32, oreg);
+          tc_wait_ld();
 #pragma unroll
-            for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * alpha);
-            TC_ST32(tmem_O + lane_off + cb * 32, oreg);
-          }
+          for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * alpha);
+          TC_ST32(tmem_O + lane_off + cb * 32, oreg);
         }
       }
-      TC_ST32(ts, (preg + 0));
-      TC_ST32(ts + 32, (preg + 32));
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int ch = 0; ch < 4; ++ch) {                 // 32 keys at a time: exponentials, bf16 P, row sum
+        uint32_t preg[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int c = ch * 32 + 2 * i;
+          float x0, x1;
+          ffma2(x0, x1, __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]), p.scale_log2, p.scale_log2, mneg, mneg);
+          const float p0 = ex2(x0), p1 = ex2(x1);
+          preg[i] = pack_bf16(p0, p1);
+          fadd2(acc[(i & 1) * 2], acc[(i & 1) * 2 + 1], acc[(i & 1) * 2], acc[(i & 1) * 2 + 1], p0, p1);
+        }
+        TC_ST16(ts + ch * 16, preg);
+        if (ch == 1) {                                 // keys 0..63 of P are in place: the first half of P V may start
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(bar_pready(b));
+        }
+      }
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(bar_pready(b));
+      mbar_arrive(bar_pready2(b));
+      l = l * alpha + ((acc[0] + acc[1]) + (acc[2] + acc[3]));
     }
     // ---- epilogue: wait for the last P V, normalise, write out -----------------------------------
+    // The loop waits on this barrier only before a rescale, so it may still be in phase nt-2 here (S_{nt-1} being
+    // complete says no more than that P_{nt-3} V_{nt-3} is): take the last two phases in order, or the parity of
+    // phase nt-1 would be mistaken for complete.
+    if (ok && nt >= 2) ok = __all_sync(0xffffffffu, mbar_wait(bar_pvdone, (uint32_t)(nt - 2) & 1u, abort_flag, p.status));
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_pvdone, (uint32_t)(nt - 1) & 1u, abort_flag, p.status));
     if (ok) {
       tc_fence_after();
