@@ -6,7 +6,9 @@
 // column sum needs no cross-thread reduction and no second pass over the tile.  K streams once through a TMA
 // ring (this kernel is HBM-bound); the query rows of one KV group stay resident in shared memory.
 //
-// Warp roles (192 threads): warp 0 TMA producer, warp 1 tcgen05.mma issuer + TMEM owner, warps 2..5 consumers.
+// Warp roles (320 threads): warp 0 TMA producer, warp 1 tcgen05.mma issuer + TMEM owner, warps 2..5 and 6..9 two
+// consumer warpgroups that take the (key tile, head) units in turn: one warpgroup alone (a 64-column row of
+// exponentials per thread and unit) was the slowest stage of the pipeline.
 #include "tc_common.cuh"
 
 using namespace tc;
@@ -17,7 +19,7 @@ constexpr int TK = 128;               // keys per tile (MMA M)
 constexpr int HD = 128;
 constexpr int SLOT_BYTES = TK * HD * 2;
 constexpr int HALF_BYTES = SLOT_BYTES / 2;
-constexpr int NTHREADS = 192;
+constexpr int NTHREADS = 320;
 constexpr int MAX_SLOTS = 6;
 constexpr int MAX_NPAD = 256;
 constexpr int MAX_BUF = 8;              // TMEM accumulator buffers (512 columns / buffer width)
@@ -35,7 +37,17 @@ struct SinkParams {
   int kv_div;                     // the kernel walks QUERY heads (Hkv = H, hpg = 1); query head h reads KV head h / kv_div
   float scale_log2;
   int32_t* status;
+#ifdef FOCUS_TIMELINE
+  unsigned long long* dbg;        // per-iteration clock stamps of CTA 0 (development builds only)
+#endif
 };
+
+#ifdef FOCUS_TIMELINE
+__device__ __forceinline__ unsigned long long tl_clock() { unsigned long long c; asm volatile("mov.u64 %0, %%clock64;" : "=l"(c) :: "memory"); return c; }
+#define TL_ITER(who, tid, it, ev) do { if (p.dbg && blockIdx.x == 0 && threadIdx.x == (tid) && (it) < 64) p.dbg[65536 + (who) * 512 + (it) * 8 + (ev)] = tl_clock(); } while (0)
+#else
+#define TL_ITER(who, tid, it, ev) do { } while (0)
+#endif
 
 #define TC_LD16(taddr, r)                                                                                         \
   asm volatile(                                                                                                   \
@@ -107,7 +119,7 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
   }
   for (int idx = threadIdx.x; idx < heads_staged * p.n_pad; idx += NTHREADS) {
     const int r = idx % p.n_pad, hs = idx / p.n_pad;
-    neg_lse2[idx] = r < n ? -p.lse[(size_t)(g0 * p.hpg + hs) * p.lse_stride + r] * 1.4426950408889634f : 0.f;
+    neg_lse2[idx] = r < n ? -p.lse[(size_t)(g0 * p.hpg + hs) * p.lse_stride + r] * 1.4426950408889634f : -INFINITY;
   }
   fence_proxy_async();
   tc_fence_before();
@@ -115,21 +127,26 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
   tc_fence_after();
   const uint32_t tmem = *tmem_holder;
   const int units = nt * p.hpg;                  // one unit = (key tile, query head of the group)
+  const int ncol = max(32, (n + 31) & ~31);       // query columns in use: the active rows, padded to 32 (one TMEM load)
 
   if (warp == 0) {
     if (lane == 0) {
       int issued = 0;
       bool ok = true;
+      // tile t of head g; ring slot and phase follow the tile counter without divisions
+      int t = u0 % T, g = u0 / T, kvh = g / p.kv_div, slot = 0;
+      uint32_t ph = 0;
       for (int i = 0; i < nt && ok; ++i) {
-        const int slot = i % p.n_slots;
-        const uint32_t ph = (uint32_t)(i / p.n_slots) & 1u;
+        TL_ITER(0, 0, i, 0);
         if (!mbar_wait(bar_empty(slot), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        TL_ITER(0, 0, i, 1);
         const uint32_t dst = sSlot + slot * SLOT_BYTES;
         mbar_expect_tx(bar_full(slot), SLOT_BYTES);
-        const int u = u0 + i;
-        tma_load_3d(dst, &tmK, bar_full(slot), 0, (u % T) * TK, u / T / p.kv_div);
-        tma_load_3d(dst + HALF_BYTES, &tmK, bar_full(slot), 64, (u % T) * TK, u / T / p.kv_div);
+        tma_load_3d(dst, &tmK, bar_full(slot), 0, t * TK, kvh);
+        tma_load_3d(dst + HALF_BYTES, &tmK, bar_full(slot), 64, t * TK, kvh);
         ++issued;
+        if (++slot == p.n_slots) { slot = 0; ph ^= 1u; }
+        if (++t == T) { t = 0; ++g; kvh = g / p.kv_div; }
       }
       if (!ok) {
         const int first = issued > p.n_slots ? issued - p.n_slots : 0;
@@ -142,17 +159,23 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc = make_idesc(TK, p.n_pad, 0);
+      const uint32_t idesc = make_idesc(TK, ncol, 0);
       bool ok = true;
+      // unit u = (key tile i, head hh of the group); slot/phase of the K ring, buffer/phase of the accumulator ring
+      // and the staged head slot follow u without divisions
+      const int nbuf_mask = p.n_buf - 1, nbuf_shift = 31 - __clz(p.n_buf);
+      int hh = 0, slot = 0, t = u0 % T, hs0 = (u0 / T - g0) * p.hpg;
+      uint32_t ph = 0;
       for (int u = 0; u < units && ok; ++u) {
-        const int i = u / p.hpg, hh = u % p.hpg;
-        const int slot = i % p.n_slots, b = u % p.n_buf;
-        if (!mbar_wait(bar_sempty(b), ((uint32_t)(u / p.n_buf) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
-        if (hh == 0 && !mbar_wait(bar_full(slot), (uint32_t)(i / p.n_slots) & 1u, abort_flag, p.status)) { ok = false; break; }
+        const int b = u & nbuf_mask;
+        TL_ITER(1, 32, u, 0);
+        if (!mbar_wait(bar_sempty(b), ((uint32_t)(u >> nbuf_shift) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        TL_ITER(1, 32, u, 1);
+        if (hh == 0 && !mbar_wait(bar_full(slot), ph, abort_flag, p.status)) { ok = false; break; }
+        TL_ITER(1, 32, u, 2);
         tc_fence_after();
         const uint64_t kdesc = make_sdesc(sSlot + slot * SLOT_BYTES, 16, 1024);
-        const int hs = ((u0 + i) / T - g0) * p.hpg + hh;
-        const uint64_t qdesc = make_sdesc(sQ + hs * q_head_bytes, 16, 1024);
+        const uint64_t qdesc = make_sdesc(sQ + (hs0 + hh) * q_head_bytes, 16, 1024);
 #pragma unroll
         for (int half = 0; half < 2; ++half)
 #pragma unroll
@@ -160,49 +183,71 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
             mma_ss(tmem + b * p.buf_cols, kdesc + (uint64_t)((half * HALF_BYTES + ks * 32) >> 4),
                    qdesc + (uint64_t)((half * (p.n_pad * 128) + ks * 32) >> 4), idesc, (half | ks) ? 1u : 0u);
         tc_commit(bar_sfull(b));
-        if (hh == p.hpg - 1) tc_commit(bar_empty(slot));
+        if (++hh == p.hpg) {
+          hh = 0;
+          tc_commit(bar_empty(slot));
+          if (++slot == p.n_slots) { slot = 0; ph ^= 1u; }
+          if (++t == T) { t = 0; hs0 += p.hpg; }
+        }
+        TL_ITER(1, 32, u, 3);
       }
     }
   } else {
-    const int rq = warp & 3;
+    const int rq = warp & 3;                                  // TMEM lane quarter this warp may access
     const int krow = rq * 32 + lane;                          // key of this thread inside the tile
     const uint32_t lane_off = (uint32_t)(rq * 32) << 16;
-    for (int u = 0; u < units; ++u) {
-      const int i = u / p.hpg, hh = u % p.hpg, b = u % p.n_buf;
-      if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(b), (uint32_t)(u / p.n_buf) & 1u, abort_flag, p.status))) break;
+    // unit u = (key tile i = u / hpg, head hh = u % hpg of the group); the counters below follow u without divisions
+    const int cw = (warp - 2) >> 2;                           // consumer warpgroup: units cw, cw + 2, ...
+    const int nbuf_mask = p.n_buf - 1, nbuf_shift = 31 - __clz(p.n_buf);   // n_buf is a power of two (2, 4 or 8)
+    int i = cw / p.hpg, hh = cw % p.hpg;
+    int t = (u0 + i) % T, g = (u0 + i) / T;
+    for (int u = cw; u < units; u += 2) {
+      const int b = u & nbuf_mask;
+      TL_ITER(2, 64, u, 0);
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(b), (uint32_t)(u >> nbuf_shift) & 1u, abort_flag, p.status))) break;
+      TL_ITER(2, 64, u, 1);
       tc_fence_after();
-      const int g = (u0 + i) / T;
       const float* nl = neg_lse2 + ((g - g0) * p.hpg + hh) * p.n_pad;
       float acc = 0.f;
       const uint32_t tsrc = tmem + lane_off + b * p.buf_cols;
-      if (p.n_pad <= 64) {
-        // common case (at most 64 active rows per head): every column chunk is requested before the single wait,
-        // and the accumulator buffer goes back to the MMA warp before the exponentials are taken
+      // columns in groups of 64: both 32-column loads of a group are requested before the single wait; the
+      // accumulator buffer goes back to the MMA warp as soon as its last group sits in registers.  Columns past
+      // the n active rows carry -inf in nl[] (their probabilities are zero).
+      float acc4[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int c0 = 0; c0 < ncol; c0 += 64) {
         uint32_t r[64];
-        TC_LD16(tsrc, (r + 0));
-        if (p.n_pad > 16) TC_LD16(tsrc + 16, (r + 16));
-        if (p.n_pad > 32) TC_LD16(tsrc + 32, (r + 32));
-        if (p.n_pad > 48) TC_LD16(tsrc + 48, (r + 48));
+        const bool two = c0 + 32 < ncol;
+        TC_LD32(tsrc + c0, (r + 0));
+        if (two) TC_LD32(tsrc + c0 + 32, (r + 32));
         tc_wait_ld();
-        tc_fence_before();
-        mbar_arrive(bar_sempty(b));
-#pragma unroll
-        for (int c = 0; c < 64; ++c)
-          if (c < n) acc += ex2(fmaf(__uint_as_float(r[c]), p.scale_log2, nl[c]));
-      } else {
-        for (int c0 = 0; c0 < n; c0 += 16) {
-          uint32_t r[16];
-          TC_LD16(tsrc + c0, r);
-          tc_wait_ld();
-#pragma unroll
-          for (int c = 0; c < 16; ++c)
-            if (c0 + c < n) acc += ex2(fmaf(__uint_as_float(r[c]), p.scale_log2, nl[c0 + c]));
+        if (c0 + 64 >= ncol) {
+          tc_fence_before();
+          mbar_arrive(bar_sempty(b));
+          TL_ITER(2, 64, u, 2);
         }
-        tc_fence_before();
-        mbar_arrive(bar_sempty(b));
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          if (hf == 0 || two) {
+#pragma unroll
+            for (int c4 = 0; c4 < 8; ++c4) {
+              const float4 nv = *reinterpret_cast<const float4*>(nl + c0 + hf * 32 + c4 * 4);
+              acc4[0] += ex2(fmaf(__uint_as_float(r[hf * 32 + c4 * 4 + 0]), p.scale_log2, nv.x));
+              acc4[1] += ex2(fmaf(__uint_as_float(r[hf * 32 + c4 * 4 + 1]), p.scale_log2, nv.y));
+              acc4[2] += ex2(fmaf(__uint_as_float(r[hf * 32 + c4 * 4 + 2]), p.scale_log2, nv.z));
+              acc4[3] += ex2(fmaf(__uint_as_float(r[hf * 32 + c4 * 4 + 3]), p.scale_log2, nv.w));
+            }
+          }
+        }
       }
-      const int key = ((u0 + i) % T) * TK + krow;
+      acc = (acc4[0] + acc4[1]) + (acc4[2] + acc4[3]);
+      const int key = t * TK + krow;
       if (key < p.L) p.part[(size_t)(g * p.hpg + hh) * p.L + key] = acc;
+      TL_ITER(2, 64, u, 3);
+      hh += 2;
+      while (hh >= p.hpg) {
+        hh -= p.hpg;
+        if (++t == T) { t = 0; ++g; }
+      }
     }
   }
   tc_fence_before();
@@ -215,7 +260,7 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
 
 }  // namespace
 
-static int sink_npad(int max_active) { return (max_active + 15) / 16 * 16; }
+static int sink_npad(int max_active) { return (max_active + 31) / 32 * 32; }
 static int sink_slots(int heads_staged, int n_pad) {
   const int fixed = 1024 + heads_staged * n_pad * 256 + (2 * MAX_SLOTS + 2 * MAX_BUF) * 8 + 16 + heads_staged * n_pad * 4 + 64;
   int s = (232448 - fixed) / SLOT_BYTES;
@@ -265,6 +310,9 @@ focus_status launch_sink_colsum_tc(focus_ctx* ctx, const focus_shape* s, const v
   p.n_slots = sink_slots(p.groups_staged * hpg, p.n_pad);
   p.scale_log2 = shape_scale(s) * 1.4426950408889634f;
   p.status = ctx->d_status;
+#ifdef FOCUS_TIMELINE
+  p.dbg = getenv("FOCUS_TIMELINE") ? (unsigned long long*)(ctx->ws + ctx->ws_bytes - (1 << 20)) : nullptr;
+#endif
   CUtensorMap tmK;
   if (!encode_kv_map(ctx->encode_tiled, &tmK, K, HD, s->L, kvh, s->kv_stride_tok, s->kv_stride_head, 64, TK))
     return FOCUS_ERR_INVALID_ARG;
