@@ -343,6 +343,30 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   int* s_last_p = reinterpret_cast<int*>(tmem_holder + 2);
   int2* tlist = reinterpret_cast<int2*>(tmem_holder + 16);      // (start | kind << 30, nvalid) per tile of this split
 
+  // Programmatic dependent launch.  Every launch of this kernel lets its successor in the stream start early
+  // (launch_dependents) and may itself have been started before its predecessor finished.  p.pdl = 2: the
+  // predecessor is unknown, so nothing in global memory is touched before griddepcontrol.wait; only the private
+  // set-up (barriers, TMEM) runs ahead.  p.pdl = 1: the predecessor is the selection kernel of the same sparse layer
+  // (see further down).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  auto arm_barriers = [&]() {                        // warp 0, lane 0
+    for (int sl = 0; sl < NSLOT; ++sl) { mbar_init(bar_full(sl), 1); mbar_init(bar_empty(sl), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pready(b), 128); mbar_init(bar_pready2(b), 128); }
+    mbar_init(bar_pvdone, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async();
+  };
+  auto alloc_tmem = [&]() {                          // warp 1, all lanes
+    tmem_alloc(smem_u32(tmem_holder), 512);
+    tmem_relinquish();
+  };
+  if (p.pdl == 2) {
+    if (warp == 0 && lane == 0) arm_barriers();
+    if (warp == 1) alloc_tmem();
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+  }
+
   // The prologue is a chain of global-memory latencies; everything that does not depend on another load is
   // requested first: the row count, this group's block count, the positions of this thread's Q rows.
   constexpr int QTHREADS = 128;                                  // the four softmax warps stage Q
@@ -358,7 +382,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   }
   const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
   const int total_fr = nrows * p.hpg;                    // stacked (row, head-of-group) rows of this KV head
-  if (mt * TM >= total_fr) return;                       // uniform: nothing to compute for this tile
+  if (mt * TM >= total_fr) {                             // uniform: nothing to compute for this tile
+    if (p.pdl == 2) {                                    // TMEM was allocated ahead of the row count
+      tc_fence_before();
+      __syncthreads();
+      tc_fence_after();
+      if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(*tmem_holder, 512);
+      }
+    }
+    return;
+  }
 
   // query rows of this thread (softmax warps only): requested now, stored to shared memory further down
   uint4 qv[QIT];
@@ -381,21 +416,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
     }
   }
-  // Launched as a programmatic dependent of the selection kernel of the same sparse layer: everything above
-  // (row list, query rows) does not come from that kernel and overlaps with it; the block lists, the gathered
-  // sink rows and their mask do, so nothing below may start before it has completed.
-  auto arm_barriers = [&]() {                        // warp 0, lane 0
-    for (int sl = 0; sl < NSLOT; ++sl) { mbar_init(bar_full(sl), 1); mbar_init(bar_empty(sl), 1); }
-    for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pready(b), 128); mbar_init(bar_pready2(b), 128); }
-    mbar_init(bar_pvdone, 1);
-    *abort_flag = 0;
-    fence_barrier_init();
-    fence_proxy_async();
-  };
-  auto alloc_tmem = [&]() {                          // warp 1, all lanes
-    tmem_alloc(smem_u32(tmem_holder), 512);
-    tmem_relinquish();
-  };
   auto store_q = [&]() {                             // softmax warps
 #pragma unroll
     for (int it = 0; it < QIT; ++it) {
@@ -405,7 +425,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       *reinterpret_cast<uint4*>(sptr + half * HALF_BYTES + r * 128 + ((cc ^ (r & 7)) << 4)) = qv[it];
     }
   };
-  if (p.pdl) {
+  // Launched as a programmatic dependent of the selection kernel of the same sparse layer: everything above
+  // (row list, query rows) does not come from that kernel and overlaps with it; the block lists, the gathered
+  // sink rows and their mask do, so nothing below may start before it has completed.
+  if (p.pdl == 1) {
     // as a programmatic dependent the whole private set-up runs while the selection kernel is still at work
     if (warp == 0 && lane == 0) arm_barriers();
     if (warp == 1) alloc_tmem();
@@ -504,7 +527,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   if (warp == 1 && !p.pdl) alloc_tmem();
   // Q tile -> shared memory in the 128-byte-swizzled K-major layout the MMA descriptor expects:
   // half h (columns 64h..64h+63) at h*16 KB, row r at r*128 bytes, 16-byte chunk c at ((c ^ (r & 7)) * 16).
-  if (qtid >= 0 && !p.pdl) store_q();
+  if (qtid >= 0 && p.pdl != 1) store_q();
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();
@@ -795,6 +818,9 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   TL_STAMP(0, 0);
   const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
+  // programmatic dependent launch: let the successor start early; wait for the predecessor before touching memory
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (p.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   constexpr int QTHREADS = 256;                                  // the eight softmax warps stage Q
   constexpr int QIT = TMW * 16 / QTHREADS;
@@ -1421,7 +1447,8 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.q_rows = a.q_rows; p.n_rows = a.n_rows; p.block_idx = a.block_idx; p.block_cnt = a.block_cnt;
   p.sink_mask = mask; p.part_O = part_O; p.part_ml = part_ml;
   p.cluster = use_cluster ? 1 : 0;
-  p.pdl = (pre != nullptr && !wide && !ctx->no_pdl) ? 1 : 0;   // pre-gathered sinks: called right after the selection kernel
+  // 1: called right after the selection kernel of a fused sparse layer (pre-gathered sinks); 2: predecessor unknown
+  p.pdl = ctx->no_pdl ? 0 : ((pre != nullptr && !wide) ? 1 : 2);
   p.counters = (n_splits > 1 && !use_cluster && !wide && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
                    ? ctx->d_counters : nullptr;
   p.q_stride_row = sh.q_stride_row; p.q_stride_head = sh.q_stride_head;
@@ -1437,7 +1464,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
 
   ctx->last_attn_variant = wide ? 3 : 2;
   if (wide) {
-    focus_status ls = launch_ex(attn_tc_wide_kernel, dim3(base, n_splits, 1), NTHREADS_W, SMEM_BYTES_W, n_splits, false, st,
+    focus_status ls = launch_ex(attn_tc_wide_kernel, dim3(base, n_splits, 1), NTHREADS_W, SMEM_BYTES_W, n_splits, p.pdl != 0, st,
                                 tmK, tmV, tmSK, tmSV, p);
     if (ls != FOCUS_OK) return ls;
   } else {

@@ -19,8 +19,11 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
                     __nv_bfloat16* __restrict__ gV, uint8_t* __restrict__ mask, int32_t* status) {
   const int tid = threadIdx.x;
   // the attention kernel of this layer is launched as a programmatic dependent: let its CTAs start their own
-  // set-up now; it waits for this grid to complete before it reads anything written here
+  // set-up now; it waits for this grid to complete before it reads anything written here.  This kernel may itself
+  // have been started before its predecessor in the stream finished: nothing is read or written before the wait
+  // (the gather below overwrites rows the previous layer's attention kernel may still be reading).
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if ((int)blockIdx.x >= Hkv) {
     // ---- gather: 64 sink rows of one KV head per CTA, one 16-byte chunk of K and of V per thread ---------
     const int gi = (int)blockIdx.x - Hkv;
@@ -195,11 +198,20 @@ extern "C" focus_status focus_sparse_layer(focus_ctx* ctx, const focus_shape* sh
   }
   if (!ws.ok) return FOCUS_ERR_WORKSPACE_TOO_SMALL;
   const int grid = Hkv + (ns_pad + 63) / 64 * Hkv;
-  fused_select_kernel<<<grid, FS_THREADS, 0, stream>>>(
-      (const __nv_bfloat16*)Q, q_base, shape->q_stride_row, shape->q_stride_head, focus_idx, n_focus, max_focus, Kbar,
-      Hkv, hpg, shape->L, shape->M, shape->kv_block, nb, C, sink_idx, n_sink, ns_pad, (const __nv_bfloat16*)K,
-      (const __nv_bfloat16*)V, shape->kv_stride_tok, shape->kv_stride_head, R, block_idx, block_cnt, sink_keep, sg.gK,
-      sg.gV, sg.mask, ctx->d_status);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid, 1, 1); cfg.blockDim = dim3(FS_THREADS, 1, 1); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at; cfg.numAttrs = ctx->no_pdl ? 0 : 1;
+  if (cudaLaunchKernelEx(&cfg, fused_select_kernel,
+      (const __nv_bfloat16*)Q, q_base, (long long)shape->q_stride_row, (long long)shape->q_stride_head, focus_idx, n_focus,
+      max_focus, Kbar, Hkv, hpg, (int)shape->L, (int)shape->M, (int)shape->kv_block, nb, C, sink_idx, n_sink, ns_pad,
+      (const __nv_bfloat16*)K, (const __nv_bfloat16*)V, (long long)shape->kv_stride_tok, (long long)shape->kv_stride_head, R,
+      block_idx, block_cnt, sink_keep, sg.gK, sg.gV, sg.mask, ctx->d_status) != cudaSuccess) {
+    cudaGetLastError();
+    return FOCUS_ERR_CUDA;
+  }
   FOCUS_CHECK_LAUNCH();
   return launch_attn_tc_ws(ctx, a, ws, &sg, stream);
 }
