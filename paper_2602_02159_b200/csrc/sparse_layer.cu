@@ -18,12 +18,14 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
                     int32_t* __restrict__ block_cnt, uint8_t* __restrict__ sink_keep, __nv_bfloat16* __restrict__ gK,
                     __nv_bfloat16* __restrict__ gV, uint8_t* __restrict__ mask, int32_t* status) {
   const int tid = threadIdx.x;
-  // the attention kernel of this layer is launched as a programmatic dependent: let its CTAs start their own
+  // The attention kernel of this layer is launched as a programmatic dependent: let its CTAs start their own
   // set-up now; it waits for this grid to complete before it reads anything written here.  This kernel may itself
-  // have been started before its predecessor in the stream finished: nothing is read or written before the wait
-  // (the gather below overwrites rows the previous layer's attention kernel may still be reading).
+  // have been started before its predecessor in the stream finished.  The only kernels that let a successor start
+  // early are this one and the attention kernels; what they may still be reading are the buffers written below
+  // after griddepcontrol.wait (block list and count, keep flags, mask, gathered rows).  Everything read before the
+  // wait (Q, pooled keys, K/V rows, focus and sink indices) comes from kernels that do not release their successors
+  // early, so it is complete once this kernel runs at all; R and the status word are read by no such kernel.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
   if ((int)blockIdx.x >= Hkv) {
     // ---- gather: 64 sink rows of one KV head per CTA, one 16-byte chunk of K and of V per thread ---------
     const int gi = (int)blockIdx.x - Hkv;
@@ -42,6 +44,7 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
       }
     }
     const size_t o = ((size_t)g * ns_pad + s) * FS_HD + c * 8;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     *reinterpret_cast<uint4*>(gK + o) = kv;
     *reinterpret_cast<uint4*>(gV + o) = vv;
     return;
@@ -121,6 +124,7 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
     sel[i] = rank < C;
   }
   __syncthreads();
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   for (int s = tid; s < ns_pad; s += FS_THREADS) {
     uint8_t keep = 0, mk = 0;
     if (s < n_sink) {
