@@ -8,7 +8,9 @@ constexpr int FS_MAX_NB = 8192;
 constexpr int FS_HD = 128;
 
 // CTAs [0, Hkv): selection for KV head g.  CTAs [Hkv, ...): gather 64 sink rows of K and V of one KV head each.
-__global__ void __launch_bounds__(FS_THREADS)
+// At most 32 registers per thread: two CTAs fit one SM, so the selection CTAs of all KV heads can run on the SMs
+// that an attention launch of 128 CTAs leaves idle, ahead of the dependency wait.
+__global__ void __launch_bounds__(FS_THREADS, 2)
 fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q_stride_row, long long q_stride_head,
                     const int32_t* __restrict__ focus_idx, const int32_t* __restrict__ n_focus, int max_focus,
                     const float* __restrict__ Kbar, int Hkv, int hpg, int L, int M, int B, int nb, int C,
@@ -59,7 +61,7 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
   const int warp = tid >> 5, lane = tid & 31;
   // Issue every load that does not depend on another one first: the kernel is a chain of global-memory
   // latencies, not of bandwidth.
-  constexpr int KPRE = 8;
+  constexpr int KPRE = 4;
   const float* kb = Kbar + (size_t)g * nb * FS_HD + lane * 4;
   float4 kpre[KPRE];
 #pragma unroll
