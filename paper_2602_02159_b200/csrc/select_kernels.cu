@@ -336,11 +336,226 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
   for (int i = tot_sel + tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Stage 2, selection half, on one thread-block cluster (SC_CTAS CTAs): exact Top-n of the head-reduced scores and
+// the ascending index list.  CTA r owns the r-th contiguous chunk of the candidates, keeps their
+// order-preserving keys in shared memory and never looks at another CTA's keys; what the CTAs exchange through
+// distributed shared memory are a few words per step:
+//   (1) AND / OR of all keys  -> the bits on which every key agrees are skipped (sink scores all sit near 1/L);
+//   (2) per 8-bit digit, MSB first, a 256-bin histogram of the keys that still match the prefix of the n-th largest
+//       key T: every CTA adds up the SC_CTAS histograms and takes the same decision (two histogram buffers in turn,
+//       so one cluster barrier per digit suffices);
+//   (3) per CTA the number of keys > T and == T: keys equal to T are taken in global index order until the quota
+//       is filled, which fixes every CTA's output offset and its share of the equals.
+// Inside a CTA the selected positions are written ascending by warp-ordered ballot compaction.
+// ------------------------------------------------------------------------------------------------
+constexpr int SC_CTAS = 8;
+constexpr int SC_THREADS = 1024;
+constexpr int SC_MAX_KEYS = 48 * 1024;                 // keys per CTA (192 KB of dynamic shared memory)
+
+__device__ __forceinline__ uint32_t sc_map(const void* p, uint32_t rank) {
+  uint32_t a = (uint32_t)__cvta_generic_to_shared(p), r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ uint32_t sc_ld(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sc_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(SC_THREADS, 1)
+sink_select_cluster_kernel(const float* __restrict__ S, const int32_t* n_active, int lo, int hi, int n_sink,
+                           int32_t* __restrict__ sink_idx, int32_t* status) {
+  extern __shared__ uint32_t skey[];                    // this CTA's keys
+  __shared__ uint32_t xch[4];                           // and, or, #keys > T, #keys == T of this CTA
+  __shared__ uint32_t hist[2][256];
+  __shared__ uint32_t tot[256];
+  __shared__ int scan_s[33];
+  __shared__ int s_digit, s_above;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  const int n = hi - lo;
+  const int want = min(n_sink, n);
+  const int n_act = *n_active;
+  const int chunk = (n + SC_CTAS - 1) / SC_CTAS;
+  const int c_lo = min((int)rank * chunk, n), c_hi = min(c_lo + chunk, n), cn = c_hi - c_lo;
+  uint32_t a = 0xFFFFFFFFu, o = 0u;
+#pragma unroll 4
+  for (int i = tid; i < cn; i += SC_THREADS) {
+    const uint32_t k = float_key(S[lo + c_lo + i]);
+    skey[i] = k;
+    a &= k; o |= k;
+  }
+  if (n_act <= 0 || want == 0) {                        // undefined scores or nothing asked for: an empty set
+    if (n_act <= 0 && tid == 0 && rank == 0) set_status(status, FOCUS_ERR_INVALID_ARG);
+    for (int i = (int)rank * SC_THREADS + tid; i < n_sink; i += SC_CTAS * SC_THREADS) sink_idx[i] = -1;
+    return;                                             // uniform over the cluster: nobody waits at a barrier
+  }
+  if (tid < 256) { hist[0][tid] = 0u; hist[1][tid] = 0u; }
+  if (tid == 0) { xch[0] = 0xFFFFFFFFu; xch[1] = 0u; }
+  __syncthreads();
+  a = __reduce_and_sync(0xffffffffu, a);
+  o = __reduce_or_sync(0xffffffffu, o);
+  if (lane == 0) { atomicAnd(&xch[0], a); atomicOr(&xch[1], o); }
+  __syncthreads();
+  sc_sync();
+  uint32_t g_and = 0xFFFFFFFFu, g_or = 0u;
+#pragma unroll
+  for (int r = 0; r < SC_CTAS; ++r) { g_and &= sc_ld(sc_map(&xch[0], r)); g_or |= sc_ld(sc_map(&xch[1], r)); }
+  const uint32_t diff = g_and ^ g_or;
+  int hb = diff ? 31 - __clz(diff) : -1;                // highest bit on which two keys differ
+  // T: key of the want-th largest element, built digit by digit below the common prefix
+  uint32_t T = hb >= 31 ? 0u : (hb >= 0 ? (g_or & ~((2u << hb) - 1u)) : g_or);
+  int need = want;                                      // rank of T among the keys that share its prefix (1 = largest)
+  int pass = 0;
+  while (hb >= 0) {
+    const int shift = hb >= 7 ? hb - 7 : 0;             // digit = bits [shift, shift + width)
+    const int width = hb - shift + 1;
+    const uint32_t dmask = (1u << width) - 1u;
+    const uint32_t pmask = (hb >= 31) ? 0u : ~((2u << hb) - 1u);     // prefix bits above the digit
+    uint32_t* hs = hist[pass & 1];
+    for (int i = tid; i < cn; i += SC_THREADS) {
+      const uint32_t k = skey[i];
+      if ((k & pmask) == (T & pmask)) atomicAdd(&hs[(k >> shift) & dmask], 1u);
+    }
+    __syncthreads();
+    sc_sync();
+    if (tid < 256) {
+      uint32_t t = 0u;
+#pragma unroll
+      for (int r = 0; r < SC_CTAS; ++r) t += sc_ld(sc_map(&hs[tid], r));
+      tot[tid] = t;
+      // the other buffer is cleared for the next digit: whoever read it (previous digit) did so before arriving at
+      // the barrier above
+      hist[(pass + 1) & 1][tid] = 0u;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // digits from the largest down: the first one whose cumulative count reaches `need`
+      int run = 0, found = -1, above = 0;
+      for (int base = 255; base >= 0 && found < 0; base -= 32) {
+        const int d = base - lane;                      // lane 0 holds the largest digit of this group of 32
+        const int c = (int)tot[d];
+        int inc = c;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, inc, off);
+          if (lane >= off) inc += y;
+        }
+        const uint32_t hit = __ballot_sync(0xffffffffu, run + inc >= need);
+        if (hit) {
+          const int l0 = __ffs(hit) - 1;
+          found = base - l0;
+          above = run + __shfl_sync(0xffffffffu, inc - c, l0);
+        }
+        run += __shfl_sync(0xffffffffu, inc, 31);
+      }
+      if (lane == 0) { s_digit = found; s_above = above; }
+    }
+    __syncthreads();
+    const int d = s_digit;
+    T |= (uint32_t)d << shift;
+    need -= s_above;
+    hb = shift - 1;
+    ++pass;
+    __syncthreads();
+  }
+  // keys > T and == T of this CTA
+  int n_gt_l = 0, n_eq_l = 0;
+  for (int i = tid; i < cn; i += SC_THREADS) {
+    const uint32_t k = skey[i];
+    n_gt_l += k > T ? 1 : 0;
+    n_eq_l += k == T ? 1 : 0;
+  }
+  n_gt_l = __reduce_add_sync(0xffffffffu, n_gt_l);
+  n_eq_l = __reduce_add_sync(0xffffffffu, n_eq_l);
+  if (tid == 0) { xch[2] = 0u; xch[3] = 0u; }
+  __syncthreads();
+  if (lane == 0) { atomicAdd(&xch[2], (uint32_t)n_gt_l); atomicAdd(&xch[3], (uint32_t)n_eq_l); }
+  __syncthreads();
+  sc_sync();
+  int gt_all = 0;
+#pragma unroll
+  for (int r = 0; r < SC_CTAS; ++r) gt_all += (int)sc_ld(sc_map(&xch[2], r));
+  const int remaining = want - gt_all;                  // keys == T to take, lowest index first
+  int out_base = 0, eq_before = 0, my_eq = 0;
+#pragma unroll
+  for (int r = 0; r < SC_CTAS; ++r) {
+    const int g = (int)sc_ld(sc_map(&xch[2], r)), e = (int)sc_ld(sc_map(&xch[3], r));
+    const int take = max(0, min(e, remaining - eq_before));
+    if (r < (int)rank) out_base += g + take;
+    if (r == (int)rank) my_eq = take;
+    eq_before += e;
+  }
+  // ordered compaction inside the CTA: warp w owns keys [w*seg, (w+1)*seg), seg a multiple of 32
+  const int seg = ((cn + 31) / 32 + 31) / 32 * 32;
+  const int w_lo = min(warp * seg, cn), w_hi = min(w_lo + seg, cn);
+  int n_gt = 0, n_eq = 0;
+  for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
+    const int i = i0 + lane;
+    const uint32_t k = i < w_hi ? skey[i] : 0u;
+    n_gt += __popc(__ballot_sync(0xffffffffu, i < w_hi && k > T));
+    n_eq += __popc(__ballot_sync(0xffffffffu, i < w_hi && k == T));
+  }
+  int tot_eq, tot_sel;
+  const int pre_eq = block_excl_scan(lane == 0 ? n_eq : 0, scan_s, tot_eq);          // per-warp values on lane 0
+  const int w_pre_eq = __shfl_sync(0xffffffffu, pre_eq, 0);
+  const int take_eq = max(0, min(n_eq, my_eq - w_pre_eq));                           // equals are taken in index order
+  const int pre_sel = block_excl_scan(lane == 0 ? n_gt + take_eq : 0, scan_s, tot_sel);
+  int out = out_base + __shfl_sync(0xffffffffu, pre_sel, 0), eq_seen = 0;
+  for (int i0 = w_lo; i0 < w_hi; i0 += 32) {
+    const int i = i0 + lane;
+    const uint32_t k = i < w_hi ? skey[i] : 0u;
+    const uint32_t m_eq = __ballot_sync(0xffffffffu, i < w_hi && k == T);
+    const int my_eq_rank = eq_seen + __popc(m_eq & ((1u << lane) - 1u));
+    const bool take = i < w_hi && (k > T || (k == T && my_eq_rank < take_eq));
+    const uint32_t m_take = __ballot_sync(0xffffffffu, take);
+    if (take) sink_idx[out + __popc(m_take & ((1u << lane) - 1u))] = lo + c_lo + i;
+    out += __popc(m_take);
+    eq_seen += __popc(m_eq);
+  }
+  for (int i = want + (int)rank * SC_THREADS + tid; i < n_sink; i += SC_CTAS * SC_THREADS) sink_idx[i] = -1;
+  sc_sync();                                            // nobody leaves while its shared memory may still be read
+}
+
 focus_status launch_sink_select(focus_ctx* ctx, const float* part, int H, int L, const int32_t* n_active, float* S,
                                 int cand_lo, int cand_hi, int n_sink, int32_t* sink_idx, cudaStream_t st) {
   sink_reduce_heads_kernel<<<(L + 255) / 256, 256, 0, st>>>(part, H, L, n_active, S);
   FOCUS_CHECK_LAUNCH();
   const int n = cand_hi - cand_lo;
+  const int chunk = (n + SC_CTAS - 1) / SC_CTAS;
+  static int cluster_ok = -1;                         // -1 not tried, 1 works, 0 the cluster launch was refused once
+  // the cluster pays for its barriers (about 1.5 us each, seven to eight of them) once a single CTA's sweeps over
+  // all keys cost more: measured cross-over between 8K and 16K candidates
+  if (n >= 12288 && chunk <= SC_MAX_KEYS && cluster_ok != 0) {
+    static bool attr_set = false;
+    if (!attr_set) {
+      if (cudaFuncSetAttribute(sink_select_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               SC_MAX_KEYS * 4) != cudaSuccess)
+        return FOCUS_ERR_CUDA;
+      attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(SC_CTAS, 1, 1); cfg.blockDim = dim3(SC_THREADS, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)chunk * 4; cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = SC_CTAS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, sink_select_cluster_kernel, (const float*)S, n_active, cand_lo, cand_hi, n_sink, sink_idx,
+                           ctx->d_status) == cudaSuccess) {
+      cluster_ok = 1;
+      FOCUS_CHECK_LAUNCH();
+      return FOCUS_OK;
+    }
+    cudaGetLastError();
+    cluster_ok = 0;                                   // fall through to the one-CTA kernels
+  }
   if (n <= TN_MAX_SMEM_KEYS) {
     static bool attr_set = false;
     if (!attr_set) {
