@@ -443,6 +443,49 @@ def test_host_side_argument_matrix(ctx):
     tiny.close()
 
 
+@pytest.mark.parametrize("case", ["all_equal", "duplicated_keys", "random"])
+def test_sink_selection_on_a_long_candidate_range(ctx, case):
+    """A candidate range long enough for the multi-CTA selection (16 000 prompt positions).  The selected set must be
+    exactly the n_sink largest of the scores the library itself reports, equal scores taken in index order
+    ("all_equal": Q = 0, every score is 1/L, the set is the first n_sink positions; "duplicated_keys": every score
+    value occurs four times or more, so the threshold cuts a run of equal scores), and agree with the oracle outside
+    the near-threshold band."""
+    L, M, H, d, n_sink, n_act = 16384, 16000, 2, 128, 161, 24
+    s = wl.Shape(L, M, H, H, d, 128, "bf16")
+    rng = np.random.default_rng(11)
+    K = rng.standard_normal((H, L, d)).astype(np.float32) / math.sqrt(d)
+    if case == "duplicated_keys":
+        K = K[:, np.arange(L) % 4000]
+    Qf = rng.standard_normal((s.N, H, d)).astype(np.float32) / math.sqrt(d)
+    if case == "all_equal":
+        Qf[:] = 0.0
+    Qs, Ks = wl.to_storage(Qf, "bf16"), wl.to_storage(np.ascontiguousarray(K), "bf16")
+    dQ, dK = fstep.to_device(Qs, "bf16"), fstep.to_device(Ks, "bf16")
+    active = np.sort(rng.choice(np.arange(M, L), size=n_act, replace=False)).astype(np.int32)
+    d_active = torch.from_numpy(active).cuda()
+    d_nact = torch.tensor([n_act], dtype=torch.int32, device="cuda")
+    sink_idx = torch.full((n_sink,), -7, dtype=torch.int32, device="cuda")
+    scores = torch.zeros(L, dtype=torch.float32, device="cuda")
+    fb.focus_find_sinks(ctx, fstep.c_shape(s), dQ, M, d_active, d_nact, n_act, dK, None, n_sink, 0, M, sink_idx, scores)
+    assert ctx.poll_status() == 0
+    got = sink_idx.cpu().numpy()
+    sc = scores.cpu().numpy()
+    # exact selection on the library's own float32 scores, ties to the lower index
+    order = np.argsort(-sc[:M].astype(np.float64), kind="stable")[:n_sink]
+    assert np.array_equal(got, np.sort(order))
+    if case == "all_equal":
+        assert np.array_equal(got, np.arange(n_sink))
+    if case == "duplicated_keys":
+        tau = sc[got].min()
+        assert (sc[:M] == tau).sum() > (sc[got] == tau).sum() >= 1, "the threshold was meant to cut a run of equal scores"
+    # oracle parity outside the band
+    Q64, K64 = wl.storage_to_f64(Qs, "bf16"), wl.storage_to_f64(Ks, "bf16")
+    S = fo.sink_scores(Q64[active - M], K64, 1.0 / math.sqrt(d))
+    ref = fo.find_sinks(S, n_sink, 0, M)
+    assert np.max(np.abs(sc - S)) <= 2e-3 * np.max(S)
+    check_topk_band(got, ref, S, range(M), 1e-3, what="sink_idx")
+
+
 def test_results_are_deterministic(ctx):
     w = small_workload("bf16", 128, 128, H=8, Hkv=2)
     host, dev = make_inputs(w)
