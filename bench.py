@@ -271,7 +271,8 @@ def run_focus(args):
         return tot / steps, launches, marks
 
     K, W = args.steps, max(args.warmup, 3)
-    # eager pass with CUDA-event marks around every attention call: per-kernel durations for the roofline
+    # eager pass with CUDA-event marks around every attention call (per-call durations; the roofline uses them only
+    # with --no-graph, otherwise the per-launch average of a graph of those launches, see below)
     ms_eager, launches, marks = timed(lambda m: step("active", marks=m), K, W, with_marks=True)
     assert ctx.poll_status() == 0, "device status word set during the timed region"
     # the same step captured once into a CUDA graph (counts stay on the device, so nothing needs the host)
@@ -300,15 +301,46 @@ def run_focus(args):
 
     dense_t = [a.elapsed_time(z) for kind, a, z in marks if kind == "dense"]
     sparse_t = [a.elapsed_time(z) for kind, a, z in marks if kind == "sparse"]
+    # The dominant kernel in the launch mode of the headline number: the dense-attention launches of one step (each on
+    # its own layer's K/V, 537 MB apiece) captured alone into a graph; average time per launch over K replays,
+    # gaps between the launches included.
+    dense_graph_ms = sparse_graph_ms = None
+    if graph is not None:
+        b_act = results["active"]["b"]
+
+        def dense_run():
+            for l in range(probe + 1):
+                fstep.dense_layer(ctx, b_act, Qs[l], Ks[l], Vs[l], O=results["active"]["O"][l])
+        dense_run()
+        torch.cuda.synchronize()
+        dgraph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(dgraph):
+            dense_run()
+        ms_dg, _, _ = timed(lambda m: dgraph.replay(), K, W)
+        dense_graph_ms = ms_dg / (probe + 1)
+
+        def sparse_run():                                  # the sparse layers of a step, sink set from the last step
+            for l in range(probe + 1, NL):
+                fstep.sparse_layer(ctx, b_act, Qs[l], Ks[l], Vs[l], Kbar=Kbars[l], O=results["active"]["O"][l])
+        if NL > probe + 1:
+            sparse_run()
+            torch.cuda.synchronize()
+            sgraph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(sgraph):
+                sparse_run()
+            ms_sg, _, _ = timed(lambda m: sgraph.replay(), K, W)
+            sparse_graph_ms = ms_sg / (NL - probe - 1)
     eb = 2
     kv_bytes = 2 * s.Hkv * s.L * s.d * eb
     na = int(results["active"]["b"].n_active.item())
     qo_bytes = 2 * na * s.H * s.d * eb
-    dense_ms = float(np.mean(dense_t))
+    dense_eager_ms = float(np.mean(dense_t))
+    dense_ms = dense_graph_ms if dense_graph_ms is not None else dense_eager_ms
     dense_gbs = (kv_bytes + qo_bytes) / (dense_ms * 1e-3) / 1e9
     retained_keys = w.C * s.B + w.n_sink + s.N                      # upper bound per head (sinks inside blocks are skipped)
     sparse_bytes = 2 * s.Hkv * retained_keys * s.d * eb + qo_bytes
-    sparse_ms = float(np.mean(sparse_t)) if sparse_t else float("nan")
+    sparse_eager_ms = float(np.mean(sparse_t)) if sparse_t else float("nan")
+    sparse_ms = sparse_graph_ms if sparse_graph_ms is not None else sparse_eager_ms
 
     # ---- own dense baseline (every layer dense), cold pooled keys, gen-region rows -----------------------
     ms_dense_step, _, _ = timed(lambda m: step("active", dense_only=True), max(2, K // 4), 2)
@@ -384,7 +416,9 @@ def run_focus(args):
         "stages": {"dense_layer_ms": dense_ms, "dense_layer_GBps": dense_gbs, "sparse_layer_ms": sparse_ms,
                    "sparse_layer_GBps": sparse_bytes / (sparse_ms * 1e-3) / 1e9,
                    "sparse_layer_frac_of_hbm": sparse_bytes / (sparse_ms * 1e-3) / 1e9 / P["hbm"],
-                   "per_layer_sparse_vs_dense": dense_ms / sparse_ms},
+                   "per_layer_sparse_vs_dense": dense_ms / sparse_ms,
+                   "timing": "average per launch of a graph holding only those launches" if graph is not None else "CUDA-event marks around eager calls",
+                   "dense_layer_eager_marks_ms": dense_eager_ms, "sparse_layer_eager_marks_ms": sparse_eager_ms},
         "roofline": {"bound": "hbm", "achieved": dense_gbs, "peak": P["hbm"], "unit": "GB/s", "frac": dense_gbs / P["hbm"],
                      "traffic": traffic, "kernel": "attn_tc_kernel incl. its in-cluster split merge (dense layer, I_active rows)",
                      "bytes_per_launch": kv_bytes + qo_bytes, "peak_source": f"{P['src']} copy bandwidth"},
