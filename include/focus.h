@@ -18,6 +18,12 @@
  *     returns without synchronising.  Nothing is allocated after focus_create: scratch comes from the
  *     context's workspace (FOCUS_ERR_WORKSPACE_TOO_SMALL if it does not fit).  Calls on one context
  *     must be issued on one stream at a time (they share the workspace).
+ *   - Stream order.  The attention kernels and the selection kernel of focus_sparse_layer are launched with
+ *     programmatic stream serialization and let their successor in the stream begin early; each of them waits
+ *     for its predecessor to complete before it writes anything, and before it reads anything that another of
+ *     these kernels may have written (outputs, lists, workspace).  Caller-visible ordering is plain stream
+ *     order: a kernel of another library placed before or after a call sees complete results, and inputs
+ *     produced on the same stream before a call are complete when the call's kernels read them.
  *   - Results are deterministic run to run (fixed reduction order, no floating-point atomics).
  *   - A device-side anomaly (index out of range, a bounded wait that ran out) never traps: the kernel
  *     skips the access, records a code in the context's device status word and returns; read it with
