@@ -493,6 +493,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     if (q & 1) { isV = false; return (q + 1) >> 1; }
     isV = true; return (q >> 1) - 1;
   };
+  const uint64_t l2_pol = l2_policy_evict_first();
   auto issue = [&](int q) {
     bool isV;
     const int idx = seq_tile(q, isV);
@@ -501,8 +502,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     const CUtensorMap* map = ti.kind ? (isV ? &tmSV : &tmSK) : (isV ? &tmV : &tmK);
     const uint32_t dst = sSlot + slot * SLOT_BYTES;
     mbar_expect_tx(bar_full(slot), SLOT_BYTES);
-    tma_load_3d(dst, map, bar_full(slot), 0, ti.start, g);
-    tma_load_3d(dst + HALF_BYTES, map, bar_full(slot), 64, ti.start, g);
+    tma_load_3d_hint(dst, map, bar_full(slot), 0, ti.start, g, l2_pol);
+    tma_load_3d_hint(dst + HALF_BYTES, map, bar_full(slot), 64, ti.start, g, l2_pol);
   };
   const int n_loads = 2 * nt;
   const int n_early = n_loads < NSLOT ? n_loads : NSLOT;
@@ -876,6 +877,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   }
 
   // load sequence: q even -> K_(q/2), q odd -> V_(q/2); the MMA warp consumes K0, V0, K1, V1, ... in this order
+  const uint64_t l2_pol = l2_policy_evict_first();
   auto issue = [&](int q) {
     const bool isV = q & 1;
     const TileInfo ti = get_tile(q >> 1);
@@ -883,8 +885,8 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const CUtensorMap* map = ti.kind ? (isV ? &tmSV : &tmSK) : (isV ? &tmV : &tmK);
     const uint32_t dst = sSlot + slot * SLOT_BYTES;
     mbar_expect_tx(bar_full(slot), SLOT_BYTES);
-    tma_load_3d(dst, map, bar_full(slot), 0, ti.start, g);
-    tma_load_3d(dst + HALF_BYTES, map, bar_full(slot), 64, ti.start, g);
+    tma_load_3d_hint(dst, map, bar_full(slot), 0, ti.start, g, l2_pol);
+    tma_load_3d_hint(dst + HALF_BYTES, map, bar_full(slot), 64, ti.start, g, l2_pol);
   };
   const int n_loads = 2 * nt;
   const int n_early = n_loads < NSLOT_W ? n_loads : NSLOT_W;

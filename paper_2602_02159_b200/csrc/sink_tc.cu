@@ -134,6 +134,7 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
       int issued = 0;
       bool ok = true;
       // tile t of head g; ring slot and phase follow the tile counter without divisions
+      const uint64_t l2_pol = l2_policy_evict_first();      // K streams through once: do not keep it in L2
       int t = u0 % T, g = u0 / T, kvh = g / p.kv_div, slot = 0;
       uint32_t ph = 0;
       for (int i = 0; i < nt && ok; ++i) {
@@ -142,8 +143,8 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
         TL_ITER(0, 0, i, 1);
         const uint32_t dst = sSlot + slot * SLOT_BYTES;
         mbar_expect_tx(bar_full(slot), SLOT_BYTES);
-        tma_load_3d(dst, &tmK, bar_full(slot), 0, t * TK, kvh);
-        tma_load_3d(dst + HALF_BYTES, &tmK, bar_full(slot), 64, t * TK, kvh);
+        tma_load_3d_hint(dst, &tmK, bar_full(slot), 0, t * TK, kvh, l2_pol);
+        tma_load_3d_hint(dst + HALF_BYTES, &tmK, bar_full(slot), 64, t * TK, kvh, l2_pol);
         ++issued;
         if (++slot == p.n_slots) { slot = 0; ph ^= 1u; }
         if (++t == T) { t = 0; ++g; kvh = g / p.kv_div; }
