@@ -1,20 +1,25 @@
 // Block-sparse / dense bidirectional attention on the 5th-generation tensor cores (Eq. 9; FullAttn of
 // Algorithm 1).  bf16 inputs, head_dim 128, fp32 accumulation in TMEM.
 //
-// One CTA = one 128-row query tile of one KV head (GQA: the rows of all query heads of the group are
-// stacked, so every K/V tile is read once per group) x one contiguous range ("split") of that head's key
-// tiles.  Key tiles are 128 keys wide and are enumerated on the fly from the selected block list, the
-// gathered sink tokens and the response region; K/V tiles arrive by TMA through a six-slot ring.
+// attn_tc_kernel: one CTA = one 128-row query tile of one KV head (GQA: the rows of all query heads of the group
+// are stacked, so every K/V tile is read once per group) x one contiguous range ("split") of that head's key
+// tiles.  Key tiles are 128 keys wide and are enumerated from the selected block list, the gathered sink tokens
+// and the response region; K/V tiles arrive by TMA through a six-slot ring.
 //
 // Warp roles (192 threads):
-//   warp 0        TMA producer (one lane): K_j, V_{j-1}, K_{j+1}, ... in the order the MMA warp consumes them
-//   warp 1        tcgen05.mma issuer (one lane) + TMEM allocation: S_b = Q K_j^T (b = j mod 2), O += P_j V_j
-//   warps 2..5    online softmax, one query row per thread: S_b -> registers, exp2, bf16 P back into TMEM
-//                 (aliasing S_b), lazy rescale of O, final normalisation and the epilogue
-// Split partials (unnormalised O, running max, running sum) go to scratch and are merged by a second kernel in
-// fixed split order, so results are deterministic.
-#include <stdlib.h>
-
+//   warp 0        TMA producer (one lane): K0, K1, V0, K2, V1, ... in the order the MMA warp consumes them
+//   warp 1        tcgen05.mma issuer (one lane) + TMEM allocation: S_b = Q K_j^T (b = j mod 2), O += P_j V_j in two
+//                 halves of 64 keys
+//   warps 2..5    online softmax, one query row per thread: S_b -> registers, exp2 in chunks of 32 keys, bf16 P back
+//                 into TMEM (aliasing S_b) and handed over half by half, lazy rescale of O, final normalisation
+// The splits of a query tile form a thread-block cluster and merge their partials (unnormalised O, running max,
+// running sum) through distributed shared memory in fixed split order; when the clusters of a launch would not all
+// be resident, partials go through global memory instead (last-arriving CTA or a second kernel merges).  Results
+// are deterministic either way.
+//
+// attn_tc_wide_kernel (further down): two query tiles per CTA for the tensor-bound regime.
+//
+// Every launch is a programmatic dependent launch: see the comment on p.pdl in attn_tc_kernel.
 #include <stdio.h>
 #include <stdlib.h>
 

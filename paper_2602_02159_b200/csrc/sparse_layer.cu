@@ -1,6 +1,7 @@
-// One sparse layer in three launches (Algorithm 1, sparse branch): a fused selection kernel (block relevance
-// against the cached pooled keys, Top-C, sink keep flags, sink row gather), the block-sparse attention kernel
-// and the split merge.  The stand-alone entry points compute the same quantities one launch per stage.
+// One sparse layer in two launches (Algorithm 1, sparse branch): a fused selection kernel (block relevance against
+// the cached pooled keys, Top-C, sink keep flags, column mask, sink row gather) and the block-sparse attention
+// kernel (split merge included), chained by programmatic dependent launch.  The stand-alone entry points compute
+// the same quantities one launch per stage.
 #include "focus_common.cuh"
 
 constexpr int FS_THREADS = 1024;
