@@ -500,3 +500,59 @@ def test_results_are_deterministic(ctx):
         outs.append([t.clone() for t in (b.sink_idx, b.sink_scores, b.R, b.block_idx, b.O.view(torch.int16), b.lse)])
     for a, c in zip(*outs):
         assert torch.equal(a, c)
+
+
+@pytest.mark.parametrize("rows", ["active", "gen"])
+def test_step_replayed_from_a_cuda_graph_matches_eager_calls(ctx, rows):
+    """The benchmark times a step as one CUDA-graph replay (counts stay on the device, the kernels are chained by
+    programmatic dependent launch).  A small step -- two dense layers, sink identification, three sparse layers with
+    cached pooled keys -- captured into a graph must reproduce the eager calls bit for bit, replay after replay."""
+    w = small_workload("bf16", 128, 128, H=8, Hkv=2, L=2600, M=2100, n_sink=21, C=5)
+    host, dev = make_inputs(w)
+    s = w.shape
+    Kbar = torch.zeros(s.Hkv, s.nb, s.d, dtype=torch.float32, device="cuda")
+    b0 = fstep.StepBuffers(w, rows=rows)
+    fb.focus_pool_keys(ctx, b0.shape, dev["K"], Kbar)
+    n_layers = 5
+
+    def step(b, outs):
+        fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
+        for l in range(2):
+            fstep.dense_layer(ctx, b, dev["Q"], dev["K"], dev["V"], O=outs[l])
+        if rows == "active":
+            fstep.find_sinks(ctx, b, dev["Q"], dev["K"], b.lse)
+        else:
+            fstep.find_sinks(ctx, b, dev["Q"], dev["K"], None)
+        for l in range(2, n_layers):
+            fstep.sparse_layer(ctx, b, dev["Q"], dev["K"], dev["V"], Kbar=Kbar, O=outs[l])
+
+    def fresh():
+        b = fstep.StepBuffers(w, rows=rows)
+        outs = [torch.zeros_like(b.O) for _ in range(n_layers)]
+        return b, outs
+
+    b_e, o_e = fresh()
+    step(b_e, o_e)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    b_g, o_g = fresh()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step(b_g, o_g)                                   # warm-up outside the capture (attributes, lazy set-up)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step(b_g, o_g)
+    for _ in range(3):
+        for t in o_g:
+            t.zero_()
+        b_g.sink_idx.fill_(-5); b_g.block_idx.fill_(-5)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        for a, c in zip(o_e, o_g):
+            assert torch.equal(a.view(torch.int16), c.view(torch.int16))
+        for name in ("sink_idx", "sink_scores", "block_idx", "block_cnt", "R", "lse", "active_idx", "focus_idx"):
+            assert torch.equal(getattr(b_e, name), getattr(b_g, name)), name
