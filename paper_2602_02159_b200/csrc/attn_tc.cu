@@ -1367,7 +1367,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   const int ns_pad = a.dense ? 0 : (a.n_sink + TN - 1) / TN * TN;
   const int n_resp = a.dense ? (sh.L + TN - 1) / TN : (sh.L - sh.M + TN - 1) / TN;
   const int max_tiles = a.dense ? n_resp : a.max_blocks + ns_pad / TN + n_resp;
-  static bool attr_set = false;
+  bool& attr_set = ctx->ls.attn_attr_set;
   if (!attr_set) {
     if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
         cudaFuncSetAttribute(attn_tc_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES_W) != cudaSuccess)
@@ -1377,8 +1377,8 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   // resident-cluster capacity per cluster size (-1 = not asked yet): a launch whose clusters do not all fit at once
   // would run in two waves, so such launches fall back to the merge through global memory (narrow kernel) or to
   // the narrow kernel (wide kernel)
-  static int cluster_cap[9] = {-1, -1, -1, -1, -1, -1, -1, -1, -1};
-  static int cluster_cap_w[9] = {-1, -1, -1, -1, -1, -1, -1, -1, -1};
+  int* cluster_cap = ctx->ls.cluster_cap;          // stored as capacity + 1: 0 means "not asked yet"
+  int* cluster_cap_w = ctx->ls.cluster_cap_w;
   // two query tiles per CTA when a KV head has at least 256 stacked rows (tensor-bound regime)
   bool wide = stacked >= TMW && !ctx->no_wide;
   int n_mtiles = 0, base = 0, n_splits = 1;
@@ -1387,9 +1387,9 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     base = n_mtiles * Hkv;
     n_splits = pick_splits(ctx, base, max_tiles);
     if (n_splits > 1) {
-      if (cluster_cap_w[n_splits] < 0)
-        cluster_cap_w[n_splits] = cluster_capacity(attn_tc_wide_kernel, n_splits, NTHREADS_W, SMEM_BYTES_W);
-      if (cluster_cap_w[n_splits] < base) wide = false;               // its splits merge through a cluster only
+      if (cluster_cap_w[n_splits] == 0)
+        cluster_cap_w[n_splits] = cluster_capacity(attn_tc_wide_kernel, n_splits, NTHREADS_W, SMEM_BYTES_W) + 1;
+      if (cluster_cap_w[n_splits] - 1 < base) wide = false;           // its splits merge through a cluster only
     }
     // it pays on long key streams (measured: +6 % on dense 32K); with a few dozen tiles per CTA the one-tile kernel
     // without a key split is faster
@@ -1417,8 +1417,8 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     // the largest split count (not above the one wanted) whose clusters are all resident at once; if even two-CTA
     // clusters do not fit, keep the wanted count and merge through global memory
     for (int sp = n_splits; sp >= 2; --sp) {
-      if (cluster_cap[sp] < 0) cluster_cap[sp] = cluster_capacity(attn_tc_kernel, sp, NTHREADS, SMEM_BYTES);
-      if (cluster_cap[sp] >= base) { n_splits = sp; use_cluster = true; break; }
+      if (cluster_cap[sp] == 0) cluster_cap[sp] = cluster_capacity(attn_tc_kernel, sp, NTHREADS, SMEM_BYTES) + 1;
+      if (cluster_cap[sp] - 1 >= base) { n_splits = sp; use_cluster = true; break; }
     }
     if (getenv("FOCUS_LOG")) fprintf(stderr, "[focus] attn: base %d splits %d cluster %d\n", base, n_splits, (int)use_cluster);
   }

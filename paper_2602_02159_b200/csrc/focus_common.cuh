@@ -19,6 +19,14 @@ struct focus_ctx {
   int no_pdl;          // 1: never launch the attention kernel as a programmatic dependent (A/B comparisons)
   int no_wide;         // 1: never use the two-query-tile attention kernel (A/B comparisons)
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime (no libcuda link)
+  // launch state that belongs to the device (function attributes, occupancy answers): kept per context, since a
+  // process may hold contexts on several devices.  Zero-initialised by focus_create.
+  struct LaunchState {
+    bool attn_attr_set, select_attr_set, topn_attr_set;
+    int sink_attr_smem;
+    int cluster_cap[9], cluster_cap_w[9];      // co-resident clusters per cluster size, value + 1 (0 = not asked yet)
+    int select_cluster;                        // 0 not tried, 1 works, 2 the cluster launch was refused once
+  } ls;
 };
 
 constexpr int FOCUS_N_COUNTERS = 4096;

@@ -529,11 +529,11 @@ focus_status launch_sink_select(focus_ctx* ctx, const float* part, int H, int L,
   FOCUS_CHECK_LAUNCH();
   const int n = cand_hi - cand_lo;
   const int chunk = (n + SC_CTAS - 1) / SC_CTAS;
-  static int cluster_ok = -1;                         // -1 not tried, 1 works, 0 the cluster launch was refused once
+  int& cluster_state = ctx->ls.select_cluster;        // 0 not tried, 1 works, 2 the cluster launch was refused once
   // the cluster pays for its barriers (about 1.5 us each, seven to eight of them) once a single CTA's sweeps over
   // all keys cost more: measured cross-over between 8K and 16K candidates
-  if (n >= 12288 && chunk <= SC_MAX_KEYS && cluster_ok != 0) {
-    static bool attr_set = false;
+  if (n >= 12288 && chunk <= SC_MAX_KEYS && cluster_state != 2) {
+    bool& attr_set = ctx->ls.select_attr_set;
     if (!attr_set) {
       if (cudaFuncSetAttribute(sink_select_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                SC_MAX_KEYS * 4) != cudaSuccess)
@@ -549,15 +549,15 @@ focus_status launch_sink_select(focus_ctx* ctx, const float* part, int H, int L,
     cfg.attrs = at; cfg.numAttrs = 1;
     if (cudaLaunchKernelEx(&cfg, sink_select_cluster_kernel, (const float*)S, n_active, cand_lo, cand_hi, n_sink, sink_idx,
                            ctx->d_status) == cudaSuccess) {
-      cluster_ok = 1;
+      cluster_state = 1;
       FOCUS_CHECK_LAUNCH();
       return FOCUS_OK;
     }
     cudaGetLastError();
-    cluster_ok = 0;                                   // fall through to the one-CTA kernels
+    cluster_state = 2;                                // fall through to the one-CTA kernels
   }
   if (n <= TN_MAX_SMEM_KEYS) {
-    static bool attr_set = false;
+    bool& attr_set = ctx->ls.topn_attr_set;
     if (!attr_set) {
       if (cudaFuncSetAttribute(sink_topn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                TN_MAX_SMEM_KEYS * 4) != cudaSuccess)

@@ -320,7 +320,7 @@ focus_status launch_sink_colsum_tc(focus_ctx* ctx, const focus_shape* s, const v
   const int hs = p.groups_staged * hpg;
   const int smem = 1024 + hs * p.n_pad * 256 + p.n_slots * SLOT_BYTES + (2 * MAX_SLOTS + 2 * MAX_BUF) * 8 + 16 +
                    hs * p.n_pad * 4 + 64;
-  static int attr_smem = 0;
+  int& attr_smem = ctx->ls.sink_attr_smem;
   if (smem > attr_smem) {
     if (cudaFuncSetAttribute(sink_colsum_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
       return FOCUS_ERR_CUDA;
