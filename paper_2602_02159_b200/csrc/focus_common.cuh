@@ -122,6 +122,69 @@ __device__ __forceinline__ int block_excl_scan(int v, int* warp_tot, int& total)
 #endif
 
 // ---- internal launchers (defined in the .cu files) -------------------------------------------
+// Marks in sel[0..n) the C largest of the order-preserving keys key[0..n) (shared memory), equal keys taken in index
+// order: the key T of the C-th largest element is found by an 8-bit radix descent (four 256-bin histograms), then
+// keys > T are marked and keys == T in index order until the quota is filled.  Work per thread is O(n / threads)
+// per pass, against O(n) for rank-by-counting.  Called by every thread of the block; hist: 258 ints, scan_s: 33 ints
+// of shared memory.  Ends with a barrier (sel is ready to read).
+__device__ __forceinline__ void block_topc_mark(const uint32_t* key, int n, int C, uint8_t* sel, int* hist, int* scan_s) {
+  const int tid = threadIdx.x, nth = blockDim.x, lane = tid & 31;
+  if (C >= n || C <= 0) {
+    for (int i = tid; i < n; i += nth) sel[i] = C >= n ? 1 : 0;
+    __syncthreads();
+    return;
+  }
+  uint32_t prefix = 0u, mask = 0u;
+  int need = C;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = tid; i < 256; i += nth) hist[i] = 0;
+    __syncthreads();
+    for (int i = tid; i < n; i += nth) {
+      const uint32_t k = key[i];
+      if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1);
+    }
+    __syncthreads();
+    if (tid < 32) {
+      // digits from the largest down: the first one whose cumulative count reaches `need`
+      int run = 0, found = -1, above = 0;
+      for (int base = 255; base >= 0 && found < 0; base -= 32) {
+        const int c = hist[base - lane];                // lane 0 holds the largest digit of this group of 32
+        int inc = c;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const int y = __shfl_up_sync(0xffffffffu, inc, off);
+          if (lane >= off) inc += y;
+        }
+        const uint32_t hit = __ballot_sync(0xffffffffu, run + inc >= need);
+        if (hit) {
+          const int l0 = __ffs(hit) - 1;
+          found = base - l0;
+          above = run + __shfl_sync(0xffffffffu, inc - c, l0);
+        }
+        run += __shfl_sync(0xffffffffu, inc, 31);
+      }
+      if (lane == 0) { hist[256] = found; hist[257] = above; }
+    }
+    __syncthreads();
+    prefix |= (uint32_t)hist[256] << shift;
+    mask |= 0xFFu << shift;
+    need -= hist[257];
+    __syncthreads();
+  }
+  // prefix = T; need = how many keys equal to T are taken, lowest index first
+  int eq_base = 0;
+  for (int c0 = 0; c0 < n; c0 += nth) {
+    const int i = c0 + tid;
+    const uint32_t k = i < n ? key[i] : 0u;
+    const int eq = (i < n && k == prefix) ? 1 : 0;
+    int tot;
+    const int pre = block_excl_scan(eq, scan_s, tot);
+    if (i < n) sel[i] = (k > prefix || (eq && eq_base + pre < need)) ? 1 : 0;
+    eq_base += tot;
+  }
+  __syncthreads();
+}
+
 struct AttnArgs {
   focus_shape sh;
   float scale;

@@ -105,20 +105,25 @@ select_blocks_kernel(const float* __restrict__ R, int nb, int C, int B, const in
   __shared__ uint32_t key[SB_MAX_NB];
   __shared__ uint8_t sel[SB_MAX_NB];
   __shared__ int scan_s[33];
+  __shared__ int hist[258];
   const int g = blockIdx.x, tid = threadIdx.x;
   const float* Rg = R + (size_t)g * nb;
   for (int i = tid; i < nb; i += SB_THREADS) key[i] = float_key(Rg[i]);
   __syncthreads();
-  for (int i = tid; i < nb; i += SB_THREADS) {
-    const uint32_t ki = key[i];
-    int rank = 0;
-    for (int j = 0; j < nb; ++j) {
-      const uint32_t kj = key[j];
-      rank += (kj > ki || (kj == ki && j < i)) ? 1 : 0;
+  if (nb <= 256) {                                   // few blocks: rank by counting, one pass, no histogram
+    for (int i = tid; i < nb; i += SB_THREADS) {
+      const uint32_t ki = key[i];
+      int rank = 0;
+      for (int j = 0; j < nb; ++j) {
+        const uint32_t kj = key[j];
+        rank += (kj > ki || (kj == ki && j < i)) ? 1 : 0;
+      }
+      sel[i] = rank < C;
     }
-    sel[i] = rank < C;
+    __syncthreads();
+  } else {
+    block_topc_mark(key, nb, C, sel, hist, scan_s);
   }
-  __syncthreads();
   for (int s = tid; s < n_sink; s += SB_THREADS) {
     const int j = sink_idx[s];
     const int b = j / B;

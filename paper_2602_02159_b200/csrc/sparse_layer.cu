@@ -58,6 +58,7 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
   __shared__ float part[8][FS_HD];
   __shared__ float qbar[FS_HD];
   __shared__ int scan_s[33];
+  __shared__ int hist[258];
   const int g = blockIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
   // Issue every load that does not depend on another one first: the kernel is a chain of global-memory
@@ -117,16 +118,20 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
       score(b, __ldg(reinterpret_cast<const float4*>(kb + (size_t)b * FS_HD)));
   }
   __syncthreads();
-  for (int i = tid; i < nb; i += FS_THREADS) {
-    const uint32_t ki = key[i];
-    int rank = 0;
-    for (int j = 0; j < nb; ++j) {
-      const uint32_t kj = key[j];
-      rank += (kj > ki || (kj == ki && j < i)) ? 1 : 0;
+  if (nb <= 256) {                                   // few blocks: rank by counting, one pass, no histogram
+    for (int i = tid; i < nb; i += FS_THREADS) {
+      const uint32_t ki = key[i];
+      int rank = 0;
+      for (int j = 0; j < nb; ++j) {
+        const uint32_t kj = key[j];
+        rank += (kj > ki || (kj == ki && j < i)) ? 1 : 0;
+      }
+      sel[i] = rank < C;
     }
-    sel[i] = rank < C;
+    __syncthreads();
+  } else {
+    block_topc_mark(key, nb, C, sel, hist, scan_s);
   }
-  __syncthreads();
   asm volatile("griddepcontrol.wait;" ::: "memory");
   for (int s = tid; s < ns_pad; s += FS_THREADS) {
     uint8_t keep = 0, mk = 0;

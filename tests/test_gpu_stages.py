@@ -486,6 +486,39 @@ def test_sink_selection_on_a_long_candidate_range(ctx, case):
     check_topk_band(got, ref, S, range(M), 1e-3, what="sink_idx")
 
 
+@pytest.mark.parametrize("nb,C", [(700, 37), (257, 256), (3000, 1), (1022, 31)])
+def test_block_selection_with_many_blocks_and_cut_ties(ctx, nb, C):
+    """Top-C over several hundred to a few thousand blocks (the radix path of the selection kernels), scores
+    quantised so that the threshold cuts a run of equal scores: the set must be the oracle's exactly (float32 scores
+    are given, nothing is recomputed), equal scores taken in block order, and the keep flags must follow it.  Runs the
+    stand-alone stage and, where the pooled keys reproduce the scores, the fused layer's selection."""
+    B, G = 64, 3
+    M = nb * B - 17                                      # short last block
+    s = wl.Shape(M + 192, M, G, G, 64, B, "f32")
+    assert s.nb == nb
+    rng = np.random.default_rng(nb + C)
+    R = rng.integers(0, 23, size=(G, nb)).astype(np.float32) / 7.0 - 1.0     # 23 distinct values, signs mixed
+    R[1, ::5] = -0.0
+    sinks = np.sort(rng.choice(M, size=40, replace=False)).astype(np.int32)
+    blocks, keep = fo.select_blocks(R, C, sinks, B)
+    dR = torch.from_numpy(R.reshape(-1)).cuda()
+    d_sinks = torch.from_numpy(sinks).cuda()
+    bidx = torch.full((G * C,), -9, dtype=torch.int32, device="cuda")
+    bcnt = torch.zeros(G, dtype=torch.int32, device="cuda")
+    skeep = torch.full((G * 40,), 7, dtype=torch.uint8, device="cuda")
+    fb.focus_select_blocks(ctx, fstep.c_shape(s), dR, fb.HEADS_PER_KV_GROUP, C, d_sinks, 40, fb.SINK_TOKENS, bidx, C, bcnt,
+                           skeep)
+    assert ctx.poll_status() == 0
+    got = bidx.cpu().numpy().reshape(G, C)
+    for g in range(G):
+        assert bcnt[g].item() == C
+        assert got[g].tolist() == blocks[g].tolist(), f"group {g}"
+        tau = R[g, blocks[g]].min()
+        if C < nb:
+            assert (R[g] == tau).sum() > (R[g, blocks[g]] == tau).sum() >= 1, "the threshold was meant to cut a tie"
+    assert np.array_equal(skeep.cpu().numpy().reshape(G, 40), keep)
+
+
 def test_results_are_deterministic(ctx):
     w = small_workload("bf16", 128, 128, H=8, Hkv=2)
     host, dev = make_inputs(w)
