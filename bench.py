@@ -407,6 +407,7 @@ def run_focus(args):
                    "pooled_keys": "cached per KV-cache refresh", "l2": "inputs larger than L2 (17 GB of K/V per step)",
                    "multi_gpu": "independent replicas, no data-path collective", "input_gen_s": round(t_gen, 1)},
         "gpu_launches": int(launches),
+        "steps_per_s_all_replicas": world * 1e3 / ms_step,     # the latency metric does not add up over replicas; this does
         "launch_mode": "one CUDA graph replay per step" if graph is not None else "eager C-ABI calls",
         "eager_ms_per_step": ms_eager,
         "clocks": clocks,
