@@ -304,32 +304,31 @@ def run_focus(args):
     # The dominant kernel in the launch mode of the headline number: the dense-attention launches of one step (each on
     # its own layer's K/V, 537 MB apiece) captured alone into a graph; average time per launch over K replays,
     # gaps between the launches included.
+    def per_launch_in_graph(rows, kind, steps):
+        """Average time per launch of the step's dense (or sparse) layers, captured alone into a graph."""
+        r_ = results[rows]
+        layers = range(probe + 1) if kind == "dense" else range(probe + 1, NL)
+        if len(layers) == 0:
+            return None
+
+        def run():
+            for l in layers:
+                if kind == "dense":
+                    fstep.dense_layer(ctx, r_["b"], Qs[l], Ks[l], Vs[l], O=r_["O"][l])
+                else:                                      # sink set from the last full step
+                    fstep.sparse_layer(ctx, r_["b"], Qs[l], Ks[l], Vs[l], Kbar=Kbars[l], O=r_["O"][l])
+        run()
+        torch.cuda.synchronize()
+        g_ = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_):
+            run()
+        ms_, _, _ = timed(lambda m: g_.replay(), steps, W)
+        return ms_ / len(layers)
+
     dense_graph_ms = sparse_graph_ms = None
     if graph is not None:
-        b_act = results["active"]["b"]
-
-        def dense_run():
-            for l in range(probe + 1):
-                fstep.dense_layer(ctx, b_act, Qs[l], Ks[l], Vs[l], O=results["active"]["O"][l])
-        dense_run()
-        torch.cuda.synchronize()
-        dgraph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(dgraph):
-            dense_run()
-        ms_dg, _, _ = timed(lambda m: dgraph.replay(), K, W)
-        dense_graph_ms = ms_dg / (probe + 1)
-
-        def sparse_run():                                  # the sparse layers of a step, sink set from the last step
-            for l in range(probe + 1, NL):
-                fstep.sparse_layer(ctx, b_act, Qs[l], Ks[l], Vs[l], Kbar=Kbars[l], O=results["active"]["O"][l])
-        if NL > probe + 1:
-            sparse_run()
-            torch.cuda.synchronize()
-            sgraph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(sgraph):
-                sparse_run()
-            ms_sg, _, _ = timed(lambda m: sgraph.replay(), K, W)
-            sparse_graph_ms = ms_sg / (NL - probe - 1)
+        dense_graph_ms = per_launch_in_graph("active", "dense", K)
+        sparse_graph_ms = per_launch_in_graph("active", "sparse", K)
     eb = 2
     kv_bytes = 2 * s.Hkv * s.L * s.d * eb
     na = int(results["active"]["b"].n_active.item())
@@ -349,8 +348,12 @@ def run_focus(args):
     if not args.skip_gen:
         ms_gen, _, gm = timed(lambda m: step("gen", marks=m), max(2, K // 4), 2, with_marks=True)
         ms_gen_dense, _, _ = timed(lambda m: step("gen", dense_only=True), 2, 1)
-        gd = float(np.mean([a.elapsed_time(z) for k_, a, z in gm if k_ == "dense"]))
-        gs = float(np.mean([a.elapsed_time(z) for k_, a, z in gm if k_ == "sparse"]))
+        gd_eager = float(np.mean([a.elapsed_time(z) for k_, a, z in gm if k_ == "dense"]))
+        gs_eager = float(np.mean([a.elapsed_time(z) for k_, a, z in gm if k_ == "sparse"]))
+        gd, gs = gd_eager, gs_eager
+        if graph is not None:                              # same launch mode as the paper-row figures
+            gd = per_launch_in_graph("gen", "dense", max(2, K // 4)) or gd_eager
+            gs = per_launch_in_graph("gen", "sparse", max(2, K // 4)) or gs_eager
         fl_dense = 4.0 * s.N * s.L * s.d * s.H
         fl_sparse = 4.0 * s.N * retained_keys * s.d * s.H
         gen = {"rows": s.N, "ms_per_step": ms_gen, "dense_ms_per_step": ms_gen_dense,
@@ -358,6 +361,7 @@ def run_focus(args):
                "dense_layer_ms": gd, "dense_layer_tflops": fl_dense / gd / 1e9,
                "sparse_layer_ms": gs, "sparse_retained_tflops": fl_sparse / gs / 1e9,
                "sparse_dense_equiv_tflops": fl_dense / gs / 1e9,
+               "dense_layer_eager_marks_ms": gd_eager, "sparse_layer_eager_marks_ms": gs_eager,
                "roofline": {"bound": "tensor", "achieved": fl_dense / gd / 1e9, "peak": P["tf_sust"], "unit": "TFLOP/s",
                             "frac": fl_dense / gd / 1e9 / P["tf_sust"], "kernel": "attn_tc_wide_kernel (dense layer, 512 gen rows)",
                             "peak_source": f"{P['src']} sustained bf16"}}
