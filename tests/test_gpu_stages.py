@@ -589,3 +589,35 @@ def test_step_replayed_from_a_cuda_graph_matches_eager_calls(ctx, rows):
             assert torch.equal(a.view(torch.int16), c.view(torch.int16))
         for name in ("sink_idx", "sink_scores", "block_idx", "block_cnt", "R", "lse", "active_idx", "focus_idx"):
             assert torch.equal(getattr(b_e, name), getattr(b_g, name)), name
+
+
+def test_step_with_nothing_left_to_unmask(ctx):
+    """No masked position in the decoding block: I_focus and I_active are empty.  The attention calls have no rows to
+    compute (outputs stay untouched), sink identification and the fused layer report the undefined inputs through
+    the status word instead of reading or writing out of range, and the context stays usable."""
+    w = small_workload("bf16", 128, 128, H=4, Hkv=4)
+    host, dev = make_inputs(w)
+    b = fstep.StepBuffers(w)
+    masked = torch.zeros_like(dev["masked"])
+    fstep.select_queries(ctx, b, dev["conf"], masked)
+    assert b.n_focus.item() == 0 and b.n_active.item() == 0
+    assert (b.focus_idx == -1).all() and (b.active_idx == -1).all()
+    b.O.fill_(3.0); b.lse.fill_(-7.0)
+    fstep.dense_layer(ctx, b, dev["Q"], dev["K"], dev["V"])
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    assert (b.O == 3.0).all() and (b.lse == -7.0).all()
+    fstep.find_sinks(ctx, b, dev["Q"], dev["K"], b.lse)
+    assert ctx.poll_status() == fb.ERR_INVALID_ARG          # scores are undefined without active rows
+    assert (b.sink_idx == -1).all()
+    Kbar = torch.zeros(w.shape.Hkv, w.shape.nb, w.shape.d, dtype=torch.float32, device="cuda")
+    fb.focus_pool_keys(ctx, b.shape, dev["K"], Kbar)
+    fstep.sparse_layer(ctx, b, dev["Q"], dev["K"], dev["V"], Kbar=Kbar)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == fb.ERR_INVALID_ARG          # no focus query to score blocks with
+    assert (b.O == 3.0).all()
+    # the same context still computes a normal step afterwards
+    fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
+    fstep.dense_layer(ctx, b, dev["Q"], dev["K"], dev["V"])
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0 and b.n_active.item() > 0
