@@ -1413,7 +1413,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     }
   }
   bool use_cluster = false;
-  if (n_splits > 1 && !wide) {
+  if (n_splits > 1 && !wide && ctx->merge_mode == 0) {
     // the largest split count (not above the one wanted) whose clusters are all resident at once; if even two-CTA
     // clusters do not fit, keep the wanted count and merge through global memory
     for (int sp = n_splits; sp >= 2; --sp) {
@@ -1456,7 +1456,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.cluster = use_cluster ? 1 : 0;
   // 1: called right after the selection kernel of a fused sparse layer (pre-gathered sinks); 2: predecessor unknown
   p.pdl = ctx->no_pdl ? 0 : ((pre != nullptr && !wide) ? 1 : 2);
-  p.counters = (n_splits > 1 && !use_cluster && !wide && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
+  p.counters = (n_splits > 1 && !use_cluster && !wide && ctx->merge_mode != 2 && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
                    ? ctx->d_counters : nullptr;
   p.q_stride_row = sh.q_stride_row; p.q_stride_head = sh.q_stride_head;
   p.q_base = a.q_base; p.n_q = a.n_q; p.rows_bound = a.max_rows; p.L = sh.L; p.M = sh.M; p.H = sh.n_q_heads;

@@ -4,6 +4,8 @@
 
 #include <new>
 
+#include <string.h>
+
 #include "focus_common.cuh"
 
 focus_status launch_sink_select(focus_ctx* ctx, const float* part, int H, int L, const int32_t* n_active, float* S,
@@ -49,6 +51,10 @@ extern "C" focus_status focus_create(focus_ctx** out, int device, size_t workspa
   c->last_attn_variant = 0;
   c->no_wide = getenv("FOCUS_NO_WIDE") != nullptr;
   c->no_pdl = getenv("FOCUS_NO_PDL") != nullptr;
+  {
+    const char* mm = getenv("FOCUS_MERGE");
+    c->merge_mode = !mm ? 0 : (!strcmp(mm, "counters") ? 1 : (!strcmp(mm, "kernel") ? 2 : 0));
+  }
   c->encode_tiled = nullptr;
   if (prop.major == 10) {   // tensor-core kernels are built for sm_100a only
     cudaDriverEntryPointQueryResult q;

@@ -18,6 +18,8 @@ struct focus_ctx {
   int last_attn_variant;   // 0 none yet, 1 SIMT, 2 tensor-core 128-row tiles, 3 tensor-core 256-row tiles
   int no_pdl;          // 1: never launch the attention kernel as a programmatic dependent (A/B comparisons)
   int no_wide;         // 1: never use the two-query-tile attention kernel (A/B comparisons)
+  int merge_mode;      // split merge of the one-tile kernel: 0 automatic (cluster where it fits), 1 never a cluster (arrival
+                       // counters), 2 neither (separate combine kernel); tests use 1 and 2 to reach the fallbacks
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime (no libcuda link)
   // launch state that belongs to the device (function attributes, occupancy answers): kept per context, since a
   // process may hold contexts on several devices.  Zero-initialised by focus_create.

@@ -621,3 +621,48 @@ def test_step_with_nothing_left_to_unmask(ctx):
     fstep.dense_layer(ctx, b, dev["Q"], dev["K"], dev["V"])
     torch.cuda.synchronize()
     assert ctx.poll_status() == 0 and b.n_active.item() > 0
+
+
+@pytest.mark.parametrize("merge", ["counters", "kernel"])
+def test_split_merge_fallbacks_match_the_default(merge, ctx, monkeypatch):
+    """When the clusters of a launch would not all be resident, the key splits of a query tile are merged through
+    global memory: by the CTA that arrives last at the tile's counter, or by a separate kernel.  Both fallbacks are
+    forced here (a context created with FOCUS_MERGE set) and must agree with the oracle and, to the last bf16 digit
+    or the one next to it, with the default path."""
+    w = small_workload("bf16", 128, 128, H=4, Hkv=2, L=5200, M=4500, n_sink=45, C=9)
+    host, dev = make_inputs(w)
+    monkeypatch.setenv("FOCUS_MERGE", merge)
+    other = fb.Context(0)
+    monkeypatch.delenv("FOCUS_MERGE")
+    try:
+        outs = []
+        for c in (ctx, other):
+            b = fstep.StepBuffers(w)
+            fstep.select_queries(c, b, dev["conf"], dev["masked"])
+            n0 = fb.focus_launch_count()
+            fstep.dense_layer(c, b, dev["Q"], dev["K"], dev["V"])
+            n_launch = fb.focus_launch_count() - n0
+            # one kernel when the merge runs inside the attention kernel, two with the separate combine kernel
+            assert n_launch == (2 if (c is other and merge == "kernel") else 1)
+            dense_O, dense_lse = b.O.clone(), b.lse.clone()
+            fstep.find_sinks(c, b, dev["Q"], dev["K"], b.lse)
+            fstep.sparse_layer(c, b, dev["Q"], dev["K"], dev["V"])
+            torch.cuda.synchronize()
+            assert c.poll_status() == 0
+            outs.append((dense_O, dense_lse, b.O.clone(), b.lse.clone(), b.sink_idx.clone(), b.block_idx.clone(), b))
+        a, o = outs
+        assert torch.equal(a[4], o[4]) and torch.equal(a[5], o[5])
+        for i in (0, 2):
+            assert (a[i].float() - o[i].float()).abs().max().item() <= 2 ** -8 * a[i].float().abs().max().item()
+        for i in (1, 3):
+            assert (a[i] - o[i]).abs().max().item() <= 1e-5
+        # and against the oracle (dense layer, all heads)
+        b = o[6]
+        na = b.n_active.item()
+        act = b.active_idx.cpu().numpy()[:na]
+        Q, K, V = host["Q"], host["K"], host["V"]
+        Od, ld = fo.dense_attn(Q[act - w.shape.M], K, V, 1.0 / math.sqrt(w.shape.d))
+        got = fstep.from_device(o[0])[:na]
+        assert max_abs(got, Od) <= TOL_ABS["bf16"] and rel_rms(got, Od) <= TOL_RMS["bf16"]
+    finally:
+        other.close()
