@@ -104,6 +104,13 @@ int32_t focus_last_attn_variant(focus_ctx* ctx);
  * kernel where supported), 1 = force the generic SIMT kernels.  Returns the previous value. */
 int32_t focus_set_force_simt(focus_ctx* ctx, int32_t force);
 
+/* Self-test of the bounded waits (no counterpart in the paper).  Every wait on a barrier inside the tensor-core
+ * kernels gives up after a time limit, records FOCUS_ERR_TIMEOUT in the status word and lets the kernel unwind
+ * instead of spinning for ever.  This call launches one small CTA that waits, with a limit of limit_us microseconds
+ * (1 .. 100 000), on a barrier nobody ever arrives at: afterwards focus_poll_status must report
+ * FOCUS_ERR_TIMEOUT and the context must still be usable.  Nothing else is touched.  Errors: INVALID_ARG. */
+focus_status focus_selftest_bounded_wait(focus_ctx* ctx, int32_t limit_us, focus_stream stream);
+
 /* ---- stage 1: past-confidence indicator (Eq. 4) and window expansion (Eq. 5) ---------------- */
 
 /* I_focus = the k positions i in [blk_lo, blk_hi) with masked[i] != 0 that have the highest

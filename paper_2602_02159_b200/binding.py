@@ -42,6 +42,7 @@ _SIGS = {
     "focus_poll_status": (_I, [_P, _P, C.POINTER(_I)]),
     "focus_status_string": (C.c_char_p, [_I]),
     "focus_set_force_simt": (_I, [_P, _I]),
+    "focus_selftest_bounded_wait": (_I, [_P, _I, _P]),
     "focus_launch_count": (C.c_uint64, []),
     "focus_last_attn_variant": (_I, [_P]),
     "focus_select_queries": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P, _P, _P, _P, _P]),
@@ -144,6 +145,12 @@ class Context:
 
     def set_force_simt(self, force: bool) -> int:
         return self._lib.focus_set_force_simt(self.handle, 1 if force else 0)
+
+    def selftest_bounded_wait(self, limit_us: int, stream=None) -> None:
+        """One small CTA waits limit_us microseconds on a barrier nobody arrives at, then gives up: poll_status()
+        reports ERR_TIMEOUT afterwards."""
+        _check(self._lib.focus_selftest_bounded_wait(self.handle, int(limit_us), _stream(stream)),
+               "focus_selftest_bounded_wait")
 
 
 def focus_launch_count() -> int:

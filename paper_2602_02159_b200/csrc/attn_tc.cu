@@ -1489,3 +1489,27 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   }
   return FOCUS_OK;
 }
+
+// ---- self-test of the bounded waits -------------------------------------------------------------------------------
+namespace {
+__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(unsigned long long limit_ns, int32_t* status) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    mbar_init(b, 1);
+    abort_flag = 0;
+    fence_barrier_init();
+  }
+  __syncwarp();
+  // nobody arrives: the wait must give up after limit_ns, raise the flag and the status word, and return false
+  mbar_wait(b, 0u, &abort_flag, status, limit_ns);
+}
+}  // namespace
+
+extern "C" focus_status focus_selftest_bounded_wait(focus_ctx* ctx, int32_t limit_us, focus_stream stream) {
+  if (!ctx || limit_us < 1 || limit_us > 100000) return FOCUS_ERR_INVALID_ARG;
+  bounded_wait_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((unsigned long long)limit_us * 1000ull, ctx->d_status);
+  FOCUS_CHECK_LAUNCH();
+  return FOCUS_OK;
+}

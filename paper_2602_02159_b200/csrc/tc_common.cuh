@@ -40,7 +40,8 @@ __device__ __forceinline__ uint64_t global_ns() {
 }
 // Waits for the phase with the given parity to complete.  Gives up after WAIT_LIMIT_NS of wall time or when
 // another thread of the CTA has raised *abort_flag; returns false then (and raises the flag + the status word).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
+                                          uint64_t limit_ns = WAIT_LIMIT_NS) {
   uint64_t t0 = 0;
   for (uint32_t n = 0;; ++n) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -48,7 +49,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       if (*abort_flag) return false;
       const uint64_t now = global_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > WAIT_LIMIT_NS) break;
+      else if (now - t0 > limit_ns) break;
       __nanosleep(32);
     }
   }

@@ -666,3 +666,25 @@ def test_split_merge_fallbacks_match_the_default(merge, ctx, monkeypatch):
         assert max_abs(got, Od) <= TOL_ABS["bf16"] and rel_rms(got, Od) <= TOL_RMS["bf16"]
     finally:
         other.close()
+
+
+def test_a_wait_that_nothing_satisfies_gives_up_and_is_reported(ctx):
+    """Every barrier wait in the tensor-core kernels is bounded.  The library's self-test lets one CTA wait two
+    milliseconds on a barrier nobody arrives at: it must come back (well inside a second), the status word must say
+    TIMEOUT, and the context must go on working."""
+    import time
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    ctx.selftest_bounded_wait(2000)
+    status = ctx.poll_status()                          # synchronises the stream
+    dt = time.perf_counter() - t0
+    assert status == fb.ERR_TIMEOUT
+    assert dt < 1.0
+    assert ctx.poll_status() == 0                       # polled once, cleared
+    w = small_workload("bf16", 128, 128)
+    host, dev = make_inputs(w)
+    b = fstep.StepBuffers(w)
+    fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
+    fstep.dense_layer(ctx, b, dev["Q"], dev["K"], dev["V"])
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0 and b.n_active.item() > 0
