@@ -1391,9 +1391,9 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
         cluster_cap_w[n_splits] = cluster_capacity(attn_tc_wide_kernel, n_splits, NTHREADS_W, SMEM_BYTES_W) + 1;
       if (cluster_cap_w[n_splits] - 1 < base) wide = false;           // its splits merge through a cluster only
     }
-    // it pays on long key streams (measured: +6 % on dense 32K); with a few dozen tiles per CTA the one-tile kernel
-    // without a key split is faster
-    static const int wide_min = getenv("FOCUS_WIDE_MIN") ? atoi(getenv("FOCUS_WIDE_MIN")) : 32;
+    // it pays from about 16 key tiles per CTA upward (measured: 256 us against 316 us on dense 32K with 512 rows,
+    // 47 against 49 us at 8K with 256 rows); below that the one-tile kernel, which needs fewer or no key splits, wins
+    static const int wide_min = getenv("FOCUS_WIDE_MIN") ? atoi(getenv("FOCUS_WIDE_MIN")) : 16;
     if (max_tiles / n_splits < wide_min) wide = false;
   }
   if (!wide) {
