@@ -231,11 +231,7 @@ __device__ __forceinline__ void cluster_merge_items(const TcParams& p, int g, in
       ml[s] = make_float2(0.f, 0.f);
       if (s < S) {
         const uint32_t off = (uint32_t)(PART_ML_OFF + row * 2) * 4u;
-#ifdef MERGE_LOCAL_ONLY
-        ml[s] = ld_smem_f2(spart + off);
-#else
         ml[s] = s == rank ? ld_smem_f2(spart + off) : ld_dsmem_f2(map_to_rank(spart, (uint32_t)s) + off);
-#endif
       }
     }
     float m = -INFINITY;
@@ -264,11 +260,7 @@ __device__ __forceinline__ void cluster_merge_items(const TcParams& p, int g, in
         for (int s = 0; s < SMAX; ++s)
           if (s < S) {
             const uint32_t off = (uint32_t)(row * PROW + (c8 + 8 * (k0 + k)) * 4) * 4u;
-#ifdef MERGE_LOCAL_ONLY
-            o[k][s] = ld_smem_f4(spart + off);
-#else
             o[k][s] = s == rank ? ld_smem_f4(spart + off) : ld_dsmem_f4(map_to_rank(spart, (uint32_t)s) + off);
-#endif
           }
 #pragma unroll
       for (int k = 0; k < KB; ++k) {
