@@ -286,6 +286,34 @@ def test_dense_equals_library_sdpa():
     assert np.allclose(O, ref, rtol=0, atol=1e-13)
 
 
+def test_sparse_equals_library_sdpa_with_a_mask_built_by_hand():
+    """Eq. 9 with a non-trivial key set: per head, the library's attention over all keys with an additive mask that
+    is written out here position by position (selected blocks of the head's group, sink tokens, every response
+    position) must give the oracle's sparse output; the log-sum-exp is checked against scipy on the same logits."""
+    torch = pytest.importorskip("torch")
+    from scipy.special import logsumexp
+    Q, K, V = _small(seed=27, L=61, M=44, H=4, Hkv=2, d=8, n=5)
+    M, B, L, scale = 44, 8, 61, 0.37                     # 6 prompt blocks, the last one 4 tokens long
+    blocks = [np.array([1, 5]), np.array([0, 3, 4])]
+    sinks = np.array([2, 9, 30, 43, 50])                 # 9 lies in block 1 (group 0), 30 in block 3 (group 1); 50 is a response token
+    Os, ls = fo.sparse_attn(Q, K, V, M, B, blocks, sinks, scale)
+    for h in range(4):
+        g = h // 2
+        allowed = np.zeros(L, dtype=bool)
+        for j in range(L):
+            in_block = j < M and (j // B) in set(blocks[g].tolist())
+            allowed[j] = in_block or (j in set(sinks.tolist())) or j >= M
+        assert allowed.sum() == len(fo.key_set(M, L, B, blocks[g], sinks))
+        mask = torch.zeros(5, L, dtype=torch.float64)
+        mask[:, torch.from_numpy(~allowed)] = -float("inf")
+        q = torch.from_numpy(Q[:, h, :])[None]
+        ref = torch.nn.functional.scaled_dot_product_attention(q, torch.from_numpy(K[g])[None], torch.from_numpy(V[g])[None],
+                                                               attn_mask=mask[None], scale=scale)[0].numpy()
+        assert np.allclose(Os[:, h, :], ref, rtol=0, atol=1e-13)
+        logits = scale * Q[:, h, :] @ K[g].T
+        assert np.allclose(ls[h], logsumexp(logits[:, allowed], axis=1), rtol=0, atol=1e-12)
+
+
 def test_keep_ratio_one_is_dense_bit_for_bit():
     Q, K, V = _small(seed=23, L=45, M=37, H=4, Hkv=2, d=8)
     M, B = 37, 8                      # ragged last block (5 tokens)
