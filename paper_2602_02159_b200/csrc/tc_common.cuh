@@ -1,4 +1,4 @@
-// sm_100a building blocks shared by the tensor-core kernels: mbarrier, TMA (no multicast), tcgen05 MMA /
+// sm_100a building blocks shared by the tensor-core kernels: mbarrier, TMA (every copy has one destination CTA), tcgen05 MMA /
 // TMEM load-store wrappers, shared-memory matrix descriptors and bounded waits.
 #pragma once
 
@@ -62,7 +62,7 @@ __device__ __forceinline__ void fence_barrier_init() {
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// ---- TMA: 3-D tiled load global -> shared, completion on an mbarrier (never multicast) -----------
+// ---- TMA: 3-D tiled load global -> shared, completion on an mbarrier; one destination CTA ------
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
