@@ -15,30 +15,53 @@ __global__ void __launch_bounds__(SQ_THREADS)
 select_queries_kernel(const float* __restrict__ conf, const uint8_t* __restrict__ masked, int blk_lo, int blk_hi,
                       int k, int hw, int clip_lo, int clip_hi, int32_t* __restrict__ focus_idx,
                       int32_t* __restrict__ n_focus, int32_t* __restrict__ active_idx, int32_t* __restrict__ n_active) {
-  __shared__ uint32_t key[SQ_MAX_RANGE];     // 0xFFFFFFFF-coded validity lives in `valid`
-  __shared__ uint8_t valid[SQ_MAX_RANGE];
+  __shared__ uint32_t key[SQ_MAX_RANGE];     // small ranges: key of every position; long ranges: keys of the candidates only
+  __shared__ uint16_t cpos[SQ_MAX_RANGE];    // long ranges: position (relative to blk_lo) of the c-th candidate
+  __shared__ uint8_t valid[SQ_MAX_RANGE];    // small ranges: masked flag; long ranges: selection flag of the c-th candidate
   __shared__ uint8_t sel[SQ_MAX_RANGE];
   __shared__ int focus_s[SQ_MAX_K];
   __shared__ int scan_s[33];
+  __shared__ int hist[258];
   const int n = blk_hi - blk_lo;
   const int tid = threadIdx.x;
-  for (int i = tid; i < n; i += SQ_THREADS) {
-    key[i] = float_key(conf[blk_lo + i]);
-    valid[i] = masked[blk_lo + i] != 0;
-  }
-  __syncthreads();
-  for (int i = tid; i < n; i += SQ_THREADS) {
-    int rank = 0;
-    if (valid[i]) {
-      const uint32_t ki = key[i];
-      for (int j = 0; j < n; ++j) {
-        const uint32_t kj = key[j];
-        rank += (valid[j] && (kj > ki || (kj == ki && j < i))) ? 1 : 0;
-      }
+  if (n <= 256) {
+    // rank by counting: one pass, quadratic in the range
+    for (int i = tid; i < n; i += SQ_THREADS) {
+      key[i] = float_key(conf[blk_lo + i]);
+      valid[i] = masked[blk_lo + i] != 0;
     }
-    sel[i] = valid[i] && rank < k;
+    __syncthreads();
+    for (int i = tid; i < n; i += SQ_THREADS) {
+      int rank = 0;
+      if (valid[i]) {
+        const uint32_t ki = key[i];
+        for (int j = 0; j < n; ++j) {
+          const uint32_t kj = key[j];
+          rank += (valid[j] && (kj > ki || (kj == ki && j < i))) ? 1 : 0;
+        }
+      }
+      sel[i] = valid[i] && rank < k;
+    }
+    __syncthreads();
+  } else {
+    // long ranges: the masked positions are compacted (index order kept), the k largest of their keys are marked by
+    // the radix descent (equal keys in index order), and the marks are scattered back
+    int n_cand = 0;
+    for (int c0 = 0; c0 < n; c0 += SQ_THREADS) {
+      const int i = c0 + tid;
+      const int f = (i < n && masked[blk_lo + i] != 0) ? 1 : 0;
+      int tot;
+      const int pre = block_excl_scan(f, scan_s, tot);
+      if (f) { key[n_cand + pre] = float_key(conf[blk_lo + i]); cpos[n_cand + pre] = (uint16_t)i; }
+      if (i < n) sel[i] = 0;
+      n_cand += tot;
+    }
+    __syncthreads();
+    block_topc_mark(key, n_cand, min(k, n_cand), valid, hist, scan_s);
+    for (int c = tid; c < n_cand; c += SQ_THREADS)
+      if (valid[c]) sel[cpos[c]] = 1;
+    __syncthreads();
   }
-  __syncthreads();
   // ascending compaction of the selected positions
   int base = 0;
   for (int c0 = 0; c0 < n; c0 += SQ_THREADS) {

@@ -94,6 +94,16 @@ def test_select_queries_exact(ctx):
         k = int(rng.integers(0, 40))
         w = int(rng.integers(0, 12))
         cases.append((conf, masked, L, lo, hi, k, w, M, L))
+    # the longest decoding block the stage takes (4096 positions), small and large k, ties cut by the threshold, NaNs
+    for k_long, quant in ((1, 0), (37, 16), (1024, 64), (600, 4)):
+        Lb = 5000
+        c = rng.beta(2, 5, size=Lb).astype(np.float32)
+        if quant:
+            c = np.round(c * quant) / quant
+        c[rng.integers(0, Lb, size=9)] = np.nan
+        msk = (rng.random(Lb) < 0.7).astype(np.uint8)
+        cases.append((c, msk, Lb, 300, 300 + 4096, k_long, 4, 0, Lb))
+    cases.append((np.full(5000, 0.25, dtype=np.float32), np.ones(5000, dtype=np.uint8), 5000, 0, 4096, 1000, 2, 0, 5000))
     conf = np.full(64, 0.5, dtype=np.float32)
     cases.append((conf, np.ones(64, dtype=np.uint8), 64, 0, 64, 8, 8, 0, 64))            # all equal
     cases.append((conf, np.zeros(64, dtype=np.uint8), 64, 0, 64, 8, 8, 0, 64))           # nothing masked
