@@ -413,7 +413,7 @@ def run_focus(args):
         cpu = {"value": v, "unit": "ms", "cores": cores, "kind": "oracle", "sample": sample}
 
     # dram__bytes_read.sum + dram__bytes_write.sum of one dense-layer launch of this shape (32 heads, L = 32768,
-    # I_active rows) from the ncu capture summarised in profiles/attn_tc_kernel_dense_and_sparse_c2_4layers.md
+    # I_active rows) from the ncu capture of that kernel summarised under profiles/
     traffic = 541_394_688 if (args.config == 2 and not args.layers) else None
     out = {
         "metric": METRIC, "value": ms_step, "unit": "ms", "n_gpus": world, "steps": K, "warmup": W,
