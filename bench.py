@@ -9,6 +9,8 @@ Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bou
 from __future__ import annotations
 
 import argparse
+import contextlib
+import datetime
 import json
 import math
 import os
@@ -37,44 +39,92 @@ def peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed regions run.
+
+    Every sample carries nvidia-smi's own timestamp; `window()` brackets a timed region with host wall-clock times
+    (same machine clock), and `stop()` keeps only the samples that fall inside a window, so that the median is a
+    clock under load and not one taken while the host was building a graph."""
+    Q = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    INTERVAL_MS = 25
 
     def __init__(self, index: int):
-        self.index, self.proc, self.lines = index, None, []
+        self.index, self.proc, self.lines, self.windows = index, None, [], []
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                                          "-i", str(self.index), "-lms", str(self.INTERVAL_MS)],
+                                         stdout=subprocess.PIPE, text=True)
             self.t = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
             self.t.start()
+            t0 = time.time()
+            while not self.lines and time.time() - t0 < 5.0:      # first sample in hand before any timed region
+                time.sleep(0.01)
         except Exception:
             self.proc = None
+
+    def window(self, headline=False):
+        """Context manager marking a timed region; samples stamped inside it count as 'under load'."""
+        sampler = self
+
+        class _W:
+            def __enter__(self):
+                self.t0 = datetime.datetime.now()
+
+            def __exit__(self, *exc):
+                sampler.windows.append((self.t0, datetime.datetime.now(), headline))
+        return _W()
 
     def stop(self):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(2 * self.INTERVAL_MS / 1000)
         self.proc.terminate()
         self.t.join(timeout=2)
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        sm, sm_head, mx, watts, reasons = [], [], [], [], set()
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
-            if len(f) < 9:
+            if len(f) < 10:
                 continue
             try:
-                sm.append(float(f[1])); mx.append(float(f[2]))
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f")
+                clk, cmax = float(f[2]), float(f[3])
             except ValueError:
                 continue
-            for n, v in zip(names, f[5:9]):
+            mx.append(cmax)
+            inside = [h for a, z, h in self.windows if a <= ts <= z]
+            if not inside:
+                continue
+            sm.append(clk)
+            if any(inside):
+                sm_head.append(clk)
+            try:
+                watts.append(float(f[4]))
+            except ValueError:
+                pass
+            for n, v in zip(names, f[6:10]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        note = None
+        if not sm and mx:                                  # a very short region can fall between two samples
+            note = "no sample fell inside a timed region; clocks of the samples around it"
+            for ln in self.lines:
+                f = [x.strip() for x in ln.split(",")]
+                try:
+                    sm.append(float(f[2]))
+                except (ValueError, IndexError):
+                    pass
+        out = {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "samples_in_headline_region": len(sm_head),
+                "sm_mhz_headline_region": statistics.median(sm_head) if sm_head else None,
+                "power_w": statistics.median(watts) if watts else None,
+                "interval_ms": self.INTERVAL_MS, "reasons": sorted(reasons)}
+        if note:
+            out["note"] = note
+        return out
 
 
 # --------------------------------------------------------------------------------------------------
@@ -259,16 +309,19 @@ def run_focus(args):
             replicas.barrier()
             torch.cuda.synchronize()
 
-    def timed(fn, steps, warmup, with_marks=False):
+    sampler = None
+
+    def timed(fn, steps, warmup, with_marks=False, headline=False):
         for _ in range(warmup):
             fn(None)
         sync_all()
         marks = [] if with_marks else None
         evs = [(ev(), ev()) for _ in range(steps)]
         n0 = fb.focus_launch_count()
-        for a, z in evs:
-            a.record(); fn(marks); z.record()
-        sync_all()
+        with (sampler.window(headline) if sampler is not None else contextlib.nullcontext()):
+            for a, z in evs:
+                a.record(); fn(marks); z.record()
+            sync_all()
         launches = fb.focus_launch_count() - n0
         ms = [a.elapsed_time(z) for a, z in evs]
         tot = float(sum(ms))
@@ -278,7 +331,11 @@ def run_focus(args):
     K, W = args.steps, max(args.warmup, 3)
     # eager pass with CUDA-event marks around every attention call (per-call durations; the roofline uses them only
     # with --no-graph, otherwise the per-launch average of a graph of those launches, see below)
-    ms_eager, launches, marks = timed(lambda m: step("active", marks=m), K, W, with_marks=True)
+    sampler = ClockSampler(local)
+    sampler.INTERVAL_MS = max(5, args.clock_interval_ms)
+    sampler.start()
+    ms_eager, launches, marks = timed(lambda m: step("active", marks=m), K, W, with_marks=True,
+                                      headline=args.no_graph)
     assert ctx.poll_status() == 0, "device status word set during the timed region"
     # the same step captured once into a CUDA graph (counts stay on the device, so nothing needs the host)
     graph = None
@@ -294,16 +351,17 @@ def run_focus(args):
         with torch.cuda.graph(graph):
             step("active")
         launches = fb.focus_launch_count() - n0          # kernels per replayed step
-    sampler = ClockSampler(local)
-    sampler.start()
     if graph is not None:
-        ms_step, _, _ = timed(lambda m: graph.replay(), K, W)
+        ms_step, _, _ = timed(lambda m: graph.replay(), K, W, headline=True)
         launches *= K
     else:
         ms_step = ms_eager
-    clocks = sampler.stop()
     assert ctx.poll_status() == 0, "device status word set during the timed region"
 
+    # The sampler stops here: with nvidia-smi polling every 25 ms the per-launch figures below came out 5-8 % slower
+    # (measured by alternating runs), while the step time above did not move beyond its run-to-run spread.
+    clocks = sampler.stop()
+    sampler = None
     dense_t = [a.elapsed_time(z) for kind, a, z in marks if kind == "dense"]
     sparse_t = [a.elapsed_time(z) for kind, a, z in marks if kind == "sparse"]
     # The dominant kernel in the launch mode of the headline number: the dense-attention launches of one step (each on
@@ -655,6 +713,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="time eager C-ABI calls instead of a CUDA graph replay")
     ap.add_argument("--stages", action="store_true", help="per-stage latencies of --config (0..3) instead of the step")
     ap.add_argument("--sweep", action="store_true", help="run the context x keep-ratio sweep (config 4) instead")
+    ap.add_argument("--clock-interval-ms", type=int, default=25, help="nvidia-smi sampling period during timed regions")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle baseline leg")
     args = ap.parse_args()
     if args.stages:
