@@ -97,7 +97,9 @@ uint64_t focus_launch_count(void);
 
 /* Which attention kernel the last focus_dense_attn / focus_sparse_attn / focus_sparse_layer call on this context
  * used: 1 = generic SIMT, 2 = tensor-core kernel with one 128-row query tile per CTA, 3 = tensor-core kernel with
- * two query tiles per CTA (taken for >= 256 stacked rows per KV head and >= 16 key tiles per CTA); 0 = none yet. */
+ * two query tiles per CTA (taken for >= 256 stacked rows per KV head and >= 24 key tiles per CTA), 4 = tensor-core
+ * kernel with one query tile and two softmax warpgroups on alternating key tiles (>= 128 stacked rows per KV head
+ * and >= 4 key tiles per CTA, where 3 does not apply); 0 = none yet. */
 int32_t focus_last_attn_variant(focus_ctx* ctx);
 
 /* Selects the attention implementation for bf16 / head_dim 128 inputs: 0 = automatic (tensor-core

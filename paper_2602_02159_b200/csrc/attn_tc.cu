@@ -17,7 +17,9 @@
 // be resident, partials go through global memory instead (last-arriving CTA or a second kernel merges).  Results
 // are deterministic either way.
 //
-// attn_tc_wide_kernel (further down): two query tiles per CTA for the tensor-bound regime.
+// attn_tc_wide_kernel<false> (further down): two query tiles per CTA for the tensor-bound regime;
+// attn_tc_wide_kernel<true>: one query tile, two softmax warpgroups on alternating key tiles, for query sets with at
+// least one full tile of rows that the two-tile form does not take.
 //
 // Every launch is a programmatic dependent launch: see the comment on p.pdl in attn_tc_kernel.
 #include <stdio.h>
@@ -369,13 +371,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   constexpr int QTHREADS = 128;                                  // the four softmax warps stage Q
   constexpr int QIT = TM * 16 / QTHREADS;                        // 16-byte chunks of the Q tile per staging thread
   const int qtid = (int)threadIdx.x - 64;
-  const int nrows_raw = p.q_rows ? __ldg(p.n_rows) : p.n_q;
+  const int nrows_raw = p.q_rows ? ld_ordered(p.n_rows) : p.n_q;
   int qpos[QIT];
 #pragma unroll
   for (int it = 0; it < QIT; ++it) {
     const int idx = qtid + it * QTHREADS;
     const int qr = (mt * TM + (idx >> 4)) / p.hpg;
-    qpos[it] = (qtid >= 0 && qr < p.rows_bound) ? (p.q_rows ? __ldg(p.q_rows + qr) : p.q_base + qr) : -1;
+    qpos[it] = (qtid >= 0 && qr < p.rows_bound) ? (p.q_rows ? ld_ordered(p.q_rows + qr) : p.q_base + qr) : -1;
   }
   const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
   const int total_fr = nrows * p.hpg;                    // stacked (row, head-of-group) rows of this KV head
@@ -406,7 +408,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         if (pos >= p.q_base && pos < p.q_base + p.n_q) {
           const __nv_bfloat16* src = p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
                                      (long long)(g * p.hpg + fr % p.hpg) * p.q_stride_head + c * 8;
-          qv[it] = __ldg(reinterpret_cast<const uint4*>(src));
+          qv[it] = ld_ordered(reinterpret_cast<const uint4*>(src));
         } else if (c == 0) {
           set_status(p.status, FOCUS_ERR_INVALID_ARG);
         }
@@ -432,7 +434,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     if (qtid >= 0) store_q();
     asm volatile("griddepcontrol.wait;" ::: "memory");
   }
-  const int cnt_raw = p.dense ? 0 : __ldg(p.block_cnt + g * p.group_stride);
+  const int cnt_raw = p.dense ? 0 : ld_ordered(p.block_cnt + g * p.group_stride);
 
   const TileEnum te = make_enum(p, g, cnt_raw);
   const int t0 = (int)(((long long)te.total * split) / p.n_splits);
@@ -809,6 +811,12 @@ constexpr int MAXT_W = 96;
 constexpr int NTHREADS_W = 384;                 // three warpgroups: {producer, MMA, two idle warps}, softmax A, softmax B
 constexpr int SMEM_BYTES_W = 1024 + Q_BYTES_W + NSLOT_W * SLOT_BYTES + NBAR_W * 8 + 64 + MAXT_W * 8;
 
+// KP = false: the two softmax warpgroups own two different 128-row query tiles and share every key tile (above).
+// KP = true ("key pair"): ONE 128-row query tile; warpgroup x takes the key tiles x, x + 2, x + 4, ... of the split
+// with its own running maximum, row sum and accumulator (S_x, O_x), so that two softmax streams run per SM on a
+// single query tile; the two halves are merged in the epilogue (each warpgroup reads both accumulators from TMEM
+// for 64 of the 128 output columns).  Used when a KV head has too few rows or key tiles for the two-tile form.
+template <bool KP>
 __global__ void __launch_bounds__(NTHREADS_W, 1)
 attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
                     const __grid_constant__ CUtensorMap tmSK, const __grid_constant__ CUtensorMap tmSV, const TcParams p) {
@@ -820,21 +828,22 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (p.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
 
+  constexpr int TMQ = KP ? TM : TMW;                             // query rows of this CTA
   constexpr int QTHREADS = 256;                                  // the eight softmax warps stage Q
-  constexpr int QIT = TMW * 16 / QTHREADS;
+  constexpr int QIT = TMQ * 16 / QTHREADS;
   const int qtid = (int)threadIdx.x - 128;
-  const int nrows_raw = p.q_rows ? __ldg(p.n_rows) : p.n_q;
-  const int cnt_raw = p.dense ? 0 : __ldg(p.block_cnt + g * p.group_stride);
+  const int nrows_raw = p.q_rows ? ld_ordered(p.n_rows) : p.n_q;
+  const int cnt_raw = p.dense ? 0 : ld_ordered(p.block_cnt + g * p.group_stride);
   int qpos[QIT];
 #pragma unroll
   for (int it = 0; it < QIT; ++it) {
     const int idx = qtid + it * QTHREADS;
-    const int qr = (mt * TMW + (idx >> 4)) / p.hpg;
-    qpos[it] = (qtid >= 0 && qr < p.rows_bound) ? (p.q_rows ? __ldg(p.q_rows + qr) : p.q_base + qr) : -1;
+    const int qr = (mt * TMQ + (idx >> 4)) / p.hpg;
+    qpos[it] = (qtid >= 0 && qr < p.rows_bound) ? (p.q_rows ? ld_ordered(p.q_rows + qr) : p.q_base + qr) : -1;
   }
   const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
   const int total_fr = nrows * p.hpg;
-  if (mt * TMW >= total_fr) return;
+  if (mt * TMQ >= total_fr) return;
 
   const TileEnum te = make_enum(p, g, cnt_raw);
   const int t0 = (int)(((long long)te.total * split) / p.n_splits);
@@ -868,8 +877,8 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   float* ps = reinterpret_cast<float*>(sptr + Q_BYTES_W);        // split partial (cluster mode), over the K/V ring
 
   if (nt <= 0) {                                                 // empty split (cluster mode only: see the launcher)
-    for (int r = threadIdx.x; r < TMW; r += NTHREADS_W) { ps[TMW * PROW + 2 * r] = -INFINITY; ps[TMW * PROW + 2 * r + 1] = 0.f; }
-    cluster_merge<TMW, 256>(p, g, mt, total_fr, split, sSlot, (int)threadIdx.x - 128);
+    for (int r = threadIdx.x; r < TMQ; r += NTHREADS_W) { ps[TMQ * PROW + 2 * r] = -INFINITY; ps[TMQ * PROW + 2 * r + 1] = 0.f; }
+    cluster_merge<TMQ, 256>(p, g, mt, total_fr, split, sSlot, (int)threadIdx.x - 128);
     return;
   }
 
@@ -923,14 +932,14 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     for (int it = 0; it < QIT; ++it) {
       const int idx = qtid + it * QTHREADS;
       const int r = idx >> 4, c = idx & 15;
-      const int fr = mt * TMW + r;
+      const int fr = mt * TMQ + r;
       qv[it] = make_uint4(0, 0, 0, 0);
       if (fr < total_fr) {
         const int pos = qpos[it];
         if (pos >= p.q_base && pos < p.q_base + p.n_q) {
           const __nv_bfloat16* src = p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
                                      (long long)(g * p.hpg + fr % p.hpg) * p.q_stride_head + c * 8;
-          qv[it] = __ldg(reinterpret_cast<const uint4*>(src));
+          qv[it] = ld_ordered(reinterpret_cast<const uint4*>(src));
         } else if (c == 0) {
           set_status(p.status, FOCUS_ERR_INVALID_ARG);
         }
@@ -976,8 +985,8 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       constexpr uint32_t IDESC_PV = make_idesc(TM, HD, 1);
       bool ok = true;
       auto wait_load = [&](int q) { return mbar_wait(bar_full(q % NSLOT_W), (uint32_t)(q / NSLOT_W) & 1u, abort_flag, p.status); };
-      auto do_qk = [&](int x, int j) {                              // S_x = Q_x K_j^T
-        const uint64_t qdesc = make_sdesc(sQ + x * Q_BYTES, 16, 1024);
+      auto do_qk = [&](int x, int j) {                              // S_x = Q_x K_j^T (KP: the one query tile)
+        const uint64_t qdesc = make_sdesc(sQ + (KP ? 0 : x) * Q_BYTES, 16, 1024);
         const uint64_t kdesc = make_sdesc(sSlot + ((2 * j) % NSLOT_W) * SLOT_BYTES, 16, 1024);
 #pragma unroll
         for (int half = 0; half < 2; ++half)
@@ -989,14 +998,14 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         tc_commit(bar_sfull(x));
       };
       // O_x += P_x(j) V_j in two halves of 64 keys: the first starts while the softmax warps still work on the second
-      auto do_pv = [&](int x, int j, uint32_t par) -> bool {
+      auto do_pv = [&](int x, int j, uint32_t par, bool first) -> bool {
         const uint64_t vdesc = make_sdesc(sSlot + ((2 * j + 1) % NSLOT_W) * SLOT_BYTES, HALF_BYTES, 1024);
         if (!mbar_wait(bar_pready(x), par, abort_flag, p.status)) return false;
         tc_fence_after();
 #pragma unroll
         for (int ks = 0; ks < TN / 32; ++ks)
           mma_ts(tmem + 256 + x * 128, tmem + x * 128 + ks * 8, vdesc + (uint64_t)(ks * (2048 >> 4)), IDESC_PV,
-                 (j > 0 || ks > 0) ? 1u : 0u);
+                 (!first || ks > 0) ? 1u : 0u);
         if (!mbar_wait(bar_pready2(x), par, abort_flag, p.status)) return false;
         tc_fence_after();
 #pragma unroll
@@ -1005,6 +1014,36 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         tc_commit(bar_pvdone(x));
         return true;
       };
+      if (KP) {
+        // key tile t belongs to warpgroup t & 1; consumption order K0, K1, V0, K2, V1, K3, ... stays inside the
+        // ring window (the oldest slot still held and the newest one needed are at most four loads apart)
+        ok = wait_load(0);
+        if (ok) {
+          tc_fence_after();
+          do_qk(0, 0);
+          tc_commit(bar_empty(0));
+        }
+        if (ok && nt > 1) {
+          ok = wait_load(2);
+          if (ok) {
+            tc_fence_after();
+            do_qk(1, 1);
+            tc_commit(bar_empty(2 % NSLOT_W));
+          }
+        }
+        for (int t = 0; t < nt && ok; ++t) {
+          const int x = t & 1;
+          if (!wait_load(2 * t + 1)) { ok = false; break; }          // V_t
+          if (!do_pv(x, t, (uint32_t)(t >> 1) & 1u, t < 2)) { ok = false; break; }
+          tc_commit(bar_empty((2 * t + 1) % NSLOT_W));
+          if (t + 2 < nt) {
+            if (!wait_load(2 * t + 4)) { ok = false; break; }        // K_(t+2)
+            tc_fence_after();
+            do_qk(x, t + 2);
+            tc_commit(bar_empty((2 * t + 4) % NSLOT_W));
+          }
+        }
+      } else {
       ok = wait_load(0);
       if (ok) {
         tc_fence_after();
@@ -1016,7 +1055,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const uint32_t par = (uint32_t)j & 1u;
         if (!wait_load(2 * j + 1)) { ok = false; break; }            // V_j
         TL_ITER(0, 32, j, 0);
-        if (!do_pv(0, j, par)) { ok = false; break; }
+        if (!do_pv(0, j, par, j == 0)) { ok = false; break; }
         TL_ITER(0, 32, j, 4);
         if (j + 1 < nt) {
           if (!wait_load(2 * j + 2)) { ok = false; break; }          // K_(j+1)
@@ -1025,7 +1064,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         }
         TL_ITER(0, 32, j, 5);
         TL_ITER(0, 32, j, 2);
-        if (!do_pv(1, j, par)) { ok = false; break; }
+        if (!do_pv(1, j, par, j == 0)) { ok = false; break; }
         tc_commit(bar_empty((2 * j + 1) % NSLOT_W));                 // V_j
         TL_ITER(0, 32, j, 6);
         if (j + 1 < nt) {
@@ -1033,6 +1072,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           tc_commit(bar_empty((2 * j + 2) % NSLOT_W));               // K_(j+1)
         }
         TL_ITER(0, 32, j, 7);
+      }
       }
       tc_commit(bar_alldone);
     }
@@ -1046,7 +1086,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       tmem_dealloc(tmem, 512);
     }
     TL_STAMP(3, 0);
-    if (p.n_splits > 1) cluster_merge<TMW, 256>(p, g, mt, total_fr, split, sSlot, -1);
+    if (p.n_splits > 1) cluster_merge<TMQ, 256>(p, g, mt, total_fr, split, sSlot, -1);
     TL_STAMP(4, 0);
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
@@ -1058,7 +1098,8 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const uint32_t to = tmem + lane_off + 256 + x * 128;
     float m_ref = -INFINITY, l = 0.f;
     bool ok = true;
-    for (int idx = 0; idx < nt; ++idx) {
+    const int nt_x = KP ? (nt - x + 1) / 2 : nt;                     // key tiles of this warpgroup
+    for (int idx = 0; idx < nt_x; ++idx) {
       TL_ITER(warp - 3, warp * 32, idx, 0);
       if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(x), (uint32_t)idx & 1u, abort_flag, p.status))) { ok = false; break; }
       TL_ITER(warp - 3, warp * 32, idx, 1);
@@ -1070,7 +1111,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       TC_LD32(ts + 96, (sreg + 96));
       tc_wait_ld();
       TL_ITER(warp - 3, warp * 32, idx, 2);
-      const TileInfo ti = get_tile(idx);
+      const TileInfo ti = get_tile(KP ? 2 * idx + x : idx);
       float tmax = -INFINITY;
       if (ti.kind == 0 && ti.nvalid == TN) {
         float t4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains instead of one of 128
@@ -1154,9 +1195,70 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       l = l * alpha + ((acc[0] + acc[1]) + (acc[2] + acc[3]));
       TL_ITER(warp - 3, warp * 32, idx, 5);
     }
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_pvdone(x), (uint32_t)(nt - 1) & 1u, abort_flag, p.status));
+    if (ok && nt_x > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_pvdone(x), (uint32_t)(nt_x - 1) & 1u, abort_flag, p.status));
     TL_STAMP(2, 128);
-    if (ok) {
+    if (KP) {
+      // Merge of the two warpgroups' halves.  Both accumulators are complete once every MMA of the CTA has retired;
+      // the (reference max, row sum) pairs cross through shared memory (over the K/V ring, idle by then).
+      ok = ok && __all_sync(0xffffffffu, mbar_wait(bar_alldone, 0u, abort_flag, p.status));
+      tc_fence_after();
+      float2* xch = reinterpret_cast<float2*>(ps + TMQ * PROW + 2 * TMQ);
+      if (ok) xch[x * TM + row] = make_float2(nt_x > 0 ? m_ref : -INFINITY, nt_x > 0 ? l : 0.f);
+      asm volatile("bar.sync 1, 256;" ::: "memory");                 // the eight softmax warps (taken on every path)
+      if (ok) {
+        const float2 ea = xch[row], eb = xch[TM + row];
+        float m = -INFINITY;
+        if (ea.y > 0.f) m = ea.x;
+        if (eb.y > 0.f) m = fmaxf(m, eb.x);
+        const float wa = ea.y > 0.f ? ex2(ea.x - m) : 0.f, wb = eb.y > 0.f ? ex2(eb.x - m) : 0.f;
+        const float tot = wa * ea.y + wb * eb.y;
+        const int fr = mt * TMQ + row;
+        const bool valid = fr < total_fr;
+        const int qr = valid ? fr / p.hpg : 0, hh = valid ? fr % p.hpg : 0;
+        const float inv = p.n_splits == 1 ? (tot > 0.f ? 1.f / tot : 0.f) : 1.f;
+        const float fa = wa * inv, fb = wb * inv;
+        const uint32_t toa = tmem + lane_off + 256, tob = tmem + lane_off + 384;
+        __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD;
+        float* prow = ps + row * PROW;
+#pragma unroll
+        for (int cb = 2 * x; cb < 2 * x + 2; ++cb) {                 // this warpgroup's 64 output columns
+          uint32_t oa[32], ob[32];
+          TC_LD32(toa + cb * 32, oa);
+          if (nt > 1) TC_LD32(tob + cb * 32, ob);                    // with one key tile O_B was never written
+          tc_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            float v = __uint_as_float(oa[c]) * fa;
+            if (nt > 1 && fb > 0.f) v = fmaf(__uint_as_float(ob[c]), fb, v);
+            oa[c] = __float_as_uint(v);
+          }
+          if (valid) {
+            if (p.n_splits == 1) {
+#pragma unroll
+              for (int c = 0; c < 32; c += 8) {
+                uint4 v;
+                v.x = pack_bf16(__uint_as_float(oa[c + 0]), __uint_as_float(oa[c + 1]));
+                v.y = pack_bf16(__uint_as_float(oa[c + 2]), __uint_as_float(oa[c + 3]));
+                v.z = pack_bf16(__uint_as_float(oa[c + 4]), __uint_as_float(oa[c + 5]));
+                v.w = pack_bf16(__uint_as_float(oa[c + 6]), __uint_as_float(oa[c + 7]));
+                *reinterpret_cast<uint4*>(orow + cb * 32 + c) = v;
+              }
+            } else {
+#pragma unroll
+              for (int c = 0; c < 32; c += 4)
+                *reinterpret_cast<uint4*>(prow + cb * 32 + c) = make_uint4(oa[c], oa[c + 1], oa[c + 2], oa[c + 3]);
+            }
+          }
+        }
+        if (valid && x == 0) {
+          if (p.n_splits == 1) {
+            if (p.lse) p.lse[(size_t)(g * p.hpg + hh) * p.lse_stride + qr] = (m + log2f(tot)) * 0.6931471805599453f;
+          } else {
+            ps[TMQ * PROW + 2 * row] = m; ps[TMQ * PROW + 2 * row + 1] = tot;
+          }
+        }
+      }
+    } else if (ok) {
       tc_fence_after();
       const int trow = x * 128 + row;                                // row inside the 256-row CTA tile
       const int fr = mt * TMW + trow;
@@ -1206,7 +1308,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     // tail of the softmax warpgroups (kept inside their register-budget region): they do the split merge
     tc_fence_before();
     asm volatile("bar.sync 0;" ::: "memory");
-    if (p.n_splits > 1) cluster_merge<TMW, 256>(p, g, mt, total_fr, split, sSlot, (int)threadIdx.x - 128);
+    if (p.n_splits > 1) cluster_merge<TMQ, 256>(p, g, mt, total_fr, split, sSlot, (int)threadIdx.x - 128);
   }
 }
 
@@ -1362,7 +1464,8 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   bool& attr_set = ctx->ls.attn_attr_set;
   if (!attr_set) {
     if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
-        cudaFuncSetAttribute(attn_tc_wide_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES_W) != cudaSuccess)
+        cudaFuncSetAttribute(attn_tc_wide_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES_W) != cudaSuccess ||
+        cudaFuncSetAttribute(attn_tc_wide_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES_W) != cudaSuccess)
       return FOCUS_ERR_CUDA;
     attr_set = true;
   }
@@ -1380,19 +1483,36 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     n_splits = pick_splits(ctx, base, max_tiles);
     if (n_splits > 1) {
       if (cluster_cap_w[n_splits] == 0)
-        cluster_cap_w[n_splits] = cluster_capacity(attn_tc_wide_kernel, n_splits, NTHREADS_W, SMEM_BYTES_W) + 1;
+        cluster_cap_w[n_splits] = cluster_capacity(attn_tc_wide_kernel<false>, n_splits, NTHREADS_W, SMEM_BYTES_W) + 1;
       if (cluster_cap_w[n_splits] - 1 < base) wide = false;           // its splits merge through a cluster only
     }
-    // it pays from about 16 key tiles per CTA upward (measured: 256 us against 316 us on dense 32K with 512 rows,
-    // 47 against 49 us at 8K with 256 rows); below that the one-tile kernel, which needs fewer or no key splits, wins
-    static const int wide_min = getenv("FOCUS_WIDE_MIN") ? atoi(getenv("FOCUS_WIDE_MIN")) : 16;
+    // it pays from about 24 key tiles per CTA upward (measured at 256 rows, 32 heads: 32 tiles per CTA 85 us against
+    // 87 us for the key-pair form, 17 to 19 tiles per CTA 3 to 12 % slower than it); below that the one-tile forms,
+    // which need fewer or no key splits, win
+    static const int wide_min = getenv("FOCUS_WIDE_MIN") ? atoi(getenv("FOCUS_WIDE_MIN")) : 24;
     if (max_tiles / n_splits < wide_min) wide = false;
   }
+  // key-pair form: one query tile per CTA, two softmax warpgroups on alternating key tiles.  For query sets with
+  // enough rows per tile to be bound by the exponentials (not by HBM) that the two-tile form does not take.
+  bool kpair = false;
   if (!wide) {
     n_mtiles = (int)((stacked + TM - 1) / TM);
     base = n_mtiles * Hkv;
     n_splits = pick_splits(ctx, base, max_tiles);
+    static const int kp_min_rows = getenv("FOCUS_KP_MIN_ROWS") ? atoi(getenv("FOCUS_KP_MIN_ROWS")) : 128;
+    static const int kp_min_tiles = getenv("FOCUS_KP_MIN_TILES") ? atoi(getenv("FOCUS_KP_MIN_TILES")) : 4;
+    if (!ctx->no_wide && stacked >= kp_min_rows && max_tiles / n_splits >= kp_min_tiles &&
+        (n_splits == 1 || ctx->merge_mode == 0)) {
+      kpair = true;
+      if (n_splits > 1) {                                                // its splits merge through a cluster only
+        int* cap = ctx->ls.cluster_cap_k;
+        if (cap[n_splits] == 0)
+          cap[n_splits] = cluster_capacity(attn_tc_wide_kernel<true>, n_splits, NTHREADS_W, SMEM_BYTES_W) + 1;
+        if (cap[n_splits] - 1 < base) kpair = false;
+      }
+    }
   }
+  const bool wg3 = wide || kpair;                                        // three-warpgroup kernel (either form)
 
   __nv_bfloat16* gK = nullptr; __nv_bfloat16* gV = nullptr; uint8_t* mask = nullptr;
   if (ns_pad > 0) {
@@ -1405,7 +1525,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     }
   }
   bool use_cluster = false;
-  if (n_splits > 1 && !wide && ctx->merge_mode == 0) {
+  if (n_splits > 1 && !wg3 && ctx->merge_mode == 0) {
     // the largest split count (not above the one wanted) whose clusters are all resident at once; if even two-CTA
     // clusters do not fit, keep the wanted count and merge through global memory
     for (int sp = n_splits; sp >= 2; --sp) {
@@ -1414,9 +1534,9 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     }
     if (getenv("FOCUS_LOG")) fprintf(stderr, "[focus] attn: base %d splits %d cluster %d\n", base, n_splits, (int)use_cluster);
   }
-  if (wide) use_cluster = n_splits > 1;
+  if (wg3) use_cluster = n_splits > 1;
   float* part_O = nullptr; float* part_ml = nullptr;
-  if (n_splits > 1 && !use_cluster && !wide) {
+  if (n_splits > 1 && !use_cluster && !wg3) {
     part_O = ws.get<float>((size_t)base * n_splits * TM * HD);
     part_ml = ws.get<float>((size_t)base * n_splits * TM * 2);
   }
@@ -1447,8 +1567,8 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.sink_mask = mask; p.part_O = part_O; p.part_ml = part_ml;
   p.cluster = use_cluster ? 1 : 0;
   // 1: called right after the selection kernel of a fused sparse layer (pre-gathered sinks); 2: predecessor unknown
-  p.pdl = ctx->no_pdl ? 0 : ((pre != nullptr && !wide) ? 1 : 2);
-  p.counters = (n_splits > 1 && !use_cluster && !wide && ctx->merge_mode != 2 && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
+  p.pdl = ctx->no_pdl ? 0 : ((pre != nullptr && !wg3) ? 1 : 2);
+  p.counters = (n_splits > 1 && !use_cluster && !wg3 && ctx->merge_mode != 2 && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
                    ? ctx->d_counters : nullptr;
   p.q_stride_row = sh.q_stride_row; p.q_stride_head = sh.q_stride_head;
   p.q_base = a.q_base; p.n_q = a.n_q; p.rows_bound = a.max_rows; p.L = sh.L; p.M = sh.M; p.H = sh.n_q_heads;
@@ -1461,9 +1581,13 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.dbg = getenv("FOCUS_TIMELINE") ? (unsigned long long*)(ctx->ws + ctx->ws_bytes - (1 << 20)) : nullptr;
 #endif
 
-  ctx->last_attn_variant = wide ? 3 : 2;
+  ctx->last_attn_variant = wide ? 3 : (kpair ? 4 : 2);
   if (wide) {
-    focus_status ls = launch_ex(attn_tc_wide_kernel, dim3(base, n_splits, 1), NTHREADS_W, SMEM_BYTES_W, n_splits, p.pdl != 0, st,
+    focus_status ls = launch_ex(attn_tc_wide_kernel<false>, dim3(base, n_splits, 1), NTHREADS_W, SMEM_BYTES_W, n_splits, p.pdl != 0, st,
+                                tmK, tmV, tmSK, tmSV, p);
+    if (ls != FOCUS_OK) return ls;
+  } else if (kpair) {
+    focus_status ls = launch_ex(attn_tc_wide_kernel<true>, dim3(base, n_splits, 1), NTHREADS_W, SMEM_BYTES_W, n_splits, p.pdl != 0, st,
                                 tmK, tmV, tmSK, tmSV, p);
     if (ls != FOCUS_OK) return ls;
   } else {
@@ -1472,7 +1596,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     if (ls != FOCUS_OK) return ls;
   }
   FOCUS_CHECK_LAUNCH();
-  if (n_splits > 1 && !p.counters && !use_cluster && !wide) {
+  if (n_splits > 1 && !p.counters && !use_cluster && !wg3) {
     const int rows_total = base * TM;
     attn_combine_kernel<<<rows_total / 8, 256, 0, st>>>(part_O, part_ml, n_splits, n_mtiles, hpg, sh.n_q_heads,
                                                         a.q_rows, a.n_rows, a.max_rows, a.n_q,

@@ -15,7 +15,7 @@ struct focus_ctx {
   int32_t* d_status;   // device status word: 0 = clean, else first anomaly's focus_status code
   int32_t* d_counters; // FOCUS_N_COUNTERS arrival counters for split merges; zero between launches
   int force_simt;
-  int last_attn_variant;   // 0 none yet, 1 SIMT, 2 tensor-core 128-row tiles, 3 tensor-core 256-row tiles
+  int last_attn_variant;   // 0 none yet, 1 SIMT, 2 tensor-core 128-row tiles, 3 tensor-core 256-row tiles, 4 key-pair form
   int no_pdl;          // 1: never launch the attention kernel as a programmatic dependent (A/B comparisons)
   int no_wide;         // 1: never use the two-query-tile attention kernel (A/B comparisons)
   int merge_mode;      // split merge of the one-tile kernel: 0 automatic (cluster where it fits), 1 never a cluster (arrival
@@ -26,7 +26,7 @@ struct focus_ctx {
   struct LaunchState {
     bool attn_attr_set, select_attr_set, topn_attr_set;
     int sink_attr_smem;
-    int cluster_cap[9], cluster_cap_w[9];      // co-resident clusters per cluster size, value + 1 (0 = not asked yet)
+    int cluster_cap[9], cluster_cap_w[9], cluster_cap_k[9];   // co-resident clusters per cluster size, value + 1 (0 = not asked yet)
     int select_cluster;                        // 0 not tried, 1 works, 2 the cluster launch was refused once
   } ls;
 };

@@ -62,6 +62,21 @@ __device__ __forceinline__ void fence_barrier_init() {
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// Coherent global loads that stay in program order with the other volatile asm statements, in particular after
+// griddepcontrol.wait.  For everything an earlier kernel of the stream may have written and that is read right after
+// that wait: a non-coherent load (__ldg) promises the compiler read-only data, so it may be moved above the wait (seen:
+// CTAs started ahead of the selection kernel read the block count of the previous call).
+__device__ __forceinline__ int ld_ordered(const int* p) {
+  int v;
+  asm volatile("ld.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint4 ld_ordered(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+  return v;
+}
+
 // ---- TMA: 3-D tiled load global -> shared, completion on an mbarrier; one destination CTA ------
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2) {
   asm volatile(

@@ -298,10 +298,70 @@ def _rand_qkv(s, seed, qk_scale=1.0):
     return Qs, Ks, Vs
 
 
+@pytest.mark.parametrize("case", ["dense_split8", "dense_nosplit", "sparse_gqa_split8", "sparse_few_tiles"])
+def test_key_pair_kernel(ctx, case):
+    """Shapes that take the key-pair attention kernel (one 128-row query tile, two softmax warpgroups on alternating
+    key tiles, halves merged in the epilogue): at least 128 stacked rows per KV head, too few key tiles per CTA for
+    the two-query-tile kernel.  Covers the cluster merge of 8 splits with odd and even tile counts per split, the
+    unsplit case with a ragged last query tile, GQA row stacking, sparse tile lists with sink tiles and a ragged
+    last block, splits that end up with one key tile or none (one warpgroup idle / empty partial), and running-max
+    rescales (logit std ~1)."""
+    if case == "dense_split8":
+        s = wl.Shape(9000, 8872, 8, 8, 128, 128, "bf16")            # 128 rows/head, 71 key tiles, 8 CTAs x 8 splits
+        heads = [0, 5]
+    elif case == "dense_nosplit":
+        s = wl.Shape(2500, 1900, 32, 32, 128, 128, "bf16")          # 600 rows/head -> 160 CTAs, 20 tiles each
+        heads = [0, 31]
+    else:
+        s = wl.Shape(20000, 19872, 8, 2, 128, 128, "bf16")          # GQA 4:1 -> 512 stacked rows per KV head
+        heads = [1, 6]
+    Qs, Ks, Vs = _rand_qkv(s, 37, qk_scale=1.5)
+    dQ, dK, dV = (fstep.to_device(x, s.dtype) for x in (Qs, Ks, Vs))
+    sh = fstep.c_shape(s)
+    O = torch.zeros(s.N, s.H, s.d, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(s.H, s.N, dtype=torch.float32, device="cuda")
+    scale = 1.0 / math.sqrt(s.d)
+    hpg = s.H // s.Hkv
+    f64h = lambda a, h, kv=True: wl.storage_to_f64(a[h // hpg:h // hpg + 1] if kv else a[:, h:h + 1], s.dtype)
+    if case.startswith("dense"):
+        fb.focus_dense_attn(ctx, sh, dQ, s.M, s.N, None, None, 0, dK, dV, O, lse)
+        ref = {h: fo.dense_attn(f64h(Qs, h, False), f64h(Ks, h), f64h(Vs, h), scale) for h in heads}
+    else:
+        nb = s.nb                                                  # 156 blocks, the last one short (32 tokens)
+        rng = np.random.default_rng(7)
+        few = case == "sparse_few_tiles"
+        # 40 (39) blocks + 3 sink tiles + 1 response tile over 8 splits: five or six tiles per split;
+        # "few": room for 40 blocks but 2 and 1 selected -> 5 or 6 tiles in all, some splits get one tile or none
+        blocks = [np.sort(rng.choice(nb, size=n, replace=False)) for n in ((2, 1) if few else (40, 39))]
+        blocks[0][-1] = nb - 1                                     # make sure the ragged block is in one list
+        blocks[0] = np.unique(blocks[0])
+        C = 40
+        bidx = np.full((s.Hkv, C), -1, dtype=np.int32)
+        for g, b in enumerate(blocks):
+            bidx[g, :len(b)] = b
+        sinks = np.sort(rng.choice(s.M, size=300, replace=False)).astype(np.int32)
+        keep = np.array([[0 if (j // s.B) in set(blocks[g].tolist()) else 1 for j in sinks] for g in range(s.Hkv)],
+                        dtype=np.uint8)
+        fb.focus_sparse_attn(ctx, sh, dQ, s.M, s.N, None, None, 0, dK, dV, fb.HEADS_PER_KV_GROUP,
+                             torch.from_numpy(bidx.reshape(-1)).cuda(), C,
+                             torch.tensor([len(b) for b in blocks], dtype=torch.int32, device="cuda"),
+                             torch.from_numpy(sinks).cuda(), torch.from_numpy(keep.reshape(-1)).cuda(), len(sinks), O, lse)
+        ref = {h: fo.sparse_attn(f64h(Qs, h, False), f64h(Ks, h), f64h(Vs, h), s.M, s.B, [blocks[h // hpg]], sinks, scale)
+               for h in heads}
+    assert ctx.last_attn_variant() == 4, "the shape was meant to take the key-pair kernel"
+    got, got_lse = fstep.from_device(O), fstep.from_device(lse)
+    for h in heads:
+        Oh, lh = ref[h]
+        assert np.sqrt(np.mean(Oh ** 2)) > 0.02
+        assert max_abs(got[:, h], Oh[:, 0]) <= 2e-2 and rel_rms(got[:, h], Oh[:, 0]) <= 1e-2
+        assert max_abs(got_lse[h], lh[0]) <= 2e-3
+    assert ctx.poll_status() == 0
+
+
 @pytest.mark.parametrize("case", ["dense_split8", "dense_nosplit", "sparse_gqa_split8"])
 def test_two_query_tile_kernel(ctx, case):
     """Shapes that take the 256-row (two query tiles per CTA) attention kernel: >= 256 stacked rows per KV head and
-    >= 32 key tiles per CTA.  Covers the cluster merge of 8 splits, the unsplit case, GQA row stacking, sparse tile
+    >= 24 key tiles per CTA (here 32 and more).  Covers the cluster merge of 8 splits, the unsplit case, GQA row stacking, sparse tile
     lists with sink tiles and a ragged last block, and running-max rescales (logit std ~1)."""
     if case == "dense_split8":
         s = wl.Shape(33000, 32744, 8, 8, 128, 128, "bf16")          # 256 rows/head, 258 key tiles, 8 CTAs x 8 splits
