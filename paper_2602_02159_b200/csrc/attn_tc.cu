@@ -61,6 +61,7 @@ struct TcParams {
   int n_mtiles, n_splits, lse_stride;
   int cluster;                 // 1: the splits of a tile are one thread-block cluster and merge through shared memory
   int pdl;                     // 1: launched as a programmatic dependent of the selection kernel (see the wait below)
+  int pair;                    // 1: 64-token KV blocks, two selected blocks per 128-key tile; tmK / tmV have 64-row boxes
   float scale_log2;            // softmax scale * log2(e)
   int32_t* status;
 #ifdef FOCUS_TIMELINE
@@ -82,20 +83,38 @@ struct TileInfo {
   int kind;     // 0: tile of the K/V tensors, 1: tile of the gathered sink rows
   int start;    // first key row of the tile in its tensor
   int nvalid;   // leading columns that are real keys (the rest is masked out)
+  int start2;   // pair mode, kind 0: first key row of the tile's second half (columns 64..127)
 };
+// staged form of a TileInfo: x = start | kind << 30; y = nvalid | code << 8, code = start2 / 64 for a pair of
+// blocks, all ones for "the 64 rows after the first half"
+constexpr int START2_NEXT = 0x7FFFFF;
+__device__ __forceinline__ int2 pack_tile(const TileInfo& ti) {
+  const int code = ti.start2 == ti.start + 64 ? START2_NEXT : (ti.start2 >> 6);
+  return make_int2(ti.start | (ti.kind << 30), ti.nvalid | (code << 8));
+}
+__device__ __forceinline__ TileInfo unpack_tile(int2 e) {
+  TileInfo ti;
+  ti.kind = e.x >> 30; ti.start = e.x & 0x3FFFFFFF; ti.nvalid = e.y & 0xff;
+  const int code = (e.y >> 8) & START2_NEXT;
+  ti.start2 = code == START2_NEXT ? ti.start + 64 : code << 6;
+  return ti;
+}
 
 struct TileEnum {
-  int n_blk, n_sinkt, n_resp, total;
+  int n_blk;        // tiles that come from the block list (pair mode: two blocks per tile)
+  int n_blocks;     // entries of the block list
+  int n_sinkt, n_resp, total;
   const int32_t* blocks;
 };
 
 __device__ __forceinline__ TileEnum make_enum(const TcParams& p, int g, int cnt_raw) {
   TileEnum e;
   if (p.dense) {
-    e.n_blk = 0; e.n_sinkt = 0; e.n_resp = (p.L + TN - 1) / TN; e.blocks = nullptr;
+    e.n_blk = 0; e.n_blocks = 0; e.n_sinkt = 0; e.n_resp = (p.L + TN - 1) / TN; e.blocks = nullptr;
   } else {
     const int row = g * p.group_stride;
-    e.n_blk = min(max(cnt_raw, 0), p.max_blocks);
+    e.n_blocks = min(max(cnt_raw, 0), p.max_blocks);
+    e.n_blk = p.pair ? (e.n_blocks + 1) >> 1 : e.n_blocks;
     e.n_sinkt = p.ns_pad / TN;
     e.n_resp = (p.L - p.M + TN - 1) / TN;
     e.blocks = p.block_idx + (size_t)row * p.max_blocks;
@@ -106,8 +125,24 @@ __device__ __forceinline__ TileEnum make_enum(const TcParams& p, int g, int cnt_
 
 __device__ __forceinline__ TileInfo tile_info(const TcParams& p, const TileEnum& e, int t) {
   TileInfo ti;
+  ti.start2 = -1;
   if (p.dense) {
     ti.kind = 0; ti.start = t * TN; ti.nvalid = min(TN, p.L - ti.start);
+  } else if (t < e.n_blk && p.pair) {
+    // two 64-token blocks side by side; a short block (the last one of the prompt) goes second so that the valid
+    // columns stay a prefix; a missing second block repeats the first (finite data, masked out)
+    int b0 = e.blocks[2 * t];
+    int b1 = 2 * t + 1 < e.n_blocks ? e.blocks[2 * t + 1] : -2;
+    ti.kind = 0;
+    if (b0 < 0 || b0 >= p.nb || b1 == -1 || b1 < -2 || b1 >= p.nb) {  // reported once by the producer; fully masked
+      ti.start = 0; ti.start2 = 0; ti.nvalid = 0;
+    } else {
+      if (b1 >= 0 && p.M - b0 * 64 < 64) { const int x = b0; b0 = b1; b1 = x; }
+      ti.start = b0 * 64;
+      const int n0 = min(64, p.M - ti.start);
+      if (b1 >= 0) { ti.start2 = b1 * 64; ti.nvalid = n0 < 64 ? n0 : 64 + min(64, p.M - ti.start2); }
+      else { ti.start2 = ti.start; ti.nvalid = n0; }
+    }
   } else if (t < e.n_blk) {
     const int b = e.blocks[t];
     ti.kind = 0;
@@ -123,7 +158,25 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams& p, const TileEnum&
     const int r = t - e.n_blk - e.n_sinkt;
     ti.kind = 0; ti.start = p.M + r * TN; ti.nvalid = min(TN, p.L - ti.start);
   }
+  if (ti.start2 < 0) ti.start2 = ti.start + 64;
   return ti;
+}
+
+// One K or V tile into a ring slot (two 64-column halves, 128-byte swizzle).  Pair mode, tiles of the K/V tensors:
+// the maps have 64-row boxes and each half of the key range comes from its own place (rows 64..127 of a half sit
+// 8 KB, a whole number of swizzle atoms, after rows 0..63).
+__device__ __forceinline__ void load_tile(const TcParams& p, const TileInfo& ti, const CUtensorMap* map, uint32_t dst,
+                                          uint32_t bar, int g, uint64_t l2_pol) {
+  mbar_expect_tx(bar, SLOT_BYTES);
+  if (p.pair && ti.kind == 0) {
+    tma_load_3d_hint(dst, map, bar, 0, ti.start, g, l2_pol);
+    tma_load_3d_hint(dst + HALF_BYTES / 2, map, bar, 0, ti.start2, g, l2_pol);
+    tma_load_3d_hint(dst + HALF_BYTES, map, bar, 64, ti.start, g, l2_pol);
+    tma_load_3d_hint(dst + HALF_BYTES + HALF_BYTES / 2, map, bar, 64, ti.start2, g, l2_pol);
+  } else {
+    tma_load_3d_hint(dst, map, bar, 0, ti.start, g, l2_pol);
+    tma_load_3d_hint(dst + HALF_BYTES, map, bar, 64, ti.start, g, l2_pol);
+  }
 }
 
 // Merge of the split partials of one (KV head, query tile): out = sum_s 2^(m_s - m) O_s / sum_s 2^(m_s - m) l_s,
@@ -446,9 +499,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   // tile descriptor: from the staged list (sparse) or by arithmetic (dense; splits longer than the list)
   auto get_tile = [&](int idx) -> TileInfo {
     if (use_list) {
-      const int2 e = tlist[idx];
-      TileInfo ti; ti.kind = e.x >> 30; ti.start = e.x & 0x3FFFFFFF; ti.nvalid = e.y;
-      return ti;
+      return unpack_tile(tlist[idx]);
     }
     return tile_info(p, te, t0 + idx);
   };
@@ -499,10 +550,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     const TileInfo ti = get_tile(idx);
     const int slot = q % NSLOT;
     const CUtensorMap* map = ti.kind ? (isV ? &tmSV : &tmSK) : (isV ? &tmV : &tmK);
-    const uint32_t dst = sSlot + slot * SLOT_BYTES;
-    mbar_expect_tx(bar_full(slot), SLOT_BYTES);
-    tma_load_3d_hint(dst, map, bar_full(slot), 0, ti.start, g, l2_pol);
-    tma_load_3d_hint(dst + HALF_BYTES, map, bar_full(slot), 64, ti.start, g, l2_pol);
+    load_tile(p, ti, map, sSlot + slot * SLOT_BYTES, bar_full(slot), g, l2_pol);
   };
   const int n_loads = 2 * nt;
   const int n_early = n_loads < NSLOT ? n_loads : NSLOT;
@@ -511,11 +559,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     if (use_list) {
       for (int t = lane; t < nt; t += 32) {
         const TileInfo ti = tile_info(p, te, t0 + t);
-        if (t0 + t < te.n_blk) {
-          const int b = te.blocks[t0 + t];
-          if (b < 0 || b >= p.nb) set_status(p.status, FOCUS_ERR_INVALID_ARG);
-        }
-        tlist[t] = make_int2(ti.start | (ti.kind << 30), ti.nvalid);
+        if (t0 + t < te.n_blk && ti.nvalid == 0) set_status(p.status, FOCUS_ERR_INVALID_ARG);   // bad block index
+        tlist[t] = pack_tile(ti);
       }
     }
     __syncwarp();
@@ -868,9 +913,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const bool use_list = !p.dense && nt <= MAXT_W;
   auto get_tile = [&](int idx) -> TileInfo {
     if (use_list) {
-      const int2 e = tlist[idx];
-      TileInfo ti; ti.kind = e.x >> 30; ti.start = e.x & 0x3FFFFFFF; ti.nvalid = e.y;
-      return ti;
+      return unpack_tile(tlist[idx]);
     }
     return tile_info(p, te, t0 + idx);
   };
@@ -889,10 +932,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const TileInfo ti = get_tile(q >> 1);
     const int slot = q % NSLOT_W;
     const CUtensorMap* map = ti.kind ? (isV ? &tmSV : &tmSK) : (isV ? &tmV : &tmK);
-    const uint32_t dst = sSlot + slot * SLOT_BYTES;
-    mbar_expect_tx(bar_full(slot), SLOT_BYTES);
-    tma_load_3d_hint(dst, map, bar_full(slot), 0, ti.start, g, l2_pol);
-    tma_load_3d_hint(dst + HALF_BYTES, map, bar_full(slot), 64, ti.start, g, l2_pol);
+    load_tile(p, ti, map, sSlot + slot * SLOT_BYTES, bar_full(slot), g, l2_pol);
   };
   const int n_loads = 2 * nt;
   const int n_early = n_loads < NSLOT_W ? n_loads : NSLOT_W;
@@ -910,11 +950,8 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (use_list) {
       for (int t = lane; t < nt; t += 32) {
         const TileInfo ti = tile_info(p, te, t0 + t);
-        if (t0 + t < te.n_blk) {
-          const int b = te.blocks[t0 + t];
-          if (b < 0 || b >= p.nb) set_status(p.status, FOCUS_ERR_INVALID_ARG);
-        }
-        tlist[t] = make_int2(ti.start | (ti.kind << 30), ti.nvalid);
+        if (t0 + t < te.n_blk && ti.nvalid == 0) set_status(p.status, FOCUS_ERR_INVALID_ARG);   // bad block index
+        tlist[t] = pack_tile(ti);
       }
     }
     __syncwarp();
@@ -1460,7 +1497,10 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   if (stacked == 0) return FOCUS_OK;
   const int ns_pad = a.dense ? 0 : (a.n_sink + TN - 1) / TN * TN;
   const int n_resp = a.dense ? (sh.L + TN - 1) / TN : (sh.L - sh.M + TN - 1) / TN;
-  const int max_tiles = a.dense ? n_resp : a.max_blocks + ns_pad / TN + n_resp;
+  // 64-token KV blocks: two selected blocks share a 128-key tile
+  static const bool no_pair = getenv("FOCUS_NO_PAIR") != nullptr;          // A/B switch: one block per tile
+  const bool pair = !a.dense && sh.kv_block == 64 && !no_pair;
+  const int max_tiles = a.dense ? n_resp : (pair ? (a.max_blocks + 1) / 2 : a.max_blocks) + ns_pad / TN + n_resp;
   bool& attr_set = ctx->ls.attn_attr_set;
   if (!attr_set) {
     if (cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess ||
@@ -1543,8 +1583,9 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   if (!ws.ok) return FOCUS_ERR_WORKSPACE_TOO_SMALL;
 
   CUtensorMap tmK, tmV, tmSK, tmSV;
-  if (!encode_kv_map(ctx->encode_tiled, &tmK, a.K, HD, sh.L, Hkv, sh.kv_stride_tok, sh.kv_stride_head, 64, TN) ||
-      !encode_kv_map(ctx->encode_tiled, &tmV, a.V, HD, sh.L, Hkv, sh.kv_stride_tok, sh.kv_stride_head, 64, TN))
+  const int box_rows = pair ? 64 : TN;
+  if (!encode_kv_map(ctx->encode_tiled, &tmK, a.K, HD, sh.L, Hkv, sh.kv_stride_tok, sh.kv_stride_head, 64, box_rows) ||
+      !encode_kv_map(ctx->encode_tiled, &tmV, a.V, HD, sh.L, Hkv, sh.kv_stride_tok, sh.kv_stride_head, 64, box_rows))
     return FOCUS_ERR_INVALID_ARG;
   if (ns_pad > 0) {
     if (!encode_kv_map(ctx->encode_tiled, &tmSK, gK, HD, ns_pad, Hkv, HD, (long long)ns_pad * HD, 64, TN) ||
@@ -1566,6 +1607,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.q_rows = a.q_rows; p.n_rows = a.n_rows; p.block_idx = a.block_idx; p.block_cnt = a.block_cnt;
   p.sink_mask = mask; p.part_O = part_O; p.part_ml = part_ml;
   p.cluster = use_cluster ? 1 : 0;
+  p.pair = pair ? 1 : 0;
   // 1: called right after the selection kernel of a fused sparse layer (pre-gathered sinks); 2: predecessor unknown
   p.pdl = ctx->no_pdl ? 0 : ((pre != nullptr && !wg3) ? 1 : 2);
   p.counters = (n_splits > 1 && !use_cluster && !wg3 && ctx->merge_mode != 2 && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)

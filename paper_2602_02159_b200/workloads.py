@@ -96,7 +96,8 @@ class Workload:
 
 
 def config(idx: int, *, L: Optional[int] = None, keep_den: Optional[int] = None) -> Workload:
-    """The five benchmark configurations.  idx 4 (sweep) takes L and keep_den (keep ratio 1/keep_den)."""
+    """The five benchmark configurations (idx 0..4; idx 4, the sweep, takes L and keep_den = 1 / keep ratio) and,
+    as idx 5, the paper's own hyper-parameters on the 32K shape."""
     if idx == 0:
         s = Shape(1024, 896, 8, 8, 64, 64, "f32")
         return Workload("c0_tiny_f32", s, k=16, w=8, n_sink=8, C=4, blk_lo=896, blk_hi=1024, masked_count=64)
@@ -111,6 +112,13 @@ def config(idx: int, *, L: Optional[int] = None, keep_den: Optional[int] = None)
         s = Shape(16384, 16128, 28, 4, 128, 128, "bf16")
         return Workload("c3_dream_gqa_16k", s, k=8, w=8, n_sink=161, C=s.nb // 8, blk_lo=16128, blk_hi=16384,
                         n_steps=16)
+    if idx == 5:
+        # not one of the five benchmark configurations: the hyper-parameters of the paper's own experiments
+        # (Implementation details: prompt block size 64, sparsity ratio 0.5, six dense layers, rho = 4, w = 8,
+        # N_sink = 0.01 M) on the LLaDA attention shape at 32K context
+        s = Shape(32768, 32256, 32, 32, 128, 64, "bf16")
+        return Workload("c5_paper_hparams_32k", s, k=8, w=8, n_sink=322, C=s.nb // 2, blk_lo=32256,
+                        blk_hi=32256 + 32, n_layers=32, probe_layer=5)
     if idx == 4:
         L = 32768 if L is None else L
         keep_den = 16 if keep_den is None else keep_den

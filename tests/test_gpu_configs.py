@@ -250,3 +250,12 @@ def test_config4_sweep_points(ctx, L, keep_den):
     w = wl.config(4, L=L, keep_den=keep_den)
     heads = [0, 21] if L > 40000 else [0, 13, 31]
     single_layer_case(ctx, w, "gen", heads=heads, check_dense=L <= 40000)
+
+
+# ---- the paper's own hyper-parameters (block 64, half of the blocks kept) on the 32K shape, one layer ---------
+@pytest.mark.parametrize("rows", ["active", "gen"])
+def test_paper_hyperparameters_one_layer(ctx, rows):
+    """Prompt block size 64 and sparsity ratio 0.5 ("Implementation details"): 504 pooled blocks per head (the radix
+    Top-C path), 252 kept, paired two per 128-key tile by the attention kernel."""
+    w = wl.config(5)
+    single_layer_case(ctx, w, rows, heads=[0, 22], check_dense=False)

@@ -254,7 +254,7 @@ def test_long_key_pipeline_single_split(ctx):
     assert ctx.poll_status() == 0
 
 
-@pytest.mark.parametrize("cfg", [SHAPES[0], SHAPES[2], SHAPES[3]])
+@pytest.mark.parametrize("cfg", [SHAPES[0], SHAPES[2], SHAPES[3], SHAPES[5]])
 def test_fused_sparse_layer_matches_stagewise_and_oracle(ctx, cfg):
     """focus_sparse_layer (fused selection + attention) against the stage-by-stage calls and the oracle."""
     dtype, d, B, H, Hkv = cfg
@@ -296,6 +296,56 @@ def _rand_qkv(s, seed, qk_scale=1.0):
     Ks = wl.to_storage(rng.standard_normal((s.Hkv, s.L, s.d)).astype(np.float32) * qk_scale, s.dtype)
     Vs = wl.to_storage(rng.standard_normal((s.Hkv, s.L, s.d)).astype(np.float32), s.dtype)
     return Qs, Ks, Vs
+
+
+@pytest.mark.parametrize("rows", [40, 128, 512])
+@pytest.mark.parametrize("lists", ["even_ragged_second", "odd_ragged_alone", "ragged_first", "single"])
+def test_64_token_blocks_are_paired_into_key_tiles(ctx, rows, lists):
+    """KV block 64 on the tensor-core path: two selected blocks share one 128-key tile (two 64-row TMA boxes per
+    half tile).  Block lists with an even and an odd number of blocks, non-adjacent pairs, the short last block of
+    the prompt as the second block of a pair, alone in the last tile, and (list not ascending) as the first of a
+    pair; 40 rows take the one-warpgroup kernel, 128 rows the key-pair form, 512 stacked rows per KV head the
+    two-tile form or the key-pair form depending on the tile count."""
+    M = 64 * 150 + 40                                              # 151 blocks, the last one 40 tokens
+    s = wl.Shape(M + rows, M, 4, 4, 128, 64, "bf16") if rows != 512 else wl.Shape(M + 128, M, 8, 2, 128, 64, "bf16")
+    nb = s.nb
+    assert nb == 151
+    rng = np.random.default_rng(11)
+    pool = np.sort(rng.choice(nb - 1, size=140, replace=False))
+    if lists == "even_ragged_second":
+        blocks = [np.concatenate([pool[:69], [nb - 1]]), pool[10:80]]                 # 70 and 70 blocks
+    elif lists == "odd_ragged_alone":
+        blocks = [np.concatenate([pool[:70], [nb - 1]]), pool[5:76]]                  # 71 and 71 blocks
+    elif lists == "ragged_first":
+        blocks = [np.concatenate([pool[:68], [nb - 1, pool[100]]]), pool[3:73][::-1].copy()]  # short block, then a full one
+    else:
+        blocks = [np.array([nb - 1]), np.array([7])]
+    blocks = (blocks * s.Hkv)[:s.Hkv]
+    C = max(len(b) for b in blocks) + 2
+    bidx = np.full((s.Hkv, C), -1, dtype=np.int32)
+    for g, b in enumerate(blocks):
+        bidx[g, :len(b)] = b
+    sinks = np.sort(rng.choice(s.M, size=70, replace=False)).astype(np.int32)
+    keep = np.array([[0 if (j // s.B) in set(blocks[g].tolist()) else 1 for j in sinks] for g in range(s.Hkv)],
+                    dtype=np.uint8)
+    Qs, Ks, Vs = _rand_qkv(s, 41, qk_scale=1.5)
+    dQ, dK, dV = (fstep.to_device(x, s.dtype) for x in (Qs, Ks, Vs))
+    O = torch.zeros(s.N, s.H, s.d, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(s.H, s.N, dtype=torch.float32, device="cuda")
+    fb.focus_sparse_attn(ctx, fstep.c_shape(s), dQ, s.M, s.N, None, None, 0, dK, dV, fb.HEADS_PER_KV_GROUP,
+                         torch.from_numpy(bidx.reshape(-1)).cuda(), C,
+                         torch.tensor([len(b) for b in blocks], dtype=torch.int32, device="cuda"),
+                         torch.from_numpy(sinks).cuda(), torch.from_numpy(keep.reshape(-1)).cuda(), len(sinks), O, lse)
+    assert ctx.last_attn_variant() in (2, 3, 4)
+    hpg = s.H // s.Hkv
+    scale = 1.0 / math.sqrt(s.d)
+    f64h = lambda a, h, kv=True: wl.storage_to_f64(a[h // hpg:h // hpg + 1] if kv else a[:, h:h + 1], s.dtype)
+    got, got_lse = fstep.from_device(O), fstep.from_device(lse)
+    for h in (0, s.H - 1):
+        Oh, lh = fo.sparse_attn(f64h(Qs, h, False), f64h(Ks, h), f64h(Vs, h), s.M, s.B, [blocks[h // hpg]], sinks, scale)
+        assert max_abs(got[:, h], Oh[:, 0]) <= 2e-2 and rel_rms(got[:, h], Oh[:, 0]) <= 1e-2
+        assert max_abs(got_lse[h], lh[0]) <= 2e-3
+    assert ctx.poll_status() == 0
 
 
 @pytest.mark.parametrize("case", ["dense_split8", "dense_nosplit", "sparse_gqa_split8", "sparse_few_tiles"])
