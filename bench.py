@@ -707,7 +707,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="focus", choices=["focus", "reference"])
-    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--config", type=int, default=2,
+                    help="workload: 2 = the headline 32-layer step; 5 = the paper's own hyper-parameters on that shape")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (quick runs)")
     ap.add_argument("--skip-gen", action="store_true", help="skip the gen-region-rows (tensor-bound) measurements")
     ap.add_argument("--no-graph", action="store_true", help="time eager C-ABI calls instead of a CUDA graph replay")
