@@ -1,31 +1,32 @@
 // Generic SIMT attention (Eq. 9 and FullAttn of Algorithm 1) and the SIMT sink column-sum (Eq. 6).
 // Any dtype (f32, bf16), head_dim 64/128, any block size: this is the fp32 path of the library and the
-// fallback for shapes the tensor-core kernels do not take.  One warp per (query row, head); the lanes of a
-// warp hold 32 different keys during the logit phase and 32 slices of the output during the value phase.
+// fallback for shapes the tensor-core kernels do not take.  One CTA of eight or sixteen warps per (eight query rows, head); the
+// lanes of a warp hold 32 different keys during the logit phase and 32 slices of the output during the value phase.
 #include "focus_common.cuh"
 
-template <typename T, int D>
-__device__ __forceinline__ float dot_row(const float* __restrict__ q, const T* __restrict__ kr) {
-  constexpr int EPC = 16 / sizeof(T);
-  float s = 0.f;
-#pragma unroll 4
-  for (int c = 0; c < D / EPC; ++c) {
-    const uint4 raw = __ldg(reinterpret_cast<const uint4*>(kr) + c);
-    if constexpr (sizeof(T) == 2) {
-      const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const float2 f = __bfloat1622float2(p[e]);
-        s = fmaf(q[c * 8 + 2 * e], f.x, s);
-        s = fmaf(q[c * 8 + 2 * e + 1], f.y, s);
-      }
+// EPL consecutive elements of a V row as floats, one vector load
+template <typename T, int EPL>
+__device__ __forceinline__ void load_slice(const T* __restrict__ p, float (&out)[EPL]) {
+  if constexpr (sizeof(T) == 4) {
+    if constexpr (EPL == 4) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(p));
+      out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
     } else {
-      const float* p = reinterpret_cast<const float*>(&raw);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) s = fmaf(q[c * 4 + e], p[e], s);
+      const float2 v = __ldg(reinterpret_cast<const float2*>(p));
+      out[0] = v.x; out[1] = v.y;
+    }
+  } else {
+    if constexpr (EPL == 4) {
+      const uint2 raw = __ldg(reinterpret_cast<const uint2*>(p));
+      const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+      const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+      out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
+    } else {
+      const uint32_t raw = __ldg(reinterpret_cast<const uint32_t*>(p));
+      const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw));
+      out[0] = a.x; out[1] = a.y;
     }
   }
-  return s;
 }
 
 __device__ __forceinline__ float warp_max(float v) {
@@ -49,57 +50,150 @@ struct SimtParams {
   int32_t* status;
 };
 
-template <typename T, int D>
-__global__ void __launch_bounds__(128) attn_simt_kernel(const SimtParams p) {
+// warps per CTA: sixteen for head_dim 64, eight for 128 (the warps' partial outputs must fit in 48 KB)
+__host__ __device__ constexpr int simt_warps(int d) { return d == 64 ? 16 : 8; }
+// loads in flight per lane in the logit / value phase (deeper unrolling measured no faster: the kernel waits on L2
+// latency with few warps per SM, not on issue slots)
+constexpr int UNROLL_DOT = 2, UNROLL_V = 4;
+
+// One CTA per (group of R query rows, head): the rows of a group share every K and V row that is loaded (without
+// that sharing the kernel is bound by L2 bandwidth: every row would stream the head's whole K and V).  The warps
+// take the 32-key chunks of the key set in turn, each with its own running (max, sum, output) per row; the
+// partials are merged through shared memory at the end.  Lane j of a warp owns key j of the chunk during the logit
+// phase and slice j of the output during the value phase.
+template <typename T, int D, int R>
+__global__ void __launch_bounds__(simt_warps(D) * 32) attn_simt_kernel(const SimtParams p) {
+  constexpr int NW = simt_warps(D), NTH = NW * 32;
   constexpr int EPL = D / 32;
-  __shared__ float qs[4][D];
+  constexpr int EPC = 16 / sizeof(T);                // elements per 16-byte load
+  __shared__ __align__(16) float qs[R][D];
+  __shared__ float part_o[NW][R][D];
+  __shared__ float part_ml[NW][R][2];
+  __shared__ int row_ok[R];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int pair = blockIdx.x * 4 + warp;
-  const int r = pair / p.H, h = pair % p.H;
+  const int r0 = (blockIdx.x / p.H) * R, h = blockIdx.x % p.H;
   const int nrows = p.q_rows ? min(*p.n_rows, p.rows_bound) : p.n_q;
-  if (r >= nrows) return;
-  const int pos = p.q_rows ? p.q_rows[r] : p.q_base + r;
-  if (pos < p.q_base || pos >= p.q_base + p.n_q) {
-    if (lane == 0) set_status(p.status, FOCUS_ERR_INVALID_ARG);
-    return;
+  if (r0 >= nrows) return;
+  if (threadIdx.x < R) {
+    const int r = r0 + threadIdx.x;
+    int ok = 0;
+    if (r < nrows) {
+      const int pos = p.q_rows ? p.q_rows[r] : p.q_base + r;
+      ok = pos >= p.q_base && pos < p.q_base + p.n_q;
+      if (!ok) set_status(p.status, FOCUS_ERR_INVALID_ARG);
+    }
+    row_ok[threadIdx.x] = ok;
   }
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < R * D; idx += NTH) {
+    const int i = idx / D, c = idx % D;
+    float v = 0.f;
+    if (row_ok[i]) {
+      const int pos = p.q_rows ? p.q_rows[r0 + i] : p.q_base + r0 + i;
+      v = load_as_float((const T*)p.Q + (long long)(pos - p.q_base) * p.q_stride_row + (long long)h * p.q_stride_head + c);
+    }
+    qs[i][c] = v;
+  }
+  __syncthreads();
   const int g = h / p.hpg;
-  const T* qrow = (const T*)p.Q + (long long)(pos - p.q_base) * p.q_stride_row + (long long)h * p.q_stride_head;
-  for (int c = lane; c < D; c += 32) qs[warp][c] = load_as_float(qrow + c);
-  __syncwarp();
   const T* Kg = (const T*)p.K + (long long)g * p.kv_stride_head;
   const T* Vg = (const T*)p.V + (long long)g * p.kv_stride_head;
   const bool want_o = p.O != nullptr;
-  float m = -INFINITY, l = 0.f, o[EPL];
+  float m[R], l[R], o[R][EPL];
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) o[e] = 0.f;
+  for (int i = 0; i < R; ++i) {
+    m[i] = -INFINITY; l[i] = 0.f;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) o[i][e] = 0.f;
+  }
+  int chunk = 0;                                     // chunk counter, the same in every warp
+  auto mine = [&]() { return (chunk++ % NW) == warp; };
 
   auto step = [&](int key) {
-    float s = -INFINITY;
-    if (key >= 0) s = dot_row<T, D>(qs[warp], Kg + (long long)key * p.kv_stride_tok) * p.scale;
-    const float mx = warp_max(s);
-    if (mx == -INFINITY) return;
-    const float m_new = fmaxf(m, mx);
-    const float corr = expf(m - m_new);
-    const float pj = key >= 0 ? expf(s - m_new) : 0.f;
-    l = l * corr + warp_sum(pj);
-    m = m_new;
-    if (want_o) {
+    float s[R];
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) o[e] *= corr;
+    for (int i = 0; i < R; ++i) s[i] = 0.f;
+    if (key >= 0) {
+      const uint4* kr = reinterpret_cast<const uint4*>(Kg + (long long)key * p.kv_stride_tok);
+#pragma unroll UNROLL_DOT
+      for (int c = 0; c < D / EPC; ++c) {
+        const uint4 raw = __ldg(kr + c);
+        float kf[EPC];
+        if constexpr (sizeof(T) == 2) {
+          const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) { const float2 f = __bfloat1622float2(pb[e]); kf[2 * e] = f.x; kf[2 * e + 1] = f.y; }
+        } else {
+          kf[0] = __uint_as_float(raw.x); kf[1] = __uint_as_float(raw.y);
+          kf[2] = __uint_as_float(raw.z); kf[3] = __uint_as_float(raw.w);
+        }
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+#pragma unroll
+          for (int e4 = 0; e4 < EPC; e4 += 4) {
+            const float4 q4 = *reinterpret_cast<const float4*>(&qs[i][c * EPC + e4]);   // same address in every lane
+            s[i] = fmaf(q4.x, kf[e4], s[i]); s[i] = fmaf(q4.y, kf[e4 + 1], s[i]);
+            s[i] = fmaf(q4.z, kf[e4 + 2], s[i]); s[i] = fmaf(q4.w, kf[e4 + 3], s[i]);
+          }
+        }
+      }
+    }
+    // row maxima and row sums of the R rows as interleaved butterflies (R independent shuffles per level)
+    float si[R], mx[R], pj[R], corr[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i) { si[i] = key >= 0 ? s[i] * p.scale : -INFINITY; mx[i] = si[i]; }
+#pragma unroll
+    for (int ofs = 16; ofs > 0; ofs >>= 1) {
+#pragma unroll
+      for (int i = 0; i < R; ++i) mx[i] = fmaxf(mx[i], __shfl_xor_sync(0xffffffffu, mx[i], ofs));
+    }
+    bool any = false;
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+      pj[i] = 0.f; corr[i] = 1.f;
+      if (mx[i] != -INFINITY) {                      // warp-uniform
+        any = true;
+        const float m_new = fmaxf(m[i], mx[i]);
+        corr[i] = expf(m[i] - m_new);
+        pj[i] = key >= 0 ? expf(si[i] - m_new) : 0.f;
+        m[i] = m_new;
+      }
+    }
+    float ps[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i) ps[i] = pj[i];
+#pragma unroll
+    for (int ofs = 16; ofs > 0; ofs >>= 1) {
+#pragma unroll
+      for (int i = 0; i < R; ++i) ps[i] += __shfl_xor_sync(0xffffffffu, ps[i], ofs);
+    }
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+      l[i] = l[i] * corr[i] + ps[i];
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) o[i][e] *= corr[i];
+    }
+    if (want_o && any) {
+      // the 32 V rows of the chunk, sixteen loads in flight; an absent key reads row 0 and is discarded
+#pragma unroll UNROLL_V
       for (int jj = 0; jj < 32; ++jj) {
-        const float pk = __shfl_sync(0xffffffffu, pj, jj);
         const int kk = __shfl_sync(0xffffffffu, key, jj);
-        if (kk >= 0) {
-          const T* vr = Vg + (long long)kk * p.kv_stride_tok + lane * EPL;
+        float v[EPL];
+        load_slice<T, EPL>(Vg + (long long)max(kk, 0) * p.kv_stride_tok + lane * EPL, v);
 #pragma unroll
-          for (int e = 0; e < EPL; ++e) o[e] = fmaf(pk, load_as_float(vr + e), o[e]);
+        for (int e = 0; e < EPL; ++e) v[e] = kk >= 0 ? v[e] : 0.f;
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+          const float pk = __shfl_sync(0xffffffffu, pj[i], jj);
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) o[i][e] = fmaf(pk, v[e], o[i][e]);
         }
       }
     }
   };
   auto span = [&](int lo, int hi) {
-    for (int j0 = lo; j0 < hi; j0 += 32) step(j0 + lane < hi ? j0 + lane : -1);
+    for (int j0 = lo; j0 < hi; j0 += 32)
+      if (mine()) step(j0 + lane < hi ? j0 + lane : -1);
   };
 
   if (p.dense) {
@@ -110,12 +204,13 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(const SimtParams p) {
     for (int bi = 0; bi < cnt; ++bi) {
       const int b = p.block_idx[(size_t)row * p.max_blocks + bi];
       if (b < 0 || b >= p.nb) {
-        if (lane == 0) set_status(p.status, FOCUS_ERR_INVALID_ARG);
+        if (threadIdx.x == 0) set_status(p.status, FOCUS_ERR_INVALID_ARG);
         continue;
       }
       span(b * p.B, min((b + 1) * p.B, p.M));
     }
     for (int s0 = 0; s0 < p.n_sink; s0 += 32) {
+      if (!mine()) continue;
       const int s = s0 + lane;
       int key = -1;
       if (s < p.n_sink && p.sink_keep[(size_t)row * p.n_sink + s]) {
@@ -131,19 +226,38 @@ __global__ void __launch_bounds__(128) attn_simt_kernel(const SimtParams p) {
     }
     span(p.M, p.L);
   }
-  if (want_o) {
-    const float inv = l > 0.f ? 1.f / l : 0.f;
-    if constexpr (sizeof(T) == 2) {
-      __nv_bfloat16* orow = (__nv_bfloat16*)p.O + ((size_t)r * p.H + h) * D + lane * EPL;
+  // merge of the warps' partials, warps in index order
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) orow[e] = __float2bfloat16_rn(o[e] * inv);
-    } else {
-      float* orow = (float*)p.O + ((size_t)r * p.H + h) * D + lane * EPL;
+  for (int i = 0; i < R; ++i) {
+    if (lane == 0) { part_ml[warp][i][0] = m[i]; part_ml[warp][i][1] = l[i]; }
+    if (want_o) {
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) orow[e] = o[e] * inv;
+      for (int e = 0; e < EPL; ++e) part_o[warp][i][lane * EPL + e] = o[i][e];
     }
   }
-  if (p.lse && lane == 0) p.lse[(size_t)h * p.lse_stride + r] = m + logf(l);
+  __syncthreads();
+  for (int idx = threadIdx.x; idx < R * D; idx += NTH) {
+    const int i = idx / D, c = idx % D;
+    if (!row_ok[i]) continue;
+    float mm = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < NW; ++w)
+      if (part_ml[w][i][1] > 0.f) mm = fmaxf(mm, part_ml[w][i][0]);
+    float acc = 0.f, tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) {
+      const float wgt = part_ml[w][i][1] > 0.f ? expf(part_ml[w][i][0] - mm) : 0.f;
+      tot += wgt * part_ml[w][i][1];
+      if (want_o && wgt > 0.f) acc = fmaf(wgt, part_o[w][i][c], acc);
+    }
+    const int r = r0 + i;
+    if (want_o) {
+      const float outv = tot > 0.f ? acc / tot : 0.f;
+      if constexpr (sizeof(T) == 2) ((__nv_bfloat16*)p.O)[((size_t)r * p.H + h) * D + c] = __float2bfloat16_rn(outv);
+      else ((float*)p.O)[((size_t)r * p.H + h) * D + c] = outv;
+    }
+    if (p.lse && c == 0) p.lse[(size_t)h * p.lse_stride + r] = mm + logf(tot);
+  }
 }
 
 focus_status launch_attn_simt(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st) {
@@ -157,16 +271,16 @@ focus_status launch_attn_simt(focus_ctx* ctx, const AttnArgs& a, cudaStream_t st
   p.hpg = a.sh.n_q_heads / a.sh.n_kv_heads; p.B = a.sh.kv_block; p.nb = shape_nb(&a.sh); p.dense = a.dense;
   p.group_stride = a.group_stride; p.max_blocks = a.max_blocks; p.n_sink = a.n_sink; p.lse_stride = a.lse_stride;
   p.scale = a.scale; p.status = ctx->d_status;
-  const long long pairs = (long long)a.max_rows * a.sh.n_q_heads;
-  if (pairs == 0) return FOCUS_OK;
-  const unsigned grid = (unsigned)((pairs + 3) / 4);
+  if (a.max_rows == 0) return FOCUS_OK;
+  constexpr int R = 8;                               // query rows per CTA
+  const unsigned grid = (unsigned)(((long long)a.max_rows + R - 1) / R * a.sh.n_q_heads);
   const bool bf = a.sh.dtype == FOCUS_BF16;
   if (a.sh.head_dim == 128) {
-    if (bf) attn_simt_kernel<__nv_bfloat16, 128><<<grid, 128, 0, st>>>(p);
-    else attn_simt_kernel<float, 128><<<grid, 128, 0, st>>>(p);
+    if (bf) attn_simt_kernel<__nv_bfloat16, 128, R><<<grid, simt_warps(128) * 32, 0, st>>>(p);
+    else attn_simt_kernel<float, 128, R><<<grid, simt_warps(128) * 32, 0, st>>>(p);
   } else {
-    if (bf) attn_simt_kernel<__nv_bfloat16, 64><<<grid, 128, 0, st>>>(p);
-    else attn_simt_kernel<float, 64><<<grid, 128, 0, st>>>(p);
+    if (bf) attn_simt_kernel<__nv_bfloat16, 64, R><<<grid, simt_warps(64) * 32, 0, st>>>(p);
+    else attn_simt_kernel<float, 64, R><<<grid, simt_warps(64) * 32, 0, st>>>(p);
   }
   FOCUS_CHECK_LAUNCH();
   return FOCUS_OK;
