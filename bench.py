@@ -397,6 +397,14 @@ def run_focus(args):
     if graph is not None:
         dense_graph_ms = per_launch_in_graph("active", "dense", K)
         sparse_graph_ms = per_launch_in_graph("active", "sparse", K)
+    # practical read ceiling: the library's read-only streaming probe over two 2 GiB buffers in turn (launch gaps
+    # are 2 % of a pass of that size), per pass inside a graph
+    probe_out = torch.zeros(1, dtype=torch.int32, device="cuda")
+    probe_bytes = 2 << 30
+    probe_bufs = [torch.randint(0, 255, (probe_bytes,), dtype=torch.uint8, device="cuda") for _ in range(2)]
+    stream_gbs = probe_bytes / (graph_time_us(lambda l: fb.focus_stream_read(ctx, probe_bufs[l], probe_bytes, probe_out),
+                                              2, warm=3, reps=20) * 1e-6) / 1e9
+    del probe_bufs
     eb = 2
     kv_bytes = 2 * s.Hkv * s.L * s.d * eb
     na = int(results["active"]["b"].n_active.item())
@@ -510,6 +518,7 @@ def run_focus(args):
                    "dense_layer_eager_marks_ms": dense_eager_ms, "sparse_layer_eager_marks_ms": sparse_eager_ms},
         "roofline": {"bound": "hbm", "achieved": dense_gbs, "peak": P["hbm"], "unit": "GB/s", "frac": dense_gbs / P["hbm"],
                      "traffic": traffic, "kernel": "attn_tc_kernel incl. its in-cluster split merge (dense layer, I_active rows)",
+                     "read_only_stream_GBps": stream_gbs, "frac_of_read_only_stream": dense_gbs / stream_gbs,
                      "bytes_per_launch": kv_bytes + qo_bytes, "peak_source": f"{P['src']} copy bandwidth"},
         "gen_mode": gen,
         "e2e": {"value": ms_e2e, "unit": "ms", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
@@ -521,6 +530,28 @@ def run_focus(args):
     if cpu:
         out["cpu_baseline"] = cpu
     print(json.dumps(out))
+
+
+def graph_time_us(fn, n_layers, warm=10, reps=50):
+    """Per-call latency in microseconds of fn(l), l = 0..n_layers-1 (rotating layer copies, so that the inputs of a
+    call are not in L2 from the call before), replayed as one CUDA graph: `warm` untimed replays, then `reps` replays
+    timed one by one with CUDA events; the median replay divided by the calls per replay."""
+    import torch
+    for l in range(n_layers):
+        fn(l)
+    torch.cuda.synchronize()
+    gr = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(gr):
+        for l in range(n_layers):
+            fn(l)
+    for _ in range(warm):
+        gr.replay()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, z in evs:
+        a.record(); gr.replay(); z.record()
+    torch.cuda.synchronize()
+    return statistics.median(a.elapsed_time(z) for a, z in evs) / n_layers * 1e3
 
 
 def run_sweep(args):
@@ -553,24 +584,7 @@ def run_sweep(args):
         masked = torch.from_numpy(wl.gen_masked(w0)).cuda()
 
         def graph_time(fn):
-            for l in range(NL):
-                fn(l)
-            torch.cuda.synchronize()
-            gr = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gr):
-                for l in range(NL):
-                    fn(l)
-            for _ in range(3):
-                gr.replay()
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            reps = max(3, min(20, int(2e-3 * 1e9 / layer_bytes) + 3))
-            e0.record()
-            for _ in range(reps):
-                gr.replay()
-            e1.record()
-            torch.cuda.synchronize()
-            return e0.elapsed_time(e1) / reps / NL * 1e3          # us per call
+            return graph_time_us(fn, NL)
 
         for rows in ("gen", "active"):
             dense_us = None
@@ -609,7 +623,8 @@ def run_sweep(args):
                 assert ctx.poll_status() == 0
         del Qs, Ks, Vs
         torch.cuda.empty_cache()
-    print(json.dumps({"sweep": out, "peaks": P}))
+    print(json.dumps({"sweep": out, "peaks": P,
+                      "timing": "median of 50 CUDA-graph replays after 10 warm-up replays, per call"}))
 
 
 def run_stages(args):
@@ -653,27 +668,12 @@ def run_stages(args):
     torch.cuda.synchronize()
 
     def graph_time(fn):
-        for l in range(NL):
-            fn(l)
-        torch.cuda.synchronize()
-        gr = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(gr):
-            for l in range(NL):
-                fn(l)
-        for _ in range(3):
-            gr.replay()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(20):
-            gr.replay()
-        e1.record()
-        torch.cuda.synchronize()
-        return round(e0.elapsed_time(e1) / 20 / NL * 1e3, 2)
+        return round(graph_time_us(fn, NL), 2)
 
     na = int(ba.n_active.item())
     keys = w.C * s.B + w.n_sink + s.N
-    out = {"workload": w.name, "n_active": na, "retained_keys_per_head": keys, "layers_rotated": NL, "us": {}}
+    out = {"workload": w.name, "n_active": na, "retained_keys_per_head": keys, "layers_rotated": NL,
+           "timing": "median of 50 CUDA-graph replays after 10 warm-up replays, per call", "us": {}}
     u = out["us"]
     u["select_queries"] = graph_time(lambda l: fstep.select_queries(ctx, ba, conf, masked))
     u["find_sinks (with LSE of the dense pass)"] = graph_time(lambda l: fstep.find_sinks(ctx, ba, Qs[l], Ks[l], lse_keep))

@@ -113,6 +113,13 @@ int32_t focus_set_force_simt(focus_ctx* ctx, int32_t force);
  * FOCUS_ERR_TIMEOUT and the context must still be usable.  Nothing else is touched.  Errors: INVALID_ARG. */
 focus_status focus_selftest_bounded_wait(focus_ctx* ctx, int32_t limit_us, focus_stream stream);
 
+/* Measurement aid (no counterpart in the paper): streams the `bytes` bytes at device pointer `ptr` once, read only,
+ * with 128-bit loads from every SM, and leaves the 32-bit xor of all 32-bit words read in *checksum (device memory,
+ * overwritten).  Its bandwidth is the practical HBM read ceiling on the device at hand, which the figures of the
+ * HBM-bound kernels are put beside.  ptr must be 16-byte aligned and bytes a multiple of 16 (0 is allowed: checksum
+ * 0).  One memset and one launch on `stream`; the buffer stays the caller's.  Errors: INVALID_ARG, CUDA. */
+focus_status focus_stream_read(focus_ctx* ctx, const void* ptr, size_t bytes, uint32_t* checksum, focus_stream stream);
+
 /* ---- stage 1: past-confidence indicator (Eq. 4) and window expansion (Eq. 5) ---------------- */
 
 /* I_focus = the k positions i in [blk_lo, blk_hi) with masked[i] != 0 that have the highest

@@ -43,6 +43,7 @@ _SIGS = {
     "focus_status_string": (C.c_char_p, [_I]),
     "focus_set_force_simt": (_I, [_P, _I]),
     "focus_selftest_bounded_wait": (_I, [_P, _I, _P]),
+    "focus_stream_read": (_I, [_P, _P, _Z, _P, _P]),
     "focus_launch_count": (C.c_uint64, []),
     "focus_last_attn_variant": (_I, [_P]),
     "focus_select_queries": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P, _P, _P, _P, _P]),
@@ -151,6 +152,12 @@ class Context:
         reports ERR_TIMEOUT afterwards."""
         _check(self._lib.focus_selftest_bounded_wait(self.handle, int(limit_us), _stream(stream)),
                "focus_selftest_bounded_wait")
+
+
+def focus_stream_read(ctx, buf, nbytes, checksum, stream=None):
+    """Read-only pass over nbytes of `buf`; the xor of its 32-bit words lands in checksum[0] (uint32 / int32 tensor)."""
+    _check(ctx._lib.focus_stream_read(ctx.handle, _ptr(buf), int(nbytes), _ptr(checksum), _stream(stream)),
+           "focus_stream_read")
 
 
 def focus_launch_count() -> int:

@@ -56,6 +56,10 @@ def test_argument_errors_need_no_device(lib):
     assert lib.focus_dense_attn(null, ctypes.byref(sh), null, 0, 0, null, null, 0, null, null, null, null, null) == fb.ERR_INVALID_ARG
 
 
+def test_stream_read_rejects_bad_arguments_on_the_host(lib):
+    assert lib.focus_stream_read(None, None, 0, None, None) == fb.ERR_INVALID_ARG            # no context
+
+
 def test_no_device_means_loud_failure(lib):
     import torch
     if torch.cuda.is_available():

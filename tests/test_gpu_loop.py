@@ -99,3 +99,21 @@ def test_update_kv_bit_exact(ctx, dtype, d, Hkv):
     rows[0] = s.L + 5
     fb.focus_update_kv(ctx, fstep.c_shape(s), dK, dV, fstep.to_device(Kn, dtype), fstep.to_device(Vn, dtype), rows, n_rows, 40)
     assert ctx.poll_status() == fb.ERR_INVALID_ARG
+
+
+@pytest.mark.gpu
+def test_stream_read_probe_checksum_is_exact(ctx):
+    """The read-only streaming probe xors every 32-bit word it reads: compared bit for bit with numpy on sizes
+    below one vector per thread, with a ragged tail of the unrolled loop, and of several grid strides."""
+    rng = np.random.default_rng(5)
+    out = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for n_words in (0, 4, 4 * 1000, 4 * (148 * 8 * 256 * 8 + 12345), 4 * 3_000_001):
+        host = rng.integers(0, 2 ** 32, size=n_words, dtype=np.uint32)
+        dev = torch.from_numpy(host.view(np.int32)).cuda() if n_words else torch.zeros(4, dtype=torch.int32, device="cuda")
+        fb.focus_stream_read(ctx, dev, n_words * 4, out)
+        torch.cuda.synchronize()
+        want = int(np.bitwise_xor.reduce(host)) if n_words else 0
+        assert int(out.cpu().numpy().view(np.uint32)[0]) == want
+    with pytest.raises(fb.FocusError):
+        fb.focus_stream_read(ctx, dev, 24, out)                     # not a multiple of 16 bytes
+    assert ctx.poll_status() == 0
