@@ -348,6 +348,46 @@ def test_64_token_blocks_are_paired_into_key_tiles(ctx, rows, lists):
     assert ctx.poll_status() == 0
 
 
+@pytest.mark.parametrize("rows", [40, 128, 256])
+@pytest.mark.parametrize("B", [128, 64])
+def test_block_lists_too_long_to_stage_in_shared_memory(ctx, B, rows):
+    """A split with more key tiles than the shared-memory tile list holds (128, or 96 in the three-warpgroup
+    kernels) derives every tile from the block list in global memory instead.  One head, every block of a 140K-token
+    prompt but a few selected: ~137 key tiles for each of the 8 splits, with both block sizes (64-token blocks are
+    paired) and all three kernel forms (40, 128, 256 rows)."""
+    nblk128 = 1100
+    M = 128 * nblk128 + 50                                         # the last block is short
+    s = wl.Shape(M + rows, M, 1, 1, 128, B, "bf16")
+    nb = s.nb
+    rng = np.random.default_rng(13)
+    drop = set(rng.choice(nb - 1, size=7, replace=False).tolist())
+    blocks = [np.array([b for b in range(nb) if b not in drop])]
+    C = nb
+    bidx = np.full((1, C), -1, dtype=np.int32)
+    bidx[0, :len(blocks[0])] = blocks[0]
+    sinks = np.sort(rng.choice(s.M, size=40, replace=False)).astype(np.int32)
+    keep = np.array([[0 if (j // s.B) in set(blocks[0].tolist()) else 1 for j in sinks]], dtype=np.uint8)
+    Qs, Ks, Vs = _rand_qkv(s, 43, qk_scale=1.5)
+    dQ, dK, dV = (fstep.to_device(x, s.dtype) for x in (Qs, Ks, Vs))
+    O = torch.zeros(s.N, s.H, s.d, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(s.H, s.N, dtype=torch.float32, device="cuda")
+    big = fb.Context(0, workspace_bytes=64 << 20)
+    try:
+        fb.focus_sparse_attn(big, fstep.c_shape(s), dQ, s.M, s.N, None, None, 0, dK, dV, fb.HEADS_PER_KV_GROUP,
+                             torch.from_numpy(bidx.reshape(-1)).cuda(), C,
+                             torch.tensor([len(blocks[0])], dtype=torch.int32, device="cuda"),
+                             torch.from_numpy(sinks).cuda(), torch.from_numpy(keep.reshape(-1)).cuda(), len(sinks), O, lse)
+        assert big.last_attn_variant() == {40: 2, 128: 4, 256: 3}[rows]
+        assert big.poll_status() == 0
+    finally:
+        big.close()
+    f64 = lambda a: wl.storage_to_f64(a, s.dtype)
+    Oh, lh = fo.sparse_attn(f64(Qs), f64(Ks), f64(Vs), s.M, s.B, blocks, sinks, 1.0 / math.sqrt(s.d))
+    got, got_lse = fstep.from_device(O), fstep.from_device(lse)
+    assert max_abs(got[:, 0], Oh[:, 0]) <= 2e-2 and rel_rms(got[:, 0], Oh[:, 0]) <= 1e-2
+    assert max_abs(got_lse[0], lh[0]) <= 2e-3
+
+
 @pytest.mark.parametrize("case", ["dense_split8", "dense_nosplit", "sparse_gqa_split8", "sparse_few_tiles"])
 def test_key_pair_kernel(ctx, case):
     """Shapes that take the key-pair attention kernel (one 128-row query tile, two softmax warpgroups on alternating
