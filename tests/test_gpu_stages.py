@@ -348,6 +348,34 @@ def test_64_token_blocks_are_paired_into_key_tiles(ctx, rows, lists):
     assert ctx.poll_status() == 0
 
 
+@pytest.mark.parametrize("B", [128, 64])
+def test_bad_block_index_on_the_tensor_core_path_is_reported_not_dereferenced(ctx, B):
+    """An out-of-range or negative entry inside the counted part of a block list masks its key tile (with 64-token
+    blocks: the pair it belongs to) and raises INVALID_ARG in the status word; the output stays finite and the
+    context usable."""
+    s = wl.Shape(6000 + 40, 6000, 4, 4, 128, B, "bf16")
+    rng = np.random.default_rng(17)
+    good = np.sort(rng.choice(s.nb, size=9, replace=False)).astype(np.int32)
+    Qs, Ks, Vs = _rand_qkv(s, 47)
+    dQ, dK, dV = (fstep.to_device(x, s.dtype) for x in (Qs, Ks, Vs))
+    sinks = np.sort(rng.choice(s.M, size=20, replace=False)).astype(np.int32)
+    for bad in (10 ** 6, -5):
+        lst = good.copy()
+        lst[4] = bad
+        bidx = np.tile(lst, (s.Hkv, 1))
+        keep = np.ones((s.Hkv, len(sinks)), dtype=np.uint8)
+        O = torch.full((s.N, s.H, s.d), 7.0, dtype=torch.bfloat16, device="cuda")
+        lse = torch.zeros(s.H, s.N, dtype=torch.float32, device="cuda")
+        fb.focus_sparse_attn(ctx, fstep.c_shape(s), dQ, s.M, s.N, None, None, 0, dK, dV, fb.HEADS_PER_KV_GROUP,
+                             torch.from_numpy(bidx.reshape(-1)).cuda(), len(lst),
+                             torch.full((s.Hkv,), len(lst), dtype=torch.int32, device="cuda"),
+                             torch.from_numpy(sinks).cuda(), torch.from_numpy(keep.reshape(-1)).cuda(), len(sinks), O, lse)
+        assert ctx.last_attn_variant() == 2
+        assert ctx.poll_status() == fb.ERR_INVALID_ARG
+        assert torch.isfinite(O.float()).all() and torch.isfinite(lse).all()
+    assert ctx.poll_status() == 0
+
+
 @pytest.mark.parametrize("rows", [40, 128, 256])
 @pytest.mark.parametrize("B", [128, 64])
 def test_block_lists_too_long_to_stage_in_shared_memory(ctx, B, rows):
