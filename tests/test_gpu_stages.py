@@ -348,6 +348,74 @@ def test_64_token_blocks_are_paired_into_key_tiles(ctx, rows, lists):
     assert ctx.poll_status() == 0
 
 
+@pytest.mark.parametrize("cfg", [SHAPES[0], SHAPES[3], SHAPES[5]])
+def test_token_major_cache_and_padded_query_rows(ctx, cfg):
+    """Strides are part of the shape: K/V cache stored token-major ([L, Hkv, d]: token stride Hkv*d, head stride d)
+    and Q rows padded (row stride H*d + 64).  Every stage must give bit for bit what it gives on the contiguous
+    layout (same arithmetic, other addresses), which the other tests tie to the oracle; the sparse-layer output is
+    also checked against the oracle directly."""
+    dtype, d, B, H, Hkv = cfg
+    w = small_workload(dtype, d, B, H=H, Hkv=Hkv, n_sink=150, C=4, seed=9)
+    s = w.shape
+    host, dev = make_inputs(w)
+    ora = oracle_chain(w, host, fb.HEADS_PER_KV_GROUP, fb.SINK_TOKENS)
+    Kt = dev["K"].permute(1, 0, 2).contiguous()                    # [L, Hkv, d]
+    Vt = dev["V"].permute(1, 0, 2).contiguous()
+    Qp = torch.zeros(s.N, H * d + 64, dtype=dev["Q"].dtype, device="cuda")
+    Qp[:, :H * d] = dev["Q"].reshape(s.N, H * d)
+    strided = fb.make_shape(s.L, s.M, H, Hkv, d, B, fb.F32 if dtype == "f32" else fb.BF16,
+                            q_stride_row=H * d + 64, q_stride_head=d, kv_stride_tok=Hkv * d, kv_stride_head=d)
+    rng = np.random.default_rng(3)
+    results = []
+    for layout in ("contiguous", "strided"):
+        Q, K, V = (dev["Q"], dev["K"], dev["V"]) if layout == "contiguous" else (Qp, Kt, Vt)
+        b = fstep.StepBuffers(w)
+        if layout == "strided":
+            b.shape = strided
+        fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
+        fstep.dense_layer(ctx, b, Q, K, V)
+        dense = (b.O.clone(), b.lse.clone())
+        fstep.find_sinks(ctx, b, Q, K, b.lse)
+        Kbar = torch.zeros(Hkv, s.nb, d, dtype=torch.float32, device="cuda")
+        fb.focus_pool_keys(ctx, b.shape, K, Kbar)
+        fb.focus_score_blocks(ctx, b.shape, Q, s.M, b.focus_idx, b.n_focus, max(1, w.k), K, None, fb.HEADS_PER_KV_GROUP, b.R)
+        R_cold = b.R.clone()
+        outs = []
+        for fused in (False, True):
+            fstep.sparse_layer(ctx, b, Q, K, V, Kbar=Kbar, fused=fused)
+            outs.append((b.O.clone(), b.lse.clone(), b.block_idx.clone(), b.sink_keep.clone(), b.R.clone()))
+        # Eq. 3 refresh of the active rows in the layout at hand
+        na = b.n_active.item()
+        Kn = torch.from_numpy(rng.standard_normal((b.max_active, Hkv, d)).astype(np.float32)).cuda().to(K.dtype)
+        Kc, Vc = K.clone(), V.clone()
+        fb.focus_update_kv(ctx, b.shape, Kc, Vc, Kn, Kn, b.active_idx, b.n_active, b.max_active)
+        if layout == "strided":
+            Kc, Vc = Kc.permute(1, 0, 2).contiguous(), Vc.permute(1, 0, 2).contiguous()
+        torch.cuda.synchronize()
+        assert ctx.poll_status() == 0
+        results.append(dict(dense=dense, sinks=b.sink_idx.clone(), scores=b.sink_scores.clone(), Kbar=Kbar, R_cold=R_cold,
+                            outs=outs, Kc=Kc, Vc=Vc, na=na, active=b.active_idx.clone()))
+        rng = np.random.default_rng(3)                              # the same new rows for the second layout
+    a, z = results
+    assert torch.equal(a["active"], z["active"]) and torch.equal(a["sinks"], z["sinks"])
+    for x, y in zip(a["dense"], z["dense"]):
+        assert torch.equal(x, y)
+    assert torch.equal(a["scores"], z["scores"]) and torch.equal(a["Kbar"], z["Kbar"]) and torch.equal(a["R_cold"], z["R_cold"])
+    for oa, oz in zip(a["outs"], z["outs"]):
+        for x, y in zip(oa, oz):
+            assert torch.equal(x, y)
+    assert torch.equal(a["Kc"], z["Kc"]) and torch.equal(a["Vc"], z["Vc"])
+    # and the strided sparse layer against the oracle
+    na = z["na"]
+    bi = z["outs"][1][2].cpu().numpy().reshape(Hkv, -1)
+    blocks = [bi[g][bi[g] >= 0] for g in range(Hkv)]
+    Os, lses = fo.sparse_attn(host["Q"][ora["active"] - s.M], host["K"], host["V"], s.M, s.B, blocks,
+                              z["sinks"].cpu().numpy(), ora["scale"])
+    got = fstep.from_device(z["outs"][1][0])[:na]
+    assert max_abs(got, Os) <= TOL_ABS[dtype] and rel_rms(got, Os) <= TOL_RMS[dtype]
+    assert max_abs(fstep.from_device(z["outs"][1][1])[:, :na], lses) <= TOL_LSE[dtype]
+
+
 @pytest.mark.parametrize("B", [128, 64])
 def test_bad_block_index_on_the_tensor_core_path_is_reported_not_dereferenced(ctx, B):
     """An out-of-range or negative entry inside the counted part of a block list masks its key tile (with 64-token
