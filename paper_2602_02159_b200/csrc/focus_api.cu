@@ -109,8 +109,9 @@ extern "C" focus_status focus_workspace_bytes(const focus_shape* shape, int32_t 
   size_t sink = H * L * 4 + L * 4 + H * (size_t)n_q * 4 + (size_t)n_q * H * shape->head_dim * 2 + 4096;
   size_t score = (size_t)shape->n_kv_heads * (shape->head_dim + shape_nb(shape)) * 4 + 1024;
   size_t attn = attn_tc_workspace(shape, n_q, max_blocks, n_sink);
-  size_t m = sink > score ? sink : score;
-  *out_bytes = (m > attn ? m : attn) + 4096;
+  // focus_find_sinks without a log-sum-exp runs an attention pass on top of its own buffers: the two add up
+  size_t m = sink + attn;
+  *out_bytes = (m > score ? m : score) + 4096;
   return FOCUS_OK;
 }
 

@@ -699,6 +699,44 @@ def test_host_side_argument_matrix(ctx):
     tiny.close()
 
 
+@pytest.mark.parametrize("merge", [None, "counters", "kernel"])
+@pytest.mark.parametrize("cfg", [SHAPES[1], SHAPES[3], SHAPES[5]])
+def test_a_context_of_exactly_the_advertised_workspace_runs_every_stage(cfg, merge, monkeypatch):
+    """focus_workspace_bytes is a promise: a context created with that many bytes must carry every call on the
+    shape — sink identification with and without a log-sum-exp from a dense pass, pooling, cold and warm scoring,
+    selection, attention in both row modes, the fused layer — also when the key splits merge through global
+    memory (forced)."""
+    dtype, d, B, H, Hkv = cfg
+    w = small_workload(dtype, d, B, H=H, Hkv=Hkv, L=5200, M=4500, n_sink=150, C=9, seed=12)
+    s = w.shape
+    host, dev = make_inputs(w)
+    need = fb.focus_workspace_bytes(fstep.c_shape(s), s.N, w.C, w.n_sink)
+    if merge:
+        monkeypatch.setenv("FOCUS_MERGE", merge)
+    c = fb.Context(0, workspace_bytes=need)
+    try:
+        Kbar = torch.zeros(Hkv, s.nb, d, dtype=torch.float32, device="cuda")
+        for rows in ("active", "gen"):
+            b = fstep.StepBuffers(w, rows=rows)
+            fstep.select_queries(c, b, dev["conf"], dev["masked"])
+            fstep.dense_layer(c, b, dev["Q"], dev["K"], dev["V"])
+            fstep.find_sinks(c, b, dev["Q"], dev["K"], None)
+            no_lse = b.sink_idx.clone()
+            if rows == "active":
+                fstep.find_sinks(c, b, dev["Q"], dev["K"], b.lse)
+                assert torch.equal(no_lse, b.sink_idx)
+            fb.focus_pool_keys(c, b.shape, dev["K"], Kbar)
+            fstep.sparse_layer(c, b, dev["Q"], dev["K"], dev["V"], Kbar=None, fused=False)       # cold scoring
+            cold = b.O.clone()
+            fstep.sparse_layer(c, b, dev["Q"], dev["K"], dev["V"], Kbar=Kbar, fused=False)
+            fstep.sparse_layer(c, b, dev["Q"], dev["K"], dev["V"], Kbar=Kbar, fused=True)
+            torch.cuda.synchronize()
+            assert c.poll_status() == 0
+            assert (cold.float() - b.O.float()).abs().max().item() <= 2e-2
+    finally:
+        c.close()
+
+
 @pytest.mark.parametrize("case", ["all_equal", "duplicated_keys", "random"])
 def test_sink_selection_on_a_long_candidate_range(ctx, case):
     """A candidate range long enough for the multi-CTA selection (16 000 prompt positions).  The selected set must be
