@@ -813,20 +813,33 @@ def test_block_selection_with_many_blocks_and_cut_ties(ctx, nb, C):
     assert np.array_equal(skeep.cpu().numpy().reshape(G, 40), keep)
 
 
-def test_results_are_deterministic(ctx):
-    w = small_workload("bf16", 128, 128, H=8, Hkv=2)
+@pytest.mark.parametrize("case", ["small_active", "llada_8k_gen", "sweep_32k_gen", "block64_gen"])
+def test_results_are_deterministic(ctx, case):
+    """Same inputs, same bits, run after run: the small GQA shape on the one-warpgroup kernel, and full-size
+    gen-row launches on the two-tile and key-pair forms with their in-cluster split merges."""
+    if case == "small_active":
+        w, rows = small_workload("bf16", 128, 128, H=8, Hkv=2), "active"
+    elif case == "llada_8k_gen":
+        w, rows = wl.config(1), "gen"
+    elif case == "sweep_32k_gen":
+        w, rows = wl.config(4, L=32768, keep_den=16), "gen"
+    else:
+        w, rows = small_workload("bf16", 128, 64, H=4, Hkv=4, L=9000, M=8744, n_sink=87, C=40), "gen"
     host, dev = make_inputs(w)
     outs = []
-    for _ in range(2):
-        b = fstep.StepBuffers(w)
+    for _ in range(3):
+        b = fstep.StepBuffers(w, rows=rows)
         fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
         fstep.dense_layer(ctx, b, dev["Q"], dev["K"], dev["V"])
-        fstep.find_sinks(ctx, b, dev["Q"], dev["K"], b.lse)
+        dense = b.O.view(torch.int16).clone()
+        fstep.find_sinks(ctx, b, dev["Q"], dev["K"], b.lse if rows == "active" else None)
         fstep.sparse_layer(ctx, b, dev["Q"], dev["K"], dev["V"])
         torch.cuda.synchronize()
-        outs.append([t.clone() for t in (b.sink_idx, b.sink_scores, b.R, b.block_idx, b.O.view(torch.int16), b.lse)])
-    for a, c in zip(*outs):
-        assert torch.equal(a, c)
+        outs.append([t.clone() for t in (dense, b.sink_idx, b.sink_scores, b.R, b.block_idx, b.O.view(torch.int16), b.lse)])
+    for other in outs[1:]:
+        for a, c in zip(outs[0], other):
+            assert torch.equal(a, c)
+    assert ctx.poll_status() == 0
 
 
 @pytest.mark.parametrize("rows", ["active", "gen"])
