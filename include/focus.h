@@ -10,8 +10,9 @@
  *     [b*kv_block, min((b+1)*kv_block, M)); there are nb = ceil(M / kv_block) blocks.
  *   - Query head h reads KV head g(h) = h / (n_q_heads / n_kv_heads).
  *   - All data pointers are DEVICE pointers owned by the caller unless a comment says "host".
- *     Q/K/V base pointers must be 16-byte aligned; the innermost (head_dim) dimension is contiguous;
- *     token and head strides are in elements and must be multiples of 8 elements.
+ *     Tensor base pointers (Q, K, V, O, pooled keys, logits, new K/V rows) must be 16-byte aligned; the innermost
+ *     (head_dim) dimension is contiguous; token and head strides are in elements and must be multiples of 8
+ *     elements.  Both are checked on the host (FOCUS_ERR_INVALID_ARG): a misaligned address would fault on the device.
  *   - Index outputs are int32, ascending, padded with -1.  Counts are written to device int32 so a
  *     whole step can be enqueued without a host round trip.
  *   - Every call validates its arguments on the host, enqueues its kernels on the caller's stream and

@@ -120,6 +120,7 @@ static focus_status attn_common(focus_ctx* ctx, const focus_shape* shape, const 
                                 const int32_t* q_rows, const int32_t* n_rows, int max_rows, const void* K,
                                 const void* V, void* O, float* lse, AttnArgs& a) {
   if (!ctx || !shape_ok_basic(shape) || !Q || !K || !V || !O) return FOCUS_ERR_INVALID_ARG;
+  if (!all_aligned16(Q, K, V, O)) return FOCUS_ERR_INVALID_ARG;
   if (n_q < 0 || q_base < 0 || q_base + n_q > shape->L) return FOCUS_ERR_INVALID_ARG;
   if ((q_rows == nullptr) != (n_rows == nullptr)) return FOCUS_ERR_INVALID_ARG;
   if (q_rows && max_rows < 0) return FOCUS_ERR_INVALID_ARG;
@@ -174,6 +175,7 @@ extern "C" focus_status focus_find_sinks(focus_ctx* ctx, const focus_shape* shap
                                          const void* K, const float* lse, int32_t n_sink, int32_t cand_lo,
                                          int32_t cand_hi, int32_t* sink_idx, float* scores, focus_stream stream) {
   if (!ctx || !shape_ok_basic(shape) || !Q || !active_idx || !n_active || !K || !sink_idx) return FOCUS_ERR_INVALID_ARG;
+  if (!all_aligned16(Q, K)) return FOCUS_ERR_INVALID_ARG;
   if (max_active <= 0 || n_sink < 0 || q_base < 0 || q_base > shape->L) return FOCUS_ERR_INVALID_ARG;
   if (cand_lo < 0 || cand_hi < cand_lo || cand_hi > shape->L) return FOCUS_ERR_INVALID_ARG;
   if (!shape_supported(shape)) return FOCUS_ERR_UNSUPPORTED;

@@ -69,6 +69,11 @@ static inline bool shape_ok_basic(const focus_shape* s) {
   if ((s->q_stride_row | s->q_stride_head | s->kv_stride_tok | s->kv_stride_head) & 7) return false;
   return true;
 }
+// Vector loads and TMA copies need 16-byte aligned tensors: checked on the host, a misaligned address on the device
+// would fault.  NULL counts as aligned (optional arguments).
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+template <typename... P>
+static inline bool all_aligned16(P... p) { return (aligned16(p) && ...); }
 static inline bool shape_supported(const focus_shape* s) {
   return (s->head_dim == 64 || s->head_dim == 128) && (s->kv_block == 64 || s->kv_block == 128);
 }

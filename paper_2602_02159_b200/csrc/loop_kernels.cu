@@ -135,7 +135,7 @@ extern "C" focus_status focus_confidence(focus_ctx* ctx, const void* logits, int
                                          int32_t vocab, int32_t pos_base, int32_t n_pos, const int32_t* rows,
                                          const int32_t* n_rows, int32_t max_rows, float* conf, int32_t* token,
                                          focus_stream stream) {
-  if (!ctx || !logits || !conf || !token) return FOCUS_ERR_INVALID_ARG;
+  if (!ctx || !logits || !conf || !token || !aligned16(logits)) return FOCUS_ERR_INVALID_ARG;
   if (dtype != FOCUS_F32 && dtype != FOCUS_BF16) return FOCUS_ERR_INVALID_ARG;
   if (vocab <= 0 || row_stride < vocab || pos_base < 0 || n_pos < 0 || max_rows < 0) return FOCUS_ERR_INVALID_ARG;
   if ((rows == nullptr) != (n_rows == nullptr)) return FOCUS_ERR_INVALID_ARG;
@@ -173,6 +173,7 @@ extern "C" focus_status focus_update_kv(focus_ctx* ctx, const focus_shape* shape
                                         const int32_t* n_rows, int32_t max_rows, focus_stream stream) {
   if (!ctx || !shape_ok_basic(shape) || !K_cache || !V_cache || !K_new || !V_new || !rows || !n_rows)
     return FOCUS_ERR_INVALID_ARG;
+  if (!all_aligned16(K_cache, V_cache, K_new, V_new)) return FOCUS_ERR_INVALID_ARG;
   if (max_rows < 0) return FOCUS_ERR_INVALID_ARG;
   if (!shape_supported(shape)) return FOCUS_ERR_UNSUPPORTED;
   if (max_rows == 0) return FOCUS_OK;

@@ -132,7 +132,7 @@ static focus_status pool_score_launch(const focus_shape* s, const void* K, float
 
 extern "C" focus_status focus_pool_keys(focus_ctx* ctx, const focus_shape* shape, const void* K, float* Kbar,
                                         focus_stream stream) {
-  if (!ctx || !shape_ok_basic(shape) || !K || !Kbar) return FOCUS_ERR_INVALID_ARG;
+  if (!ctx || !shape_ok_basic(shape) || !K || !Kbar || !all_aligned16(K, Kbar)) return FOCUS_ERR_INVALID_ARG;
   if (!shape_supported(shape)) return FOCUS_ERR_UNSUPPORTED;
   return shape->dtype == FOCUS_BF16 ? pool_score_launch<__nv_bfloat16>(shape, K, Kbar, nullptr, nullptr, stream)
                                     : pool_score_launch<float>(shape, K, Kbar, nullptr, nullptr, stream);
@@ -143,7 +143,7 @@ extern "C" focus_status focus_score_blocks(focus_ctx* ctx, const focus_shape* sh
                                            const void* K, const float* Kbar, int32_t head_reduce, float* R,
                                            focus_stream stream) {
   if (!ctx || !shape_ok_basic(shape) || !Q || !focus_idx || !n_focus || !R) return FOCUS_ERR_INVALID_ARG;
-  if ((K == nullptr) == (Kbar == nullptr)) return FOCUS_ERR_INVALID_ARG;
+  if ((K == nullptr) == (Kbar == nullptr) || !all_aligned16(Q, K, Kbar)) return FOCUS_ERR_INVALID_ARG;
   if (max_focus <= 0 || q_base < 0 || q_base > shape->L) return FOCUS_ERR_INVALID_ARG;
   if (head_reduce != FOCUS_HEADS_PER_KV_GROUP && head_reduce != FOCUS_HEADS_ALL) return FOCUS_ERR_INVALID_ARG;
   if (!shape_supported(shape)) return FOCUS_ERR_UNSUPPORTED;
@@ -217,7 +217,7 @@ extern "C" focus_status focus_score_blocks_static(const focus_shape* shape, cons
                                                   int32_t head_reduce, float* R, int32_t* device_status,
                                                   focus_stream stream) {
   if (!shape_ok_basic(shape) || !Q || !focus_idx || !n_focus || !R) return FOCUS_ERR_INVALID_ARG;
-  if ((K == nullptr) == (Kbar == nullptr)) return FOCUS_ERR_INVALID_ARG;
+  if ((K == nullptr) == (Kbar == nullptr) || !all_aligned16(Q, K, Kbar)) return FOCUS_ERR_INVALID_ARG;
   if (max_focus <= 0 || q_base < 0 || q_base > shape->L) return FOCUS_ERR_INVALID_ARG;
   if (head_reduce != FOCUS_HEADS_PER_KV_GROUP && head_reduce != FOCUS_HEADS_ALL) return FOCUS_ERR_INVALID_ARG;
   if (!shape_supported(shape)) return FOCUS_ERR_UNSUPPORTED;

@@ -169,6 +169,7 @@ extern "C" focus_status focus_sparse_layer(focus_ctx* ctx, const focus_shape* sh
   if (!ctx || !shape_ok_basic(shape) || !Q || !K || !V || !Kbar || !O || !focus_idx || !n_focus || !block_idx ||
       !block_cnt)
     return FOCUS_ERR_INVALID_ARG;
+  if (!all_aligned16(Q, K, V, Kbar, O)) return FOCUS_ERR_INVALID_ARG;
   const int nb = shape_nb(shape);
   if (C < 0 || C > nb || n_sink < 0 || max_focus <= 0) return FOCUS_ERR_INVALID_ARG;
   if (n_sink > 0 && (!sink_idx || !sink_keep)) return FOCUS_ERR_INVALID_ARG;

@@ -699,6 +699,39 @@ def test_host_side_argument_matrix(ctx):
     tiny.close()
 
 
+def test_misaligned_tensors_are_refused_on_the_host(ctx):
+    """A tensor that does not start on a 16-byte boundary is turned away before anything is launched (the kernels use
+    128-bit loads and TMA copies, which would fault on it)."""
+    w = small_workload("bf16", 128, 128)
+    s = w.shape
+    host, dev = make_inputs(w)
+    b = fstep.StepBuffers(w)
+    fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
+    off = lambda t: torch.cat([t.reshape(-1), t.reshape(-1)[:8]])[1:]          # same values, start + 2 bytes
+    Kbar = torch.zeros(s.Hkv, s.nb, s.d, dtype=torch.float32, device="cuda")
+    n0 = fb.focus_launch_count()
+    calls = [
+        lambda: fb.focus_dense_attn(ctx, b.shape, off(dev["Q"]), s.M, s.N, None, None, 0, dev["K"], dev["V"], b.O, b.lse),
+        lambda: fb.focus_dense_attn(ctx, b.shape, dev["Q"], s.M, s.N, None, None, 0, off(dev["K"]), dev["V"], b.O, b.lse),
+        lambda: fb.focus_dense_attn(ctx, b.shape, dev["Q"], s.M, s.N, None, None, 0, dev["K"], off(dev["V"]), b.O, b.lse),
+        lambda: fb.focus_dense_attn(ctx, b.shape, dev["Q"], s.M, s.N, None, None, 0, dev["K"], dev["V"], off(b.O), b.lse),
+        lambda: fstep.find_sinks(ctx, b, dev["Q"], off(dev["K"]), None),
+        lambda: fb.focus_pool_keys(ctx, b.shape, off(dev["K"]), Kbar),
+        lambda: fb.focus_score_blocks(ctx, b.shape, off(dev["Q"]), s.M, b.focus_idx, b.n_focus, w.k, dev["K"], None, 0, b.R),
+        lambda: fstep.sparse_layer(ctx, b, dev["Q"], dev["K"], off(dev["V"]), Kbar=Kbar),
+        lambda: fb.focus_update_kv(ctx, b.shape, dev["K"].clone(), dev["V"].clone(),
+                                   off(torch.zeros(b.max_active, s.Hkv, s.d, dtype=torch.bfloat16, device="cuda")),
+                                   torch.zeros(b.max_active, s.Hkv, s.d, dtype=torch.bfloat16, device="cuda"),
+                                   b.active_idx, b.n_active, b.max_active),
+    ]
+    for call in calls:
+        with pytest.raises(fb.FocusError) as e:
+            call()
+        assert e.value.code == fb.ERR_INVALID_ARG
+    assert fb.focus_launch_count() == n0
+    assert ctx.poll_status() == 0
+
+
 @pytest.mark.parametrize("merge", [None, "counters", "kernel"])
 @pytest.mark.parametrize("cfg", [SHAPES[1], SHAPES[3], SHAPES[5]])
 def test_a_context_of_exactly_the_advertised_workspace_runs_every_stage(cfg, merge, monkeypatch):
