@@ -3,8 +3,9 @@
 //
 // attn_tc_kernel: one CTA = one 128-row query tile of one KV head (GQA: the rows of all query heads of the group
 // are stacked, so every K/V tile is read once per group) x one contiguous range ("split") of that head's key
-// tiles.  Key tiles are 128 keys wide and are enumerated from the selected block list, the gathered sink tokens
-// and the response region; K/V tiles arrive by TMA through a six-slot ring.
+// tiles.  Key tiles are 128 keys wide and are enumerated from the selected block list (one 128-token block, or two
+// 64-token blocks side by side, per tile), the gathered sink tokens and the response region; K/V tiles arrive by
+// TMA through a six-slot ring.
 //
 // Warp roles (192 threads):
 //   warp 0        TMA producer (one lane): K0, K1, V0, K2, V1, ... in the order the MMA warp consumes them
