@@ -43,6 +43,10 @@ constexpr int NBAR = 2 * NSLOT + 7;
 constexpr int MAXT = 128;            // key tiles of a split whose descriptors are staged in shared memory
 constexpr int SMEM_BYTES = 1024 + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8 + 64 + MAXT * 8;
 constexpr int NTHREADS = 192;
+#ifndef FOCUS_PREF_TILES
+#define FOCUS_PREF_TILES 1
+#endif
+constexpr int PREF_TILES = FOCUS_PREF_TILES;   // key tiles (K and V) warmed in L2 ahead of the dependency wait
 constexpr float RESCALE_THRESHOLD = 8.0f;      // log2 units: O is rescaled only when the row max grew by more
 
 struct TcParams {
@@ -71,11 +75,14 @@ struct TcParams {
 };
 
 #ifdef FOCUS_TIMELINE
-#define TL_STAMP(slot, tid) do { if (p.dbg && threadIdx.x == (tid)) p.dbg[(blockIdx.x * gridDim.y + blockIdx.y) * 8 + (slot)] = global_ns(); } while (0)
+#define TL_STAMP(slot, tid) do { if (p.dbg && threadIdx.x == (tid)) p.dbg[(blockIdx.x * gridDim.y + blockIdx.y) * 16 + (slot)] = global_ns(); } while (0)
 // per-iteration trace of CTA (0,0): who 0 = MMA thread, 1 = first softmax thread of tile A, 2 = of tile B
 __device__ __forceinline__ unsigned long long tl_clock() { unsigned long long c; asm volatile("mov.u64 %0, %%clock64;" : "=l"(c) :: "memory"); return c; }
 #define TL_ITER(who, tid, it, ev) do { if (p.dbg && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == (tid) && (it) < 64) p.dbg[65536 + (who) * 512 + (it) * 8 + (ev)] = tl_clock(); } while (0)
+// per-CTA stamp in SM cycles (cheap to take: for intervals inside one CTA)
+#define TL_CLK(slot, tid) do { if (p.dbg && threadIdx.x == (tid)) p.dbg[(blockIdx.x * gridDim.y + blockIdx.y) * 16 + (slot)] = tl_clock(); } while (0)
 #else
+#define TL_CLK(slot, tid) do { } while (0)
 #define TL_STAMP(slot, tid) do { } while (0)
 #define TL_ITER(who, tid, it, ev) do { } while (0)
 #endif
@@ -107,6 +114,27 @@ struct TileEnum {
   int n_sinkt, n_resp, total;
   const int32_t* blocks;
 };
+
+// The kernel parameters sit in constant memory that is new for every launch: the first touch of each line is a
+// round trip to L2 or DRAM, and the code after the dependency wait walks through them one by one (measured: 1.8 us of
+// the 3.1 us between the wait and the first TMA issue).  Touching one word per 32 bytes -- and the tensor maps --
+// while the predecessor is still draining takes those misses off the critical path.
+__device__ __forceinline__ void warm_params(const TcParams& p, const CUtensorMap* a, const CUtensorMap* b,
+                                            const CUtensorMap* c, const CUtensorMap* d) {
+  const unsigned w = (unsigned)(size_t)p.Q ^ (unsigned)(size_t)p.n_rows ^ (unsigned)(size_t)p.part_O ^
+                     (unsigned)p.q_stride_head ^ (unsigned)p.Hkv ^ (unsigned)p.ns_pad ^ (unsigned)(size_t)p.status;
+  asm volatile("" ::"r"(w));
+  if (threadIdx.x == 0) {
+    prefetch_tmap(a); prefetch_tmap(b);
+    if (!p.dense) { prefetch_tmap(c); prefetch_tmap(d); }
+  }
+}
+
+// First key tile of split s of n: floor(total * s / n).  total < 2^23 tiles (2^30 tokens) and s <= 8, so the product
+// fits 32 bits (a 64-bit division is a subroutine of a few hundred cycles on the set-up path of every CTA).
+__device__ __forceinline__ int split_lo(int total, int s, int n) {
+  return (int)((unsigned)total * (unsigned)s / (unsigned)n);
+}
 
 __device__ __forceinline__ TileEnum make_enum(const TcParams& p, int g, int cnt_raw) {
   TileEnum e;
@@ -346,13 +374,13 @@ __device__ __forceinline__ void cluster_merge(const TcParams& p, int g, int mt, 
   const int rows = min(ROWS, total_fr - mt * ROWS);
   const int S = p.n_splits;                                   // <= 8 in cluster mode
   const int mine = rank < rows ? (rows - rank + S - 1) / S : 0;
-  TL_STAMP(5, 0);
+  TL_STAMP(13, 0);
   if (tid >= 0) {
     if (S <= 2) cluster_merge_items<ROWS, NTH, 2>(p, g, mt, rank, spart, mine, tid);
     else if (S <= 4) cluster_merge_items<ROWS, NTH, 4>(p, g, mt, rank, spart, mine, tid);
     else cluster_merge_items<ROWS, NTH, 8>(p, g, mt, rank, spart, mine, tid);
   }
-  TL_STAMP(6, 128);
+  TL_STAMP(14, 128);
   cluster_sync_all();                                          // nobody leaves while its partial may still be read
 }
 
@@ -402,6 +430,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   // set-up (barriers, TMEM) runs ahead.  p.pdl = 1: the predecessor is the selection kernel of the same sparse layer
   // (see further down).
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (p.pdl) warm_params(p, &tmK, &tmV, &tmSK, &tmSV);
   auto arm_barriers = [&]() {                        // warp 0, lane 0
     for (int sl = 0; sl < NSLOT; ++sl) { mbar_init(bar_full(sl), 1); mbar_init(bar_empty(sl), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pready(b), 128); mbar_init(bar_pready2(b), 128); }
@@ -417,26 +446,94 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   if (p.pdl == 2) {
     if (warp == 0 && lane == 0) arm_barriers();
     if (warp == 1) alloc_tmem();
+    // While the predecessor drains (a CTA is resident a few microseconds before the wait returns), warm L2 with what
+    // the chain of dependent loads after the wait will ask for: the row count and row list, this tile's query rows
+    // and, for the dense key set (known without reading anything), the first ring-full of K/V tiles.  Values read
+    // here serve as prefetch addresses only (bounds-checked) and are read again after the wait.
+    if (warp == 0 && lane == 0 && p.dense) {
+      const int total = (p.L + TN - 1) / TN;
+      const int pt0 = split_lo(total, split, p.n_splits), pt1 = split_lo(total, split + 1, p.n_splits);
+      for (int t = pt0; t < pt1 && t < pt0 + PREF_TILES; ++t) {
+        tma_prefetch_3d(&tmK, 0, t * TN, g); tma_prefetch_3d(&tmK, 64, t * TN, g);
+        tma_prefetch_3d(&tmV, 0, t * TN, g); tma_prefetch_3d(&tmV, 64, t * TN, g);
+      }
+    }
+    if (warp >= 2) {
+      const int ptid = (int)threadIdx.x - 64;                            // 0..127: one query row each
+      const int qr = (mt * TM + ptid) / p.hpg, hh = (mt * TM + ptid) % p.hpg;
+      if (qr < p.rows_bound) {
+        int pos = p.q_base + qr;
+        if (p.q_rows) {
+          if (ptid == 0) prefetch_l2(p.n_rows);
+          pos = *reinterpret_cast<const volatile int*>(p.q_rows + qr);
+        }
+        if (pos >= p.q_base && pos < p.q_base + p.n_q) {
+          const __nv_bfloat16* row = p.Q + (long long)(pos - p.q_base) * p.q_stride_row + (long long)(g * p.hpg + hh) * p.q_stride_head;
+          prefetch_l2(row); prefetch_l2(row + 64);
+        }
+      }
+    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    TL_STAMP(7, 0);
+    TL_CLK(15, 0);
+  }
+  // Dense key set: which tiles this split streams is known without reading anything, so the first ring-full of
+  // K/V copies starts right here, ahead of the chain row count -> row list -> query rows (about 3 us sooner than
+  // from their usual place further down).  Should the tile then turn out to have no rows, the copies are awaited
+  // before the CTA leaves.
+  // the two loads every thread's set-up hangs on are requested first (their values are consumed further down)
+  constexpr int QCH = HD * 2 / 16;                               // 16-byte chunks per query row
+  const int qtid = (int)threadIdx.x - 64;                        // row of the tile staged by this thread (warps 2..5)
+  const int nrows_raw = p.q_rows ? ld_ordered(p.n_rows) : p.n_q;
+  const int my_fr = mt * TM + qtid;
+  const int my_qr = my_fr / p.hpg, my_hh = my_fr - my_qr * p.hpg;
+  const int my_pos = (qtid >= 0 && my_qr < p.rows_bound) ? (p.q_rows ? ld_ordered(p.q_rows + my_qr) : p.q_base + my_qr) : -1;
+  int early_issued = 0;
+  if (p.pdl == 2 && p.dense && warp == 0) {
+    const int total = (p.L + TN - 1) / TN;
+    const int pt0 = split_lo(total, split, p.n_splits), pt1 = split_lo(total, split + 1, p.n_splits);
+    const int ntd = pt1 - pt0;
+    const int n_e = 2 * ntd < NSLOT ? 2 * ntd : NSLOT;
+    const uint64_t pol = l2_policy_evict_first();
+    if (lane < n_e) {                                // lane q issues copy q: K0, K1, V0, K2, V1, ... as in seq_tile below
+      const int q = lane;
+      bool isV; int idx;
+      if (q == 0) { isV = false; idx = 0; }
+      else if (q == 2 * ntd - 1) { isV = true; idx = ntd - 1; }
+      else if (q & 1) { isV = false; idx = (q + 1) >> 1; }
+      else { isV = true; idx = (q >> 1) - 1; }
+      TileInfo ti;
+      ti.kind = 0; ti.start = (pt0 + idx) * TN; ti.nvalid = min(TN, p.L - ti.start); ti.start2 = ti.start + 64;
+      load_tile(p, ti, isV ? &tmV : &tmK, sSlot + (q % NSLOT) * SLOT_BYTES, bar_full(q % NSLOT), g, pol);
+    }
+    early_issued = n_e;
+    __syncwarp();
   }
 
   // The prologue is a chain of global-memory latencies; everything that does not depend on another load is
-  // requested first: the row count, this group's block count, the positions of this thread's Q rows.
-  constexpr int QTHREADS = 128;                                  // the four softmax warps stage Q
-  constexpr int QIT = TM * 16 / QTHREADS;                        // 16-byte chunks of the Q tile per staging thread
-  const int qtid = (int)threadIdx.x - 64;
-  const int nrows_raw = p.q_rows ? ld_ordered(p.n_rows) : p.n_q;
-  int qpos[QIT];
+  // requested first: the row count and the position of this thread's query row.  Each of the 128 softmax threads
+  // stages one whole row (sixteen 16-byte chunks): one row-list entry and one division per thread, and a short
+  // stretch of straight-line code (the earlier chunk-interleaved mapping cost every thread sixteen of each).
+  // The query row is requested as soon as its position is known, without waiting for the row count: an entry of
+  // the row list beyond the count is either a valid position (a row read for nothing) or not (skipped).
+  uint4 qv[QCH];
 #pragma unroll
-  for (int it = 0; it < QIT; ++it) {
-    const int idx = qtid + it * QTHREADS;
-    const int qr = (mt * TM + (idx >> 4)) / p.hpg;
-    qpos[it] = (qtid >= 0 && qr < p.rows_bound) ? (p.q_rows ? ld_ordered(p.q_rows + qr) : p.q_base + qr) : -1;
+  for (int c = 0; c < QCH; ++c) qv[c] = make_uint4(0, 0, 0, 0);
+  const bool pos_ok = my_pos >= p.q_base && my_pos < p.q_base + p.n_q;
+  if (pos_ok) {
+    const uint4* src = reinterpret_cast<const uint4*>(p.Q + (long long)(my_pos - p.q_base) * p.q_stride_row +
+                                                      (long long)(g * p.hpg + my_hh) * p.q_stride_head);
+#pragma unroll
+    for (int c = 0; c < QCH; ++c) qv[c] = ld_ordered(src + c);
   }
   const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
   const int total_fr = nrows * p.hpg;                    // stacked (row, head-of-group) rows of this KV head
+  TL_CLK(8, 0);
   if (mt * TM >= total_fr) {                             // uniform: nothing to compute for this tile
     if (p.pdl == 2) {                                    // TMEM was allocated ahead of the row count
+      if (lane == 0)
+        for (int q = 0; q < early_issued; ++q)           // copies already on their way land before the CTA leaves
+          mbar_wait(bar_full(q % NSLOT), 0u, abort_flag, p.status);
       tc_fence_before();
       __syncthreads();
       tc_fence_after();
@@ -448,34 +545,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     return;
   }
 
-  // query rows of this thread (softmax warps only): requested now, stored to shared memory further down
-  uint4 qv[QIT];
+  // a listed row whose position is out of range is reported; rows beyond the count are staged as zeros
+  if (qtid >= 0 && my_fr < total_fr && !pos_ok) set_status(p.status, FOCUS_ERR_INVALID_ARG);
+  if (my_fr >= total_fr) {
 #pragma unroll
-  for (int it = 0; it < QIT; ++it) {
-    qv[it] = make_uint4(0, 0, 0, 0);
-    if (qtid >= 0) {
-      const int idx = qtid + it * QTHREADS;
-      const int r = idx >> 4, c = idx & 15;
-      const int fr = mt * TM + r;
-      if (fr < total_fr) {
-        const int pos = qpos[it];
-        if (pos >= p.q_base && pos < p.q_base + p.n_q) {
-          const __nv_bfloat16* src = p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
-                                     (long long)(g * p.hpg + fr % p.hpg) * p.q_stride_head + c * 8;
-          qv[it] = ld_ordered(reinterpret_cast<const uint4*>(src));
-        } else if (c == 0) {
-          set_status(p.status, FOCUS_ERR_INVALID_ARG);
-        }
-      }
-    }
+    for (int c = 0; c < QCH; ++c) qv[c] = make_uint4(0, 0, 0, 0);
   }
-  auto store_q = [&]() {                             // softmax warps
+  auto store_q = [&]() {                             // softmax warps: row qtid, chunk c -> swizzled K-major tile
 #pragma unroll
-    for (int it = 0; it < QIT; ++it) {
-      const int idx = qtid + it * QTHREADS;
-      const int r = idx >> 4, c = idx & 15;
+    for (int c = 0; c < QCH; ++c) {
       const int half = c >> 3, cc = c & 7;
-      *reinterpret_cast<uint4*>(sptr + half * HALF_BYTES + r * 128 + ((cc ^ (r & 7)) << 4)) = qv[it];
+      *reinterpret_cast<uint4*>(sptr + half * HALF_BYTES + qtid * 128 + ((cc ^ (qtid & 7)) << 4)) = qv[c];
     }
   };
   // Launched as a programmatic dependent of the selection kernel of the same sparse layer: everything above
@@ -491,10 +571,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   const int cnt_raw = p.dense ? 0 : ld_ordered(p.block_cnt + g * p.group_stride);
 
   const TileEnum te = make_enum(p, g, cnt_raw);
-  const int t0 = (int)(((long long)te.total * split) / p.n_splits);
-  const int t1 = (int)(((long long)te.total * (split + 1)) / p.n_splits);
+  const int t0 = split_lo(te.total, split, p.n_splits);
+  const int t1 = split_lo(te.total, split + 1, p.n_splits);
   const int nt = t1 - t0;
   const int cta_lin = blockIdx.x * p.n_splits + split;
+  TL_CLK(9, 0);
 
   const bool use_list = !p.dense && nt <= MAXT;
   // tile descriptor: from the staged list (sparse) or by arithmetic (dense; splits longer than the list)
@@ -545,6 +626,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     isV = true; return (q >> 1) - 1;
   };
   const uint64_t l2_pol = l2_policy_evict_first();
+  TL_CLK(11, 0);
   auto issue = [&](int q) {
     bool isV;
     const int idx = seq_tile(q, isV);
@@ -565,9 +647,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
     }
     __syncwarp();
-    if (lane == 0)
-      for (int q = 0; q < n_early; ++q) issue(q);
+    TL_CLK(10, 0);
+    if (lane >= early_issued && lane < n_early) issue(lane);       // one copy per lane
     __syncwarp();
+    TL_CLK(12, 0);
     TL_STAMP(6, 0);
   }
   if (warp == 1 && !p.pdl) alloc_tmem();
@@ -872,28 +955,39 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
   // programmatic dependent launch: let the successor start early; wait for the predecessor before touching memory
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (p.pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (p.pdl) {
+    warm_params(p, &tmK, &tmV, &tmSK, &tmSV);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+  }
 
   constexpr int TMQ = KP ? TM : TMW;                             // query rows of this CTA
-  constexpr int QTHREADS = 256;                                  // the eight softmax warps stage Q
-  constexpr int QIT = TMQ * 16 / QTHREADS;
+  constexpr int QCH = HD * 2 / 16;                               // 16-byte chunks per query row
+  // one query row per softmax thread (the key-pair form has 128 rows for 256 such threads: the upper half idles);
+  // the row is requested as soon as its position is known, without waiting for the row count
   const int qtid = (int)threadIdx.x - 128;
+  const bool stager = qtid >= 0 && qtid < TMQ;
   const int nrows_raw = p.q_rows ? ld_ordered(p.n_rows) : p.n_q;
   const int cnt_raw = p.dense ? 0 : ld_ordered(p.block_cnt + g * p.group_stride);
-  int qpos[QIT];
+  const int my_fr = mt * TMQ + qtid;
+  const int my_qr = my_fr / p.hpg, my_hh = my_fr - my_qr * p.hpg;
+  const int my_pos = (stager && my_qr < p.rows_bound) ? (p.q_rows ? ld_ordered(p.q_rows + my_qr) : p.q_base + my_qr) : -1;
+  uint4 qv[QCH];
 #pragma unroll
-  for (int it = 0; it < QIT; ++it) {
-    const int idx = qtid + it * QTHREADS;
-    const int qr = (mt * TMQ + (idx >> 4)) / p.hpg;
-    qpos[it] = (qtid >= 0 && qr < p.rows_bound) ? (p.q_rows ? ld_ordered(p.q_rows + qr) : p.q_base + qr) : -1;
+  for (int c = 0; c < QCH; ++c) qv[c] = make_uint4(0, 0, 0, 0);
+  const bool pos_ok = my_pos >= p.q_base && my_pos < p.q_base + p.n_q;
+  if (pos_ok) {
+    const uint4* src = reinterpret_cast<const uint4*>(p.Q + (long long)(my_pos - p.q_base) * p.q_stride_row +
+                                                      (long long)(g * p.hpg + my_hh) * p.q_stride_head);
+#pragma unroll
+    for (int c = 0; c < QCH; ++c) qv[c] = ld_ordered(src + c);
   }
   const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
   const int total_fr = nrows * p.hpg;
   if (mt * TMQ >= total_fr) return;
 
   const TileEnum te = make_enum(p, g, cnt_raw);
-  const int t0 = (int)(((long long)te.total * split) / p.n_splits);
-  const int t1 = (int)(((long long)te.total * (split + 1)) / p.n_splits);
+  const int t0 = split_lo(te.total, split, p.n_splits);
+  const int t1 = split_lo(te.total, split + 1, p.n_splits);
   const int nt = t1 - t0;
 
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -956,39 +1050,22 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       }
     }
     __syncwarp();
-    if (lane == 0)
-      for (int q = 0; q < n_early; ++q) issue(q);
+    if (lane < n_early) issue(lane);                             // one copy per lane
     __syncwarp();
   }
   if (warp == 1) {
     tmem_alloc(smem_u32(tmem_holder), 512);
     tmem_relinquish();
   }
-  if (qtid >= 0) {                                               // both Q tiles: tile X at X * 32 KB, swizzled K-major
-    uint4 qv[QIT];
+  if (stager) {                                                  // query tile X at X * 32 KB, swizzled K-major
+    if (my_fr < total_fr && !pos_ok) set_status(p.status, FOCUS_ERR_INVALID_ARG);
+    const bool live = my_fr < total_fr;                          // rows beyond the count are staged as zeros
+    const int x = qtid >> 7, rr = qtid & 127;
 #pragma unroll
-    for (int it = 0; it < QIT; ++it) {
-      const int idx = qtid + it * QTHREADS;
-      const int r = idx >> 4, c = idx & 15;
-      const int fr = mt * TMQ + r;
-      qv[it] = make_uint4(0, 0, 0, 0);
-      if (fr < total_fr) {
-        const int pos = qpos[it];
-        if (pos >= p.q_base && pos < p.q_base + p.n_q) {
-          const __nv_bfloat16* src = p.Q + (long long)(pos - p.q_base) * p.q_stride_row +
-                                     (long long)(g * p.hpg + fr % p.hpg) * p.q_stride_head + c * 8;
-          qv[it] = ld_ordered(reinterpret_cast<const uint4*>(src));
-        } else if (c == 0) {
-          set_status(p.status, FOCUS_ERR_INVALID_ARG);
-        }
-      }
-    }
-#pragma unroll
-    for (int it = 0; it < QIT; ++it) {
-      const int idx = qtid + it * QTHREADS;
-      const int r = idx >> 4, c = idx & 15;
-      const int x = r >> 7, rr = r & 127, half = c >> 3, cc = c & 7;
-      *reinterpret_cast<uint4*>(sptr + x * Q_BYTES + half * HALF_BYTES + rr * 128 + ((cc ^ (rr & 7)) << 4)) = qv[it];
+    for (int c = 0; c < QCH; ++c) {
+      const int half = c >> 3, cc = c & 7;
+      *reinterpret_cast<uint4*>(sptr + x * Q_BYTES + half * HALF_BYTES + rr * 128 + ((cc ^ (rr & 7)) << 4)) =
+          live ? qv[c] : make_uint4(0, 0, 0, 0);
     }
   }
   fence_proxy_async();
