@@ -682,7 +682,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       int issued = n_early;
       bool ok = true;
       for (int q = n_early; q < n_loads; ++q) {
+        TL_ITER(2, 0, q, 0);
         if (!mbar_wait(bar_empty(q % NSLOT), (uint32_t)((q / NSLOT) & 1) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        TL_ITER(2, 0, q, 1);
         issue(q);
         ++issued;
       }
@@ -729,7 +731,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       for (int idx = 0; idx < nt && ok; ++idx) {
         const int b = idx & 1;
         const int slot = q % NSLOT;
+        TL_ITER(0, 32, idx, 0);
         if (!mbar_wait(bar_full(slot), (q / NSLOT) & 1u, abort_flag, p.status)) { ok = false; break; }
+        TL_ITER(0, 32, idx, 1);
         tc_fence_after();
         const uint64_t kdesc = make_sdesc(sSlot + slot * SLOT_BYTES, 16, 1024);
 #pragma unroll
@@ -742,7 +746,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         tc_commit(bar_empty(slot));
         tc_commit(bar_sfull(b));
         ++q;
+        TL_ITER(0, 32, idx, 2);
         if (idx > 0) ok = do_pv(idx - 1);
+        TL_ITER(0, 32, idx, 3);
       }
       if (ok) ok = do_pv(nt - 1);
     }
@@ -755,8 +761,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     bool ok = true;
     for (int idx = 0; idx < nt; ++idx) {
       const int b = idx & 1;
+      TL_ITER(1, 64, idx, 0);
       // votes keep the warp together: the TMEM loads and stores below are warp-collective
       if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(b), (uint32_t)(idx >> 1) & 1u, abort_flag, p.status))) { ok = false; break; }
+      TL_ITER(1, 64, idx, 1);
       tc_fence_after();
       if (idx == 0) TL_STAMP(5, 64);
       uint32_t sreg[128];
@@ -766,6 +774,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       TC_LD32(ts + 64, (sreg + 64));
       TC_LD32(ts + 96, (sreg + 96));
       tc_wait_ld();
+      TL_ITER(1, 64, idx, 2);
       const TileInfo ti = get_tile(idx);
       float tmax = -INFINITY;
       if (ti.kind == 0 && ti.nvalid == TN) {
@@ -824,6 +833,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           TC_ST32(tmem_O + lane_off + cb * 32, oreg);
         }
       }
+      TL_ITER(1, 64, idx, 3);
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {                 // 32 keys at a time: exponentials, bf16 P, row sum
@@ -842,11 +852,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           tc_wait_st();
           tc_fence_before();
           mbar_arrive(bar_pready(b));
+          TL_ITER(1, 64, idx, 4);
         }
       }
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar_pready2(b));
+      TL_ITER(1, 64, idx, 5);
       l = l * alpha + ((acc[0] + acc[1]) + (acc[2] + acc[3]));
     }
     // ---- epilogue: wait for the last P V, normalise, write out -----------------------------------
