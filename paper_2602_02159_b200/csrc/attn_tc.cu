@@ -780,9 +780,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       if (ti.kind == 0 && ti.nvalid == TN) {
         float t4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains instead of one of 128
 #pragma unroll
-        for (int c = 0; c < 128; c += 4) {
-          t4[0] = fmaxf(t4[0], __uint_as_float(sreg[c]));     t4[1] = fmaxf(t4[1], __uint_as_float(sreg[c + 1]));
-          t4[2] = fmaxf(t4[2], __uint_as_float(sreg[c + 2])); t4[3] = fmaxf(t4[3], __uint_as_float(sreg[c + 3]));
+        for (int c = 0; c < 128; c += 8) {
+          t4[0] = fmax3(t4[0], __uint_as_float(sreg[c]), __uint_as_float(sreg[c + 1]));
+          t4[1] = fmax3(t4[1], __uint_as_float(sreg[c + 2]), __uint_as_float(sreg[c + 3]));
+          t4[2] = fmax3(t4[2], __uint_as_float(sreg[c + 4]), __uint_as_float(sreg[c + 5]));
+          t4[3] = fmax3(t4[3], __uint_as_float(sreg[c + 6]), __uint_as_float(sreg[c + 7]));
         }
         tmax = fmaxf(fmaxf(t4[0], t4[1]), fmaxf(t4[2], t4[3]));
       } else if (ti.kind == 0) {
