@@ -245,11 +245,16 @@ def test_config3_gqa_16_steps(ctx):
 
 
 # ---- config 4: sweep points (context x keep ratio), gen-region rows ---------------------------------------------
-@pytest.mark.parametrize("L,keep_den", [(4096, 4), (32768, 16), (131072, 32), (8192, 1)])
-def test_config4_sweep_points(ctx, L, keep_den):
+@pytest.mark.parametrize("rows", ["gen", "active"])
+@pytest.mark.parametrize("keep_den", wl.SWEEP_KEEP_DEN)
+@pytest.mark.parametrize("L", wl.SWEEP_L)
+def test_config4_sweep_points(ctx, L, keep_den, rows):
+    """Every point of the context x keep-ratio grid that the sweep times, in both row modes: between them they take
+    the one-warpgroup kernel (I_active rows), the key-pair form and the two-tile form (gen rows), short and long
+    block lists, with and without staged tile lists."""
     w = wl.config(4, L=L, keep_den=keep_den)
     heads = [0, 21] if L > 40000 else [0, 13, 31]
-    single_layer_case(ctx, w, "gen", heads=heads, check_dense=L <= 40000)
+    single_layer_case(ctx, w, rows, heads=heads, check_dense=L <= 40000)
 
 
 # ---- the paper's own hyper-parameters (block 64, half of the blocks kept) on the 32K shape, one layer ---------
