@@ -204,6 +204,12 @@ def test_config2_full_32_layer_step(ctx):
     assert na > 0 and ctx.poll_status() == 0
 
 
+def test_config2_one_layer_with_all_gen_rows(ctx):
+    """The gen-row figures of the benchmark (512 query rows, 32 heads, 32K keys): one layer of config 2 with the whole
+    gen region as query set -- dense on the two-tile form, sparse on the key-pair form."""
+    single_layer_case(ctx, wl.config(2), "gen", heads=[0, 19])
+
+
 # ---- config 3: Dream-like GQA, 16 consecutive steps with AR(1) confidences ------------------------------------
 def test_config3_gqa_16_steps(ctx):
     w = wl.config(3)
