@@ -210,6 +210,11 @@ def test_config2_one_layer_with_all_gen_rows(ctx):
     single_layer_case(ctx, wl.config(2), "gen", heads=[0, 19])
 
 
+def test_config3_one_layer_with_all_gen_rows(ctx):
+    """Config 3 with the whole gen region as query set: 256 rows x 7 query heads per KV head stacked on each K/V tile."""
+    single_layer_case(ctx, wl.config(3), "gen", heads=[0, 13, 27])
+
+
 # ---- config 3: Dream-like GQA, 16 consecutive steps with AR(1) confidences ------------------------------------
 def test_config3_gqa_16_steps(ctx):
     w = wl.config(3)
