@@ -84,7 +84,7 @@ class ClockSampler:
         self.proc.terminate()
         self.t.join(timeout=2)
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        sm, sm_head, mx, watts, reasons = [], [], [], [], set()
+        sm, sm_head, mx, watts, reasons, counts = [], [], [], [], set(), {n: 0 for n in names}
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 10:
@@ -108,6 +108,7 @@ class ClockSampler:
             for n, v in zip(names, f[6:10]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
+                    counts[n] += 1
         note = None
         if not sm and mx:                                  # a very short region can fall between two samples
             note = "no sample fell inside a timed region; clocks of the samples around it"
@@ -121,7 +122,8 @@ class ClockSampler:
                 "samples": len(sm), "samples_in_headline_region": len(sm_head),
                 "sm_mhz_headline_region": statistics.median(sm_head) if sm_head else None,
                 "power_w": statistics.median(watts) if watts else None,
-                "interval_ms": self.INTERVAL_MS, "reasons": sorted(reasons)}
+                "interval_ms": self.INTERVAL_MS, "reasons": sorted(reasons),
+                "reason_share": {n: round(c / len(sm), 3) for n, c in counts.items() if c and sm}}
         if note:
             out["note"] = note
         return out
@@ -188,15 +190,20 @@ def run_reference(args):
         return
     w = wl.config(args.config)
     smp = OracleSample(w)
-    vals = []
+    vals, timed_s = [], 0.0
     for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
         ms, cores, sample = smp.run()
         if i >= args.warmup:
             vals.append(ms)
+            timed_s += time.perf_counter() - t0
     v = float(np.mean(vals))
+    # `value` is an extrapolation: each timed pass runs a bounded sample of a step (see cpu_baseline.sample) and is
+    # scaled to the whole step, so steps x value is far more than the wall time of this run
     out = {"impl": "reference", "metric": METRIC, "value": v, "unit": "ms", "n_gpus": args.gpus, "steps": len(vals),
            "warmup": args.warmup, "ms_per_step": v, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-           "dtype": "f64", "data": "synthetic",
+           "dtype": "f64", "data": "synthetic", "extrapolated": True, "timed_passes": len(vals),
+           "timed_s": round(timed_s, 3),
            "config": {"workload": w.name, "rows": "I_active (paper)", "note": "CPU oracle, bounded sample scaled to a step"},
            "cpu_baseline": {"value": v, "unit": "ms", "cores": cores, "kind": "oracle", "sample": sample},
            "e2e": {"value": v, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
@@ -378,13 +385,19 @@ def run_focus(args):
         layers = range(probe + 1) if kind == "dense" else range(probe + 1, NL)
         if len(layers) == 0:
             return None
+        b_ = r_["b"]
+        q_rows_, n_rows_, max_rows_ = b_._rows()
 
         def run():
             for l in layers:
                 if kind == "dense":
-                    fstep.dense_layer(ctx, r_["b"], Qs[l], Ks[l], Vs[l], O=r_["O"][l])
-                else:                                      # sink set from the last full step
-                    fstep.sparse_layer(ctx, r_["b"], Qs[l], Ks[l], Vs[l], Kbar=Kbars[l], O=r_["O"][l])
+                    fstep.dense_layer(ctx, b_, Qs[l], Ks[l], Vs[l], O=r_["O"][l])
+                elif kind == "sparse":                     # sink set from the last full step
+                    fstep.sparse_layer(ctx, b_, Qs[l], Ks[l], Vs[l], Kbar=Kbars[l], O=r_["O"][l])
+                else:                                      # the attention call alone, on the lists the last layer call left
+                    fb.focus_sparse_attn(ctx, b_.shape, Qs[l], b_.q_base, b_.n_q, q_rows_, n_rows_, max_rows_, Ks[l],
+                                         Vs[l], fb.HEADS_PER_KV_GROUP, b_.block_idx, b_.max_blocks, b_.block_cnt,
+                                         b_.sink_idx, b_.sink_keep, w.n_sink, r_["O"][l], b_.lse)
         run()
         torch.cuda.synchronize()
         g_ = torch.cuda.CUDAGraph()
@@ -426,10 +439,11 @@ def run_focus(args):
         ms_gen_dense, _, _ = timed(lambda m: step("gen", dense_only=True), 2, 1)
         gd_eager = float(np.mean([a.elapsed_time(z) for k_, a, z in gm if k_ == "dense"]))
         gs_eager = float(np.mean([a.elapsed_time(z) for k_, a, z in gm if k_ == "sparse"]))
-        gd, gs = gd_eager, gs_eager
+        gd, gs, gsa = gd_eager, gs_eager, None
         if graph is not None:                              # same launch mode as the paper-row figures
             gd = per_launch_in_graph("gen", "dense", max(2, K // 4)) or gd_eager
             gs = per_launch_in_graph("gen", "sparse", max(2, K // 4)) or gs_eager
+            gsa = per_launch_in_graph("gen", "sparse_attn", max(2, K // 4))
         fl_dense = 4.0 * s.N * s.L * s.d * s.H
         fl_sparse = 4.0 * s.N * retained_keys * s.d * s.H
         gen = {"rows": s.N, "ms_per_step": ms_gen, "dense_ms_per_step": ms_gen_dense,
@@ -438,9 +452,16 @@ def run_focus(args):
                "sparse_layer_ms": gs, "sparse_retained_tflops": fl_sparse / gs / 1e9,
                "sparse_dense_equiv_tflops": fl_dense / gs / 1e9,
                "dense_layer_eager_marks_ms": gd_eager, "sparse_layer_eager_marks_ms": gs_eager,
-               "roofline": {"bound": "tensor", "achieved": fl_dense / gd / 1e9, "peak": P["tf_sust"], "unit": "TFLOP/s",
-                            "frac": fl_dense / gd / 1e9 / P["tf_sust"], "kernel": "attn_tc_wide_kernel (dense layer, 512 gen rows)",
-                            "peak_source": f"{P['src']} sustained bf16"}}
+               # these launches are timed alone in millisecond replays (burst conditions): frac is of the burst peak, the
+               # sustained-peak and nominal fractions stand beside it
+               "roofline": tensor_roofline(fl_dense / gd / 1e9, P, "attn_tc_wide_kernel<false> (dense layer, 512 gen rows)"),
+               "sparse_roofline": tensor_roofline(fl_sparse / gs / 1e9, P,
+                                                  "sparse layer on retained blocks, 512 gen rows: selection kernel + "
+                                                  "sparse attention kernel"),
+               "sparse_attn_only_ms": gsa,
+               "sparse_attn_only_roofline": tensor_roofline(fl_sparse / gsa / 1e9, P,
+                                                            "sparse attention kernel alone (lists from the last layer call)")
+               if gsa else None}
     assert ctx.poll_status() == 0
 
     # ---- end to end through the C ABI with host buffers (K/V cache resident: it is model state, Eq. 3) -------
@@ -478,8 +499,118 @@ def run_focus(args):
         main.wait_stream(back_stream)
         main.synchronize()
 
-    ms_e2e, _, _ = timed(e2e_step, max(2, K // 2), 2)
+    ms_e2e_all, _, _ = timed(e2e_step, max(2, K // 2), 2)
 
+    # The same step with only the rows that are read crossing PCIe.  After the indicator the host reads I_focus and
+    # I_active back (a few hundred bytes), gathers those rows of every layer's Q in pinned memory (index bookkeeping on
+    # the host, no arithmetic) and uploads them as a compact [layer, row] array; the library is handed local row
+    # numbers.  Layers run as graphs of a few layers each so that the gather of the next chunk overlaps the GPU work of
+    # the current one; every chunk's outputs go home inside the next chunk's graph, on a second captured stream.
+    bc = fstep.StepBuffers(w, rows="compact", device=dev)
+    MA = bc.max_active
+    Qc = torch.zeros(NL, MA, s.H, s.d, dtype=torch.bfloat16, device=dev)
+    Oc = torch.zeros(NL, MA, s.H, s.d, dtype=torch.bfloat16, device=dev)
+    Qc_host = torch.zeros(NL, MA, s.H, s.d, dtype=torch.bfloat16).pin_memory()
+    Oc_host = torch.zeros(NL, MA, s.H, s.d, dtype=torch.bfloat16).pin_memory()
+    sel_dev = torch.zeros(2 + max(1, w.k) + MA, dtype=torch.int32, device=dev)
+    sel_host = torch.zeros(2 + max(1, w.k) + MA, dtype=torch.int32).pin_memory()
+    sink_host = torch.zeros(bc.sink_idx.numel(), dtype=torch.int32).pin_memory()
+    n_chunks = max(1, min(4, NL // 2))
+    bounds = [round(i * NL / n_chunks) for i in range(n_chunks + 1)]
+    chunk_ready = [torch.cuda.Event() for _ in range(n_chunks)]
+
+    def chunk_layers(c, home_prev):
+        side = torch.cuda.Stream()
+        cur = torch.cuda.current_stream()
+        if home_prev and c > 0:                          # outputs of the previous chunk go home beside this chunk's work
+            side.wait_stream(cur)
+            with torch.cuda.stream(side):
+                Oc_host[bounds[c - 1]:bounds[c]].copy_(Oc[bounds[c - 1]:bounds[c]], non_blocking=True)
+        for l in range(bounds[c], bounds[c + 1]):
+            if l <= probe:
+                fstep.dense_layer(ctx, bc, Qc[l], Ks[l], Vs[l], O=Oc[l])
+                if l == probe:
+                    fstep.find_sinks(ctx, bc, Qc[l], Ks[l], bc.lse)
+            else:
+                fstep.sparse_layer(ctx, bc, Qc[l], Ks[l], Vs[l], Kbar=Kbars[l], O=Oc[l])
+        if home_prev and c > 0:
+            cur.wait_stream(side)
+
+    chunk_graphs = None
+    if graph is not None:
+        # warm every call of the compact path once (function attributes, occupancy queries) before capturing
+        fstep.select_queries(ctx, bc, conf, masked)
+        bc.set_local_focus(results["active"]["b"].focus_idx.cpu().numpy()[:int(results["active"]["b"].n_focus.item())],
+                           results["active"]["b"].active_idx.cpu().numpy()[:na])
+        for c in range(n_chunks):
+            chunk_layers(c, False)
+        torch.cuda.synchronize()
+        chunk_graphs = []
+        for c in range(n_chunks):
+            g_ = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_):
+                chunk_layers(c, True)
+            chunk_graphs.append(g_)
+
+    def e2e_compact_step(_m):
+        main = torch.cuda.current_stream()
+        conf.copy_(conf_host, non_blocking=True)
+        masked.copy_(masked_host, non_blocking=True)
+        fstep.select_queries(ctx, bc, conf, masked)
+        sel_dev[0:1].copy_(bc.n_focus, non_blocking=True); sel_dev[1:2].copy_(bc.n_active, non_blocking=True)
+        sel_dev[2:2 + bc.focus_idx.numel()].copy_(bc.focus_idx, non_blocking=True)
+        sel_dev[2 + bc.focus_idx.numel():].copy_(bc.active_idx, non_blocking=True)
+        sel_host.copy_(sel_dev, non_blocking=True)
+        main.synchronize()
+        nf_, na_ = int(sel_host[0]), int(sel_host[1])
+        fpos = sel_host[2:2 + nf_]
+        apos = sel_host[2 + bc.focus_idx.numel():2 + bc.focus_idx.numel() + na_]
+        bc.set_local_focus(fpos.tolist(), apos.tolist())
+        rows_idx = (apos - s.M).to(torch.int64)
+        for c in range(n_chunks):
+            for l in range(bounds[c], bounds[c + 1]):
+                torch.index_select(Q_host[l], 0, rows_idx, out=Qc_host[l, :na_])
+            with torch.cuda.stream(copy_stream):
+                if c == 0:
+                    copy_stream.wait_stream(main)
+                Qc[bounds[c]:bounds[c + 1], :na_].copy_(Qc_host[bounds[c]:bounds[c + 1], :na_], non_blocking=True)
+                chunk_ready[c].record(copy_stream)
+            main.wait_event(chunk_ready[c])
+            if chunk_graphs is not None:
+                chunk_graphs[c].replay()
+            else:
+                chunk_layers(c, True)
+        Oc_host[bounds[-2]:].copy_(Oc[bounds[-2]:], non_blocking=True)
+        sink_host.copy_(bc.sink_idx, non_blocking=True)
+        main.synchronize()
+
+    ms_e2e, _, _ = timed(e2e_compact_step, max(2, K // 2), 2)
+    h2d_c = conf_host.numel() * 4 + masked_host.numel() + NL * na * s.H * s.d * 2 + 4 * max(1, w.k)
+    d2h_c = Oc_host.numel() * 2 + sel_host.numel() * 4 + sink_host.numel() * 4
+
+    # ---- sustained leg: the same graph replayed back to back for >= 2 s of device time, clocks sampled inside --------
+    sustained = None
+    if graph is not None and args.sustain_s > 0:
+        n_rep = max(K, int(math.ceil(args.sustain_s * 1e3 / ms_step)))
+        sus = ClockSampler(local)
+        sus.INTERVAL_MS = 25
+        sus.start()
+        a, z = ev(), ev()
+        sync_all()
+        with sus.window(True):
+            a.record()
+            for _ in range(n_rep):
+                graph.replay()
+            z.record()
+            sync_all()
+        tot = replicas.max_over_ranks(a.elapsed_time(z), dev)
+        ck = sus.stop()
+        sustained = {"ms_per_step": tot / n_rep, "replays": n_rep, "seconds": tot / 1e3, "sm_mhz_median": ck["sm_mhz"],
+                     "clock_samples": ck["samples"], "power_w_median": ck["power_w"], "reasons": ck["reasons"],
+                     "reason_share": ck.get("reason_share", {}),
+                     "ms_x_mhz": (tot / n_rep) * ck["sm_mhz"] if ck["sm_mhz"] else None,
+                     "burst_ms_x_mhz": ms_step * clocks["sm_mhz_headline_region"] if clocks.get("sm_mhz_headline_region") else None,
+                     "note": "back-to-back replays of the headline graph; the headline value above is a burst of K replays"}
     if rank != 0:
         replicas.shutdown()
         return
@@ -520,16 +651,38 @@ def run_focus(args):
                      "traffic": traffic, "kernel": "attn_tc_kernel incl. its in-cluster split merge (dense layer, I_active rows)",
                      "read_only_stream_GBps": stream_gbs, "frac_of_read_only_stream": dense_gbs / stream_gbs,
                      "bytes_per_launch": kv_bytes + qo_bytes, "peak_source": f"{P['src']} copy bandwidth"},
+        "sparse_roofline": {"bound": "hbm", "achieved": sparse_bytes / (sparse_ms * 1e-3) / 1e9, "peak": P["hbm"], "unit": "GB/s",
+                            "frac": sparse_bytes / (sparse_ms * 1e-3) / 1e9 / P["hbm"],
+                            "frac_of_nominal": sparse_bytes / (sparse_ms * 1e-3) / 1e9 / 8000.0,
+                            "kernel": "sparse layer, I_active rows: selection kernel + sparse attention kernel on retained K/V "
+                                      f"({retained_keys} keys per head)", "bytes_per_launch": sparse_bytes,
+                            "peak_source": f"{P['src']} copy bandwidth; nominal 8000"},
         "gen_mode": gen,
-        "e2e": {"value": ms_e2e, "unit": "ms", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                "resident": "K/V cache stays in HBM between steps (approximate KV cache, Eq. 3); confidence, masks and "
-                            "all layers' Q rows come from pinned host memory (layer by layer on a copy stream, each layer waits "
-                            "for its own rows), every layer's output goes back on a third stream as soon as it exists, the index sets at the end"},
+        "e2e": {"value": ms_e2e, "unit": "ms", "h2d_bytes_per_step": int(h2d_c), "d2h_bytes_per_step": int(d2h_c),
+                "resident": "K/V cache stays in HBM between steps (approximate KV cache, Eq. 3); confidence and masks come "
+                            "from pinned host memory; after the indicator the host reads I_focus / I_active back, gathers "
+                            "those rows of every layer's Q in pinned memory and uploads only them (chunks of layers, the "
+                            "gather of the next chunk overlapping the GPU work of the current one); outputs of the "
+                            "I_active rows of every layer and the index sets go back to pinned memory",
+                "launch_mode": f"{n_chunks} CUDA graphs of {NL // n_chunks} layers per step + eager indicator call"
+                               if chunk_graphs is not None else "eager C-ABI calls"},
+        "e2e_all_gen_rows": {"value": ms_e2e_all, "unit": "ms", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                             "note": "all 512 gen rows of Q of every layer uploaded although only the I_active rows are read "
+                                     "(PCIe-bound); layer by layer on a copy stream, outputs back on a third stream"},
+        "sustained": sustained,
         "paper_context": "paper reports >29x end-to-end speedup at 32K on H200 (whole model vs no KV cache): context only",
     }
     if cpu:
         out["cpu_baseline"] = cpu
     print(json.dumps(out))
+
+
+def tensor_roofline(tflops, P, kernel):
+    """Roofline object of a tensor-bound launch timed alone: fraction of the measured burst bf16 peak, with the
+    sustained and nominal fractions beside it."""
+    return {"bound": "tensor", "achieved": tflops, "peak": P["tf_burst"], "unit": "TFLOP/s", "frac": tflops / P["tf_burst"],
+            "frac_of_sustained": tflops / P["tf_sust"], "frac_of_nominal": tflops / 2250.0, "kernel": kernel,
+            "peak_source": f"{P['src']} burst bf16 (cuBLAS 8192^3); sustained {P['tf_sust']}, nominal 2250"}
 
 
 def graph_time_us(fn, n_layers, warm=10, reps=50):
@@ -713,6 +866,36 @@ def run_stages(args):
     print(json.dumps(out))
 
 
+def spawn_ranks(n, argv):
+    """`bench.py --gpus N` started as a plain process: start the N ranks here (one per GPU, rendezvous on 127.0.0.1)
+    the way an outer launcher would have, and hand their exit code back."""
+    import socket
+    with socket.socket() as so:
+        so.bind(("127.0.0.1", 0))
+        port = so.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr",
+           "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+    return subprocess.call(cmd)
+
+
+def run_stub(args):
+    """Host-only stand-in for the step (no GPU, gloo): exercises the launcher, the rendezvous, the barrier and the
+    max-over-ranks timing that the real arm uses, and prints a line of the same outer shape."""
+    from paper_2602_02159_b200 import replicas
+    rank, world, _ = replicas.init("gloo")
+    replicas.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(0.001 * (1 + rank))                 # rank r takes r + 1 ms per step: the slowest rank sets the time
+    ms = replicas.max_over_ranks((time.perf_counter() - t0) * 1e3) / max(1, args.steps)
+    replicas.barrier()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": ms, "unit": "ms", "n_gpus": world, "steps": args.steps,
+                          "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak",
+                          "stub": True}))
+    replicas.shutdown()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -728,8 +911,15 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="run the context x keep-ratio sweep (config 4) instead")
     ap.add_argument("--clock-interval-ms", type=int, default=25, help="nvidia-smi sampling period during timed regions")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle baseline leg")
+    ap.add_argument("--sustain-s", type=float, default=2.0,
+                    help="seconds of back-to-back graph replays for the sustained figure (0 = skip)")
+    ap.add_argument("--stub-step", action="store_true", help=argparse.SUPPRESS)   # host-only step: tests of the launcher
     args = ap.parse_args()
-    if args.stages:
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.stages or args.sweep):
+        sys.exit(spawn_ranks(args.gpus, sys.argv[1:]))
+    if args.stub_step:
+        run_stub(args)
+    elif args.stages:
         run_stages(args)
     elif args.sweep:
         run_sweep(args)

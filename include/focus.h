@@ -24,7 +24,11 @@
  *     for its predecessor to complete before it writes anything, and before it reads anything that another of
  *     these kernels may have written (outputs, lists, workspace).  Caller-visible ordering is plain stream
  *     order: a kernel of another library placed before or after a call sees complete results, and inputs
- *     produced on the same stream before a call are complete when the call's kernels read them.
+ *     produced on the same stream before a call by any kernel that does not release its successor early -- every
+ *     kernel outside this library, and every kernel of this library except the attention kernels and the selection
+ *     kernel of focus_sparse_layer -- are complete when the call's kernels read them.  The one thing not to do is
+ *     to feed the O or lse of one attention call straight in as the Q, q_rows or n_rows of the next attention or
+ *     focus_sparse_layer call with no other kernel in between: those three are read ahead of the wait.
  *   - Results are deterministic run to run (fixed reduction order, no floating-point atomics).
  *   - A device-side anomaly (index out of range, a bounded wait that ran out) never traps: the kernel
  *     skips the access, records a code in the context's device status word and returns; read it with
@@ -107,6 +111,17 @@ int32_t focus_last_attn_variant(focus_ctx* ctx);
  * kernel where supported), 1 = force the generic SIMT kernels.  Returns the previous value. */
 int32_t focus_set_force_simt(focus_ctx* ctx, int32_t force);
 
+/* Launch options of the attention kernels (no counterpart in the paper): every one of them selects between
+ * implementations that return the same results, for tests that must reach a fallback and for A/B measurements.
+ *   FOCUS_OPT_MERGE_MODE  how the key splits of a query tile are merged: 0 = automatic (inside a thread-block cluster
+ *                         where all clusters of the launch are resident), 1 = through global memory by the CTA that
+ *                         arrives last at the tile's counter, 2 = through global memory by a separate kernel
+ *   FOCUS_OPT_NO_WIDE     1 = never use the three-warpgroup kernels (variants 3 and 4 of focus_last_attn_variant)
+ *   FOCUS_OPT_NO_PDL      1 = plain stream order, no programmatic dependent launches
+ * Returns the previous value, or -1 for a bad context, option or value. */
+typedef enum { FOCUS_OPT_MERGE_MODE = 0, FOCUS_OPT_NO_WIDE = 1, FOCUS_OPT_NO_PDL = 2 } focus_option;
+int32_t focus_set_option(focus_ctx* ctx, int32_t option, int32_t value);
+
 /* Self-test of the bounded waits (no counterpart in the paper).  Every wait on a barrier inside the tensor-core
  * kernels gives up after a time limit, records FOCUS_ERR_TIMEOUT in the status word and lets the kernel unwind
  * instead of spinning for ever.  This call launches one small CTA that waits, with a limit of limit_us microseconds
@@ -184,8 +199,9 @@ focus_status focus_score_blocks(focus_ctx* ctx, const focus_shape* shape, const 
  * rejected with FOCUS_ERR_WORKSPACE_TOO_SMALL before anything is launched: n_kv_heads * head_dim <= 8192 and, in
  * FOCUS_HEADS_ALL mode, n_kv_heads * nb <= 65536.
  *
- * The first call on each device looks up the array's device address (that device must be current); make that
- * first call before any stream capture begins.  All calls share the one array and it keeps the previous call's
+ * The first call on each device looks up the array's device address (that device must be current); if nothing of
+ * the library has run on that device yet, this lookup is also the moment the runtime loads the library's device
+ * code there and places the array.  Make that first call before any stream capture begins.  All calls share the one array and it keeps the previous call's
  * contents; every element a call reads it has first rewritten, so nothing needs clearing, but two calls whose
  * kernels overlap on the GPU (different streams, or several processes' worth of threads on one context) race on
  * it: serialise them.
@@ -249,7 +265,7 @@ focus_status focus_dense_attn(focus_ctx* ctx, const focus_shape* shape, const vo
 /* Eq. 2: for each listed position, the predicted token argmax_v p(v) (lowest v on ties; NaN logits count as
  * -inf) and its confidence c = max_v p(v), p = softmax over the vocabulary of that position's logits row.
  * The confidences are the conf_prev of the next step's focus_select_queries; the same selection call with
- * k = n^(t) and w = 0 picks the positions to unmask ("unmasks the highest-confidence positions").
+ * k = n^(t) and w = 0 picks the positions to unmask (the unmasking rule of the section on diffusion LLM inference).
  *   logits    [n_pos rows, vocab] for positions [pos_base, pos_base + n_pos), dtype FOCUS_F32 or FOCUS_BF16;
  *             row_stride in elements, a multiple of 8 (bf16) / 4 (f32); base 16-byte aligned
  *   rows      int32[max_rows] positions (device) with n_rows int32[1] (device), or both NULL: the first max_rows
@@ -259,7 +275,7 @@ focus_status focus_confidence(focus_ctx* ctx, const void* logits, int32_t dtype,
                               int32_t pos_base, int32_t n_pos, const int32_t* rows, const int32_t* n_rows,
                               int32_t max_rows, float* conf, int32_t* token, focus_stream stream);
 
-/* Eq. 3 / Algorithm 1 ("Update KV Cache for indices in I_active"): the key and value states computed this
+/* Eq. 3; Algorithm 1, the cache-update step of the non-block-entry branch: the key and value states computed this
  * step for the listed positions replace the cached rows; every other row keeps its cached state.
  *   K_cache, V_cache  [Hkv, L, d] by the shape's strides (updated in place)
  *   K_new, V_new      [max_rows, Hkv, d] contiguous; row r belongs to position rows[r]

@@ -16,6 +16,8 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_TIM
 F32, BF16 = 0, 1
 HEADS_PER_KV_GROUP, HEADS_ALL = 0, 1
 SINK_TOKENS, SINK_BLOCKS = 0, 1
+OPT_MERGE_MODE, OPT_NO_WIDE, OPT_NO_PDL = 0, 1, 2
+MERGE_AUTO, MERGE_COUNTERS, MERGE_KERNEL = 0, 1, 2
 
 
 class FocusError(RuntimeError):
@@ -42,6 +44,7 @@ _SIGS = {
     "focus_poll_status": (_I, [_P, _P, C.POINTER(_I)]),
     "focus_status_string": (C.c_char_p, [_I]),
     "focus_set_force_simt": (_I, [_P, _I]),
+    "focus_set_option": (_I, [_P, _I, _I]),
     "focus_selftest_bounded_wait": (_I, [_P, _I, _P]),
     "focus_stream_read": (_I, [_P, _P, _Z, _P, _P]),
     "focus_launch_count": (C.c_uint64, []),
@@ -146,6 +149,13 @@ class Context:
 
     def set_force_simt(self, force: bool) -> int:
         return self._lib.focus_set_force_simt(self.handle, 1 if force else 0)
+
+    def set_option(self, option: int, value: int) -> int:
+        """focus_set_option: returns the previous value; raises on a bad option or value."""
+        prev = self._lib.focus_set_option(self.handle, int(option), int(value))
+        if prev < 0:
+            raise FocusError(ERR_INVALID_ARG, "focus_set_option")
+        return prev
 
     def selftest_bounded_wait(self, limit_us: int, stream=None) -> None:
         """One small CTA waits limit_us microseconds on a barrier nobody arrives at, then gives up: poll_status()

@@ -44,9 +44,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
     if verbose:
         flags += ["-Xptxas", "-v"]
-    if os.environ.get("FOCUS_TIMELINE"):          # development: per-CTA timestamps in the attention kernel
-        flags += ["-DFOCUS_TIMELINE"]
-    flags += os.environ.get("FOCUS_EXTRA_NVCC_FLAGS", "").split()     # development: experiment switches
 
     def compile_one(src):
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")

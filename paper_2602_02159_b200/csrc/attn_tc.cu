@@ -43,11 +43,12 @@ constexpr int NBAR = 2 * NSLOT + 7;
 constexpr int MAXT = 128;            // key tiles of a split whose descriptors are staged in shared memory
 constexpr int SMEM_BYTES = 1024 + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8 + 64 + MAXT * 8;
 constexpr int NTHREADS = 192;
-#ifndef FOCUS_PREF_TILES
-#define FOCUS_PREF_TILES 1
-#endif
-constexpr int PREF_TILES = FOCUS_PREF_TILES;   // key tiles (K and V) warmed in L2 ahead of the dependency wait
+constexpr int PREF_TILES = 1;                  // key tiles (K and V) warmed in L2 ahead of the dependency wait
 constexpr float RESCALE_THRESHOLD = 8.0f;      // log2 units: O is rescaled only when the row max grew by more
+// which kernel form a launch takes (measured cross-overs, see the launcher)
+constexpr int WIDE_MIN_TILES = 24;             // two-tile form: at least this many key tiles per CTA
+constexpr int KP_MIN_ROWS = 128;               // key-pair form: at least this many stacked rows per KV head ...
+constexpr int KP_MIN_TILES = 4;                // ... and this many key tiles per CTA
 
 struct TcParams {
   const __nv_bfloat16* Q;
@@ -69,23 +70,8 @@ struct TcParams {
   int pair;                    // 1: 64-token KV blocks, two selected blocks per 128-key tile; tmK / tmV have 64-row boxes
   float scale_log2;            // softmax scale * log2(e)
   int32_t* status;
-#ifdef FOCUS_TIMELINE
-  unsigned long long* dbg;     // per-CTA timestamps (development builds only)
-#endif
 };
 
-#ifdef FOCUS_TIMELINE
-#define TL_STAMP(slot, tid) do { if (p.dbg && threadIdx.x == (tid)) p.dbg[(blockIdx.x * gridDim.y + blockIdx.y) * 16 + (slot)] = global_ns(); } while (0)
-// per-iteration trace of CTA (0,0): who 0 = MMA thread, 1 = first softmax thread of tile A, 2 = of tile B
-__device__ __forceinline__ unsigned long long tl_clock() { unsigned long long c; asm volatile("mov.u64 %0, %%clock64;" : "=l"(c) :: "memory"); return c; }
-#define TL_ITER(who, tid, it, ev) do { if (p.dbg && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == (tid) && (it) < 64) p.dbg[65536 + (who) * 512 + (it) * 8 + (ev)] = tl_clock(); } while (0)
-// per-CTA stamp in SM cycles (cheap to take: for intervals inside one CTA)
-#define TL_CLK(slot, tid) do { if (p.dbg && threadIdx.x == (tid)) p.dbg[(blockIdx.x * gridDim.y + blockIdx.y) * 16 + (slot)] = tl_clock(); } while (0)
-#else
-#define TL_CLK(slot, tid) do { } while (0)
-#define TL_STAMP(slot, tid) do { } while (0)
-#define TL_ITER(who, tid, it, ev) do { } while (0)
-#endif
 
 struct TileInfo {
   int kind;     // 0: tile of the K/V tensors, 1: tile of the gathered sink rows
@@ -383,13 +369,11 @@ __device__ __forceinline__ void cluster_merge(const TcParams& p, int g, int mt, 
   const int rows = min(ROWS, total_fr - mt * ROWS);
   const int S = p.n_splits;                                   // <= 8 in cluster mode
   const int mine = rank < rows ? (rows - rank + S - 1) / S : 0;
-  TL_STAMP(13, 0);
   if (tid >= 0) {
     if (S <= 2) cluster_merge_items<ROWS, NTH, 2>(p, g, mt, rank, spart, mine, tid);
     else if (S <= 4) cluster_merge_items<ROWS, NTH, 4>(p, g, mt, rank, spart, mine, tid);
     else cluster_merge_items<ROWS, NTH, 8>(p, g, mt, rank, spart, mine, tid);
   }
-  TL_STAMP(14, 128);
   cluster_sync_exit();                                         // nobody leaves while its partial may still be read
 }
 
@@ -415,7 +399,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   extern __shared__ uint8_t smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
-  TL_STAMP(0, 0);
 
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sptr = smem_raw + (sbase - smem_u32(smem_raw));
@@ -483,8 +466,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    TL_STAMP(7, 0);
-    TL_CLK(15, 0);
   }
   // Dense key set: which tiles this split streams is known without reading anything, so the first ring-full of
   // K/V copies starts right here, ahead of the chain row count -> row list -> query rows (about 3 us sooner than
@@ -537,7 +518,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   }
   const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
   const int total_fr = nrows * p.hpg;                    // stacked (row, head-of-group) rows of this KV head
-  TL_CLK(8, 0);
   if (mt * TM >= total_fr) {                             // uniform: nothing to compute for this tile
     if (p.pdl == 2) {                                    // TMEM was allocated ahead of the row count
       if (lane == 0)
@@ -576,8 +556,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     if (warp == 1) alloc_tmem();
     if (qtid >= 0) store_q();
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    TL_STAMP(7, 0);
-    TL_CLK(15, 0);
   }
   const int cnt_raw = p.dense ? 0 : ld_ordered(p.block_cnt + g * p.group_stride);
 
@@ -586,7 +564,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   const int t1 = split_lo(te.total, split + 1, p.n_splits);
   const int nt = t1 - t0;
   const int cta_lin = blockIdx.x * p.n_splits + split;
-  TL_CLK(9, 0);
 
   const bool use_list = !p.dense && nt <= MAXT;
   // tile descriptor: from the staged list (sparse) or by arithmetic (dense; splits longer than the list)
@@ -637,7 +614,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     isV = true; return (q >> 1) - 1;
   };
   const uint64_t l2_pol = l2_policy_evict_first();
-  TL_CLK(11, 0);
   auto issue = [&](int q) {
     bool isV;
     const int idx = seq_tile(q, isV);
@@ -658,11 +634,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
     }
     __syncwarp();
-    TL_CLK(10, 0);
     if (lane >= early_issued && lane < n_early) issue(lane);       // one copy per lane
     __syncwarp();
-    TL_CLK(12, 0);
-    TL_STAMP(6, 0);
   }
   if (warp == 1 && !p.pdl) alloc_tmem();
   // Q tile -> shared memory in the 128-byte-swizzled K-major layout the MMA descriptor expects:
@@ -674,7 +647,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem = *tmem_holder;
   const uint32_t tmem_O = tmem + 256;
-  TL_STAMP(1, 0);
 
   if (warp == 0) {
     // ================================ TMA producer ================================================
@@ -682,9 +654,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       int issued = n_early;
       bool ok = true;
       for (int q = n_early; q < n_loads; ++q) {
-        TL_ITER(2, 0, q, 0);
         if (!mbar_wait(bar_empty(q % NSLOT), (uint32_t)((q / NSLOT) & 1) ^ 1u, abort_flag, p.status)) { ok = false; break; }
-        TL_ITER(2, 0, q, 1);
         issue(q);
         ++issued;
       }
@@ -731,9 +701,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       for (int idx = 0; idx < nt && ok; ++idx) {
         const int b = idx & 1;
         const int slot = q % NSLOT;
-        TL_ITER(0, 32, idx, 0);
         if (!mbar_wait(bar_full(slot), (q / NSLOT) & 1u, abort_flag, p.status)) { ok = false; break; }
-        TL_ITER(0, 32, idx, 1);
         tc_fence_after();
         const uint64_t kdesc = make_sdesc(sSlot + slot * SLOT_BYTES, 16, 1024);
 #pragma unroll
@@ -746,9 +714,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         tc_commit(bar_empty(slot));
         tc_commit(bar_sfull(b));
         ++q;
-        TL_ITER(0, 32, idx, 2);
         if (idx > 0) ok = do_pv(idx - 1);
-        TL_ITER(0, 32, idx, 3);
       }
       if (ok) ok = do_pv(nt - 1);
     }
@@ -761,12 +727,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     bool ok = true;
     for (int idx = 0; idx < nt; ++idx) {
       const int b = idx & 1;
-      TL_ITER(1, 64, idx, 0);
       // votes keep the warp together: the TMEM loads and stores below are warp-collective
       if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(b), (uint32_t)(idx >> 1) & 1u, abort_flag, p.status))) { ok = false; break; }
-      TL_ITER(1, 64, idx, 1);
       tc_fence_after();
-      if (idx == 0) TL_STAMP(5, 64);
       uint32_t sreg[128];
       const uint32_t ts = tmem + lane_off + b * 128;
       TC_LD32(ts, (sreg + 0));
@@ -774,7 +737,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       TC_LD32(ts + 64, (sreg + 64));
       TC_LD32(ts + 96, (sreg + 96));
       tc_wait_ld();
-      TL_ITER(1, 64, idx, 2);
       const TileInfo ti = get_tile(idx);
       float tmax = -INFINITY;
       if (ti.kind == 0 && ti.nvalid == TN) {
@@ -835,7 +797,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           TC_ST32(tmem_O + lane_off + cb * 32, oreg);
         }
       }
-      TL_ITER(1, 64, idx, 3);
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {                 // 32 keys at a time: exponentials, bf16 P, row sum
@@ -854,13 +815,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           tc_wait_st();
           tc_fence_before();
           mbar_arrive(bar_pready(b));
-          TL_ITER(1, 64, idx, 4);
         }
       }
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar_pready2(b));
-      TL_ITER(1, 64, idx, 5);
       l = l * alpha + ((acc[0] + acc[1]) + (acc[2] + acc[3]));
     }
     // ---- epilogue: wait for the last P V, normalise, write out -----------------------------------
@@ -933,7 +892,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
     }
   }
-  TL_STAMP(2, 64);
   // ---- teardown: every role converges here, also after a timed-out wait --------------------------
   tc_fence_before();
   __syncthreads();
@@ -941,10 +899,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     __syncwarp();
     tmem_dealloc(tmem, 512);
   }
-  TL_STAMP(3, 0);
   if (p.cluster) cluster_merge<TM, NTHREADS>(p, g, mt, total_fr, split, sSlot, (int)threadIdx.x);
   else if (p.n_splits > 1 && p.counters) finish_split(p, blockIdx.x, g, mt, total_fr, s_last_p, reinterpret_cast<float*>(sptr + Q_BYTES));
-  TL_STAMP(4, 0);
 }
 
 // ================================================================================================================
@@ -976,7 +932,6 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                     const __grid_constant__ CUtensorMap tmSK, const __grid_constant__ CUtensorMap tmSV, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  TL_STAMP(0, 0);
   const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
   // programmatic dependent launch: let the successor start early; wait for the predecessor before touching memory
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -1098,7 +1053,6 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_holder;
-  TL_STAMP(1, 0);
   if (warp < 4) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
   if (warp == 0) {
@@ -1194,24 +1148,18 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       for (int j = 0; j < nt && ok; ++j) {
         const uint32_t par = (uint32_t)j & 1u;
         if (!wait_load(2 * j + 1)) { ok = false; break; }            // V_j
-        TL_ITER(0, 32, j, 0);
         if (!do_pv(0, j, par, j == 0)) { ok = false; break; }
-        TL_ITER(0, 32, j, 4);
         if (j + 1 < nt) {
           if (!wait_load(2 * j + 2)) { ok = false; break; }          // K_(j+1)
           tc_fence_after();
           do_qk(0, j + 1);
         }
-        TL_ITER(0, 32, j, 5);
-        TL_ITER(0, 32, j, 2);
         if (!do_pv(1, j, par, j == 0)) { ok = false; break; }
         tc_commit(bar_empty((2 * j + 1) % NSLOT_W));                 // V_j
-        TL_ITER(0, 32, j, 6);
         if (j + 1 < nt) {
           do_qk(1, j + 1);
           tc_commit(bar_empty((2 * j + 2) % NSLOT_W));               // K_(j+1)
         }
-        TL_ITER(0, 32, j, 7);
       }
       }
       tc_commit(bar_alldone);
@@ -1225,9 +1173,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       __syncwarp();
       tmem_dealloc(tmem, 512);
     }
-    TL_STAMP(3, 0);
     if (p.n_splits > 1) cluster_merge<TMQ, 256>(p, g, mt, total_fr, split, sSlot, -1);
-    TL_STAMP(4, 0);
   } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
     const int x = (warp - 4) >> 2;                                   // query tile of this softmax warp
@@ -1240,9 +1186,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     bool ok = true;
     const int nt_x = KP ? (nt - x + 1) / 2 : nt;                     // key tiles of this warpgroup
     for (int idx = 0; idx < nt_x; ++idx) {
-      TL_ITER(warp - 3, warp * 32, idx, 0);
       if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(x), (uint32_t)idx & 1u, abort_flag, p.status))) { ok = false; break; }
-      TL_ITER(warp - 3, warp * 32, idx, 1);
       tc_fence_after();
       uint32_t sreg[128];
       TC_LD32(ts, (sreg + 0));
@@ -1250,7 +1194,6 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       TC_LD32(ts + 64, (sreg + 64));
       TC_LD32(ts + 96, (sreg + 96));
       tc_wait_ld();
-      TL_ITER(warp - 3, warp * 32, idx, 2);
       const TileInfo ti = get_tile(KP ? 2 * idx + x : idx);
       float tmax = -INFINITY;
       if (ti.kind == 0 && ti.nvalid == TN) {
@@ -1307,7 +1250,6 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           TC_ST32(to + cb * 32, oreg);
         }
       }
-      TL_ITER(warp - 3, warp * 32, idx, 3);
       float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int ch = 0; ch < 4; ++ch) {                               // 32 keys at a time: exponentials, bf16 P, row sum
@@ -1326,17 +1268,14 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
           tc_wait_st();
           tc_fence_before();
           mbar_arrive(bar_pready(x));
-          TL_ITER(warp - 3, warp * 32, idx, 4);
         }
       }
       tc_wait_st();
       tc_fence_before();
       mbar_arrive(bar_pready2(x));
       l = l * alpha + ((acc[0] + acc[1]) + (acc[2] + acc[3]));
-      TL_ITER(warp - 3, warp * 32, idx, 5);
     }
     if (ok && nt_x > 0) ok = __all_sync(0xffffffffu, mbar_wait(bar_pvdone(x), (uint32_t)(nt_x - 1) & 1u, abort_flag, p.status));
-    TL_STAMP(2, 128);
     if (KP) {
       // Merge of the two warpgroups' halves.  Both accumulators are complete once every MMA of the CTA has retired;
       // the (reference max, row sum) pairs cross through shared memory (over the K/V ring, idle by then).
@@ -1601,8 +1540,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   const int ns_pad = a.dense ? 0 : (a.n_sink + TN - 1) / TN * TN;
   const int n_resp = a.dense ? (sh.L + TN - 1) / TN : (sh.L - sh.M + TN - 1) / TN;
   // 64-token KV blocks: two selected blocks share a 128-key tile
-  static const bool no_pair = getenv("FOCUS_NO_PAIR") != nullptr;          // A/B switch: one block per tile
-  const bool pair = !a.dense && sh.kv_block == 64 && !no_pair;
+  const bool pair = !a.dense && sh.kv_block == 64;
   const int max_tiles = a.dense ? n_resp : (pair ? (a.max_blocks + 1) / 2 : a.max_blocks) + ns_pad / TN + n_resp;
   bool& attr_set = ctx->ls.attn_attr_set;
   if (!attr_set) {
@@ -1632,8 +1570,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     // it pays from about 24 key tiles per CTA upward (measured at 256 rows, 32 heads: 32 tiles per CTA 85 us against
     // 87 us for the key-pair form, 17 to 19 tiles per CTA 3 to 12 % slower than it); below that the one-tile forms,
     // which need fewer or no key splits, win
-    static const int wide_min = getenv("FOCUS_WIDE_MIN") ? atoi(getenv("FOCUS_WIDE_MIN")) : 24;
-    if (max_tiles / n_splits < wide_min) wide = false;
+    if (max_tiles / n_splits < WIDE_MIN_TILES) wide = false;
   }
   // key-pair form: one query tile per CTA, two softmax warpgroups on alternating key tiles.  For query sets with
   // enough rows per tile to be bound by the exponentials (not by HBM) that the two-tile form does not take.
@@ -1642,9 +1579,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     n_mtiles = (int)((stacked + TM - 1) / TM);
     base = n_mtiles * Hkv;
     n_splits = pick_splits(ctx, base, max_tiles);
-    static const int kp_min_rows = getenv("FOCUS_KP_MIN_ROWS") ? atoi(getenv("FOCUS_KP_MIN_ROWS")) : 128;
-    static const int kp_min_tiles = getenv("FOCUS_KP_MIN_TILES") ? atoi(getenv("FOCUS_KP_MIN_TILES")) : 4;
-    if (!ctx->no_wide && stacked >= kp_min_rows && max_tiles / n_splits >= kp_min_tiles &&
+    if (!ctx->no_wide && stacked >= KP_MIN_ROWS && max_tiles / n_splits >= KP_MIN_TILES &&
         (n_splits == 1 || ctx->merge_mode == 0)) {
       kpair = true;
       if (n_splits > 1) {                                                // its splits merge through a cluster only
@@ -1722,9 +1657,6 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.n_mtiles = n_mtiles; p.n_splits = n_splits; p.lse_stride = a.lse_stride;
   p.scale_log2 = a.scale * 1.4426950408889634f;
   p.status = ctx->d_status;
-#ifdef FOCUS_TIMELINE
-  p.dbg = getenv("FOCUS_TIMELINE") ? (unsigned long long*)(ctx->ws + ctx->ws_bytes - (1 << 20)) : nullptr;
-#endif
 
   ctx->last_attn_variant = wide ? 3 : (kpair ? 4 : 2);
   if (wide) {

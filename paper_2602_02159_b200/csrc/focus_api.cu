@@ -49,12 +49,9 @@ extern "C" focus_status focus_create(focus_ctx** out, int device, size_t workspa
   c->ws_bytes = workspace_bytes ? workspace_bytes : (size_t)256 << 20;
   c->force_simt = 0;
   c->last_attn_variant = 0;
-  c->no_wide = getenv("FOCUS_NO_WIDE") != nullptr;
-  c->no_pdl = getenv("FOCUS_NO_PDL") != nullptr;
-  {
-    const char* mm = getenv("FOCUS_MERGE");
-    c->merge_mode = !mm ? 0 : (!strcmp(mm, "counters") ? 1 : (!strcmp(mm, "kernel") ? 2 : 0));
-  }
+  c->no_wide = 0;
+  c->no_pdl = 0;
+  c->merge_mode = 0;
   c->encode_tiled = nullptr;
   if (prop.major == 10) {   // tensor-core kernels are built for sm_100a only
     cudaDriverEntryPointQueryResult q;
@@ -88,6 +85,22 @@ extern "C" int32_t focus_set_force_simt(focus_ctx* ctx, int32_t force) {
   if (!ctx) return -1;
   const int prev = ctx->force_simt;
   ctx->force_simt = force ? 1 : 0;
+  return prev;
+}
+
+extern "C" int32_t focus_set_option(focus_ctx* ctx, int32_t option, int32_t value) {
+  if (!ctx) return -1;
+  int* slot = nullptr;
+  int max_value = 1;
+  switch (option) {
+    case FOCUS_OPT_MERGE_MODE: slot = &ctx->merge_mode; max_value = 2; break;
+    case FOCUS_OPT_NO_WIDE: slot = &ctx->no_wide; break;
+    case FOCUS_OPT_NO_PDL: slot = &ctx->no_pdl; break;
+    default: return -1;
+  }
+  if (value < 0 || value > max_value) return -1;
+  const int prev = *slot;
+  *slot = value;
   return prev;
 }
 
@@ -213,7 +226,3 @@ extern "C" focus_status focus_find_sinks(focus_ctx* ctx, const focus_shape* shap
   return launch_sink_select(ctx, part, H, L, n_active, S, cand_lo, cand_hi, n_sink, sink_idx, stream);
 }
 
-#ifdef FOCUS_TIMELINE
-// Development builds only: where the attention kernel drops its per-CTA timestamps (last MiB of the workspace).
-extern "C" void* focus_debug_ptr(focus_ctx* ctx) { return ctx->ws + ctx->ws_bytes - (1 << 20); }
-#endif

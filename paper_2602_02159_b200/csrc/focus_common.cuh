@@ -16,8 +16,8 @@ struct focus_ctx {
   int32_t* d_counters; // FOCUS_N_COUNTERS arrival counters for split merges; zero between launches
   int force_simt;
   int last_attn_variant;   // 0 none yet, 1 SIMT, 2 tensor-core 128-row tiles, 3 tensor-core 256-row tiles, 4 key-pair form
-  int no_pdl;          // 1: never launch the attention kernel as a programmatic dependent (A/B comparisons)
-  int no_wide;         // 1: never use the two-query-tile attention kernel (A/B comparisons)
+  int no_pdl;          // 1: never launch the attention kernel as a programmatic dependent (focus_set_option)
+  int no_wide;         // 1: never use the three-warpgroup attention kernels (focus_set_option)
   int merge_mode;      // split merge of the one-tile kernel: 0 automatic (cluster where it fits), 1 never a cluster (arrival
                        // counters), 2 neither (separate combine kernel); tests use 1 and 2 to reach the fallbacks
   void* encode_tiled;  // cuTensorMapEncodeTiled, resolved through the runtime (no libcuda link)
@@ -93,6 +93,12 @@ __device__ __forceinline__ uint32_t float_key(float x) {
   uint32_t u = __float_as_uint(x);
   u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
   return u == 0u ? 1u : u;   // keep 0 for NaN only (~0xFFFFFFFF is a NaN pattern anyway)
+}
+
+// Inverse of float_key: the float a key came from (NaN for key 0; -0 comes back as +0).
+__device__ __forceinline__ float key_to_float(uint32_t k) {
+  if (k == 0u) return __uint_as_float(0x7FC00000u);
+  return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
 }
 
 __device__ __forceinline__ float load_as_float(const float* p) { return *p; }

@@ -3,8 +3,8 @@
 //                        (an HBM-bound streaming reduction over the vocabulary; its output is the conf_prev of the
 //                        next step's focus_select_queries, and with k = n, w = 0 the same call picks the tokens
 //                        to unmask);
-//   focus_update_kv   -- Eq. 3 / Algorithm 1 "Update KV Cache for indices in I_active": the refreshed rows replace
-//                        the cached K and V rows.
+//   focus_update_kv   -- Eq. 3; Algorithm 1, the cache-update step of the non-block-entry branch: the refreshed
+//                        rows replace the cached K and V rows.
 #include "focus_common.cuh"
 
 namespace {

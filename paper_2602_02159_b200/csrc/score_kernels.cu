@@ -195,7 +195,10 @@ constexpr int STATIC_SCRATCH_FLOATS = STATIC_QBAR_FLOATS + STATIC_RG_FLOATS + 64
 static __device__ __align__(256) float g_static_scratch[STATIC_SCRATCH_FLOATS];
 
 // In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel may use: the device
-// address is looked up once per device (with that device current) and cached here.
+// address is looked up once per device (with that device current) and cached here.  The cache is written without a
+// lock: two host threads racing on a device's first call both store the same address, so whichever store lands
+// last changes nothing.  That first lookup also makes the runtime load this module onto the device (which is where
+// the array gets its memory), one more reason to make the first call outside any stream capture.
 constexpr int STATIC_MAX_DEVICES = 64;
 static float* g_static_scratch_dev[STATIC_MAX_DEVICES] = {nullptr};
 

@@ -37,17 +37,8 @@ struct SinkParams {
   int kv_div;                     // the kernel walks QUERY heads (Hkv = H, hpg = 1); query head h reads KV head h / kv_div
   float scale_log2;
   int32_t* status;
-#ifdef FOCUS_TIMELINE
-  unsigned long long* dbg;        // per-iteration clock stamps of CTA 0 (development builds only)
-#endif
 };
 
-#ifdef FOCUS_TIMELINE
-__device__ __forceinline__ unsigned long long tl_clock() { unsigned long long c; asm volatile("mov.u64 %0, %%clock64;" : "=l"(c) :: "memory"); return c; }
-#define TL_ITER(who, tid, it, ev) do { if (p.dbg && blockIdx.x == 0 && threadIdx.x == (tid) && (it) < 64) p.dbg[65536 + (who) * 512 + (it) * 8 + (ev)] = tl_clock(); } while (0)
-#else
-#define TL_ITER(who, tid, it, ev) do { } while (0)
-#endif
 
 #define TC_LD16(taddr, r)                                                                                         \
   asm volatile(                                                                                                   \
@@ -138,9 +129,7 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
       int t = u0 % T, g = u0 / T, kvh = g / p.kv_div, slot = 0;
       uint32_t ph = 0;
       for (int i = 0; i < nt && ok; ++i) {
-        TL_ITER(0, 0, i, 0);
         if (!mbar_wait(bar_empty(slot), ph ^ 1u, abort_flag, p.status)) { ok = false; break; }
-        TL_ITER(0, 0, i, 1);
         const uint32_t dst = sSlot + slot * SLOT_BYTES;
         mbar_expect_tx(bar_full(slot), SLOT_BYTES);
         tma_load_3d_hint(dst, &tmK, bar_full(slot), 0, t * TK, kvh, l2_pol);
@@ -169,11 +158,8 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
       uint32_t ph = 0;
       for (int u = 0; u < units && ok; ++u) {
         const int b = u & nbuf_mask;
-        TL_ITER(1, 32, u, 0);
         if (!mbar_wait(bar_sempty(b), ((uint32_t)(u >> nbuf_shift) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
-        TL_ITER(1, 32, u, 1);
         if (hh == 0 && !mbar_wait(bar_full(slot), ph, abort_flag, p.status)) { ok = false; break; }
-        TL_ITER(1, 32, u, 2);
         tc_fence_after();
         const uint64_t kdesc = make_sdesc(sSlot + slot * SLOT_BYTES, 16, 1024);
         const uint64_t qdesc = make_sdesc(sQ + (hs0 + hh) * q_head_bytes, 16, 1024);
@@ -190,7 +176,6 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
           if (++slot == p.n_slots) { slot = 0; ph ^= 1u; }
           if (++t == T) { t = 0; hs0 += p.hpg; }
         }
-        TL_ITER(1, 32, u, 3);
       }
     }
   } else {
@@ -204,9 +189,7 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
     int t = (u0 + i) % T, g = (u0 + i) / T;
     for (int u = cw; u < units; u += 2) {
       const int b = u & nbuf_mask;
-      TL_ITER(2, 64, u, 0);
       if (!__all_sync(0xffffffffu, mbar_wait(bar_sfull(b), (uint32_t)(u >> nbuf_shift) & 1u, abort_flag, p.status))) break;
-      TL_ITER(2, 64, u, 1);
       tc_fence_after();
       const float* nl = neg_lse2 + ((g - g0) * p.hpg + hh) * p.n_pad;
       float acc = 0.f;
@@ -224,7 +207,6 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
         if (c0 + 64 >= ncol) {
           tc_fence_before();
           mbar_arrive(bar_sempty(b));
-          TL_ITER(2, 64, u, 2);
         }
 #pragma unroll
         for (int hf = 0; hf < 2; ++hf) {
@@ -243,7 +225,6 @@ sink_colsum_tc_kernel(const __grid_constant__ CUtensorMap tmK, const SinkParams 
       acc = (acc4[0] + acc4[1]) + (acc4[2] + acc4[3]);
       const int key = t * TK + krow;
       if (key < p.L) p.part[(size_t)(g * p.hpg + hh) * p.L + key] = acc;
-      TL_ITER(2, 64, u, 3);
       hh += 2;
       while (hh >= p.hpg) {
         hh -= p.hpg;
@@ -311,9 +292,6 @@ focus_status launch_sink_colsum_tc(focus_ctx* ctx, const focus_shape* s, const v
   p.n_slots = sink_slots(p.groups_staged * hpg, p.n_pad);
   p.scale_log2 = shape_scale(s) * 1.4426950408889634f;
   p.status = ctx->d_status;
-#ifdef FOCUS_TIMELINE
-  p.dbg = getenv("FOCUS_TIMELINE") ? (unsigned long long*)(ctx->ws + ctx->ws_bytes - (1 << 20)) : nullptr;
-#endif
   CUtensorMap tmK;
   if (!encode_kv_map(ctx->encode_tiled, &tmK, K, HD, s->L, kvh, s->kv_stride_tok, s->kv_stride_head, 64, TK))
     return FOCUS_ERR_INVALID_ARG;

@@ -103,10 +103,7 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
       float s = kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-      if (lane == 0) {
-        key[b] = float_key(s);
-        if (R) R[(size_t)g * nb + b] = s;
-      }
+      if (lane == 0) key[b] = float_key(s);             // R itself is written after the dependency wait, from the key
     };
 #pragma unroll
     for (int u = 0; u < KPRE; ++u) {
@@ -133,6 +130,10 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
     block_topc_mark(key, nb, C, sel, hist, scan_s);
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");
+  // every store comes after the wait: the previous layer's selection kernel (which may still have been storing when
+  // this one started) wrote the same R, lists and flags
+  if (R)
+    for (int b = tid; b < nb; b += FS_THREADS) R[(size_t)g * nb + b] = key_to_float(key[b]);
   for (int s = tid; s < ns_pad; s += FS_THREADS) {
     uint8_t keep = 0, mk = 0;
     if (s < n_sink) {

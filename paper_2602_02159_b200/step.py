@@ -42,7 +42,10 @@ class StepBuffers:
     wl: Workload
     head_reduce: int = fb.HEADS_PER_KV_GROUP
     sink_mode: int = fb.SINK_TOKENS
-    rows: str = "active"              # "active": attention rows are I_active (the paper); "gen": all N gen rows
+    # "active": attention rows are I_active (the paper), Q holds every gen row; "gen": all N gen rows are attention rows;
+    # "compact": attention rows are I_active and Q holds ONLY those rows, in list order (a caller that computed or
+    # uploaded nothing else): row r of Q belongs to position active_idx[r]
+    rows: str = "active"
     device: str = "cuda"
 
     def __post_init__(self):
@@ -63,15 +66,32 @@ class StepBuffers:
         self.block_idx = torch.full((self.G * self.max_blocks,), -1, **i32)
         self.block_cnt = torch.zeros(self.G, **i32)
         self.sink_keep = torch.zeros(self.G * max(1, w.n_sink), dtype=torch.uint8, device=dev)
-        self.max_rows = self.max_active if self.rows == "active" else s.N
+        self.max_rows = s.N if self.rows == "gen" else self.max_active
         self.O = torch.zeros(self.max_rows, s.H, s.d, dtype=torch_dtype(s.dtype), device=dev)
         self.lse = torch.zeros(s.H, self.max_rows, dtype=torch.float32, device=dev)
+        # compact mode: Q row r <-> active_idx[r]; the library is handed local row numbers
+        self.row_ids = torch.arange(self.max_active, **i32)
+        self.focus_local = torch.full((max(1, w.k),), -1, **i32)
+        self.q_base = 0 if self.rows == "compact" else s.M
+        self.n_q = self.max_active if self.rows == "compact" else s.N
 
     # rows argument triple of the attention calls
     def _rows(self):
         if self.rows == "active":
             return self.active_idx, self.n_active, self.max_active
+        if self.rows == "compact":
+            return self.row_ids, self.n_active, self.max_active
         return None, None, 0
+
+    def _focus(self):
+        return self.focus_local if self.rows == "compact" else self.focus_idx
+
+    def set_local_focus(self, focus_pos, active_pos):
+        """Compact mode: where each focus position sits in the active list (index bookkeeping on the host, after the
+        caller has read the two lists back to gather its query rows)."""
+        where = {int(p): r for r, p in enumerate(active_pos)}
+        loc = [where[int(p)] for p in focus_pos]
+        self.focus_local[:len(loc)].copy_(torch.tensor(loc, dtype=torch.int32), non_blocking=True)
 
 
 def select_queries(ctx, b: StepBuffers, conf_prev: torch.Tensor, masked: torch.Tensor, stream=None):
@@ -83,14 +103,15 @@ def select_queries(ctx, b: StepBuffers, conf_prev: torch.Tensor, masked: torch.T
 def dense_layer(ctx, b: StepBuffers, Q, K, V, O=None, lse=None, stream=None):
     s = b.wl.shape
     q_rows, n_rows, max_rows = b._rows()
-    fb.focus_dense_attn(ctx, b.shape, Q, s.M, s.N, q_rows, n_rows, max_rows, K, V, b.O if O is None else O,
+    fb.focus_dense_attn(ctx, b.shape, Q, b.q_base, b.n_q, q_rows, n_rows, max_rows, K, V, b.O if O is None else O,
                         b.lse if lse is None else lse, stream)
 
 
 def find_sinks(ctx, b: StepBuffers, Q, K, lse: Optional[torch.Tensor], stream=None):
     """lse must be the [H, max_active] log-sum-exp of a dense pass over the I_active rows, or None."""
     w, s = b.wl, b.wl.shape
-    fb.focus_find_sinks(ctx, b.shape, Q, s.M, b.active_idx, b.n_active, b.max_active, K, lse, w.n_sink, 0, s.M,
+    act = b.row_ids if b.rows == "compact" else b.active_idx
+    fb.focus_find_sinks(ctx, b.shape, Q, b.q_base, act, b.n_active, b.max_active, K, lse, w.n_sink, 0, s.M,
                         b.sink_idx, b.sink_scores, stream)
 
 
@@ -101,15 +122,15 @@ def sparse_layer(ctx, b: StepBuffers, Q, K, V, Kbar: Optional[torch.Tensor] = No
     w, s = b.wl, b.wl.shape
     q_rows, n_rows, max_rows = b._rows()
     if Kbar is not None and b.head_reduce == fb.HEADS_PER_KV_GROUP and b.sink_mode == fb.SINK_TOKENS and fused:
-        fb.focus_sparse_layer(ctx, b.shape, Q, s.M, s.N, q_rows, n_rows, max_rows, b.focus_idx, b.n_focus, max(1, w.k),
+        fb.focus_sparse_layer(ctx, b.shape, Q, b.q_base, b.n_q, q_rows, n_rows, max_rows, b._focus(), b.n_focus, max(1, w.k),
                               K, V, Kbar, w.C, b.sink_idx, w.n_sink, b.R, b.block_idx, b.block_cnt, b.sink_keep,
                               b.O if O is None else O, b.lse if lse is None else lse, stream)
         return
-    fb.focus_score_blocks(ctx, b.shape, Q, s.M, b.focus_idx, b.n_focus, max(1, w.k), None if Kbar is not None else K,
+    fb.focus_score_blocks(ctx, b.shape, Q, b.q_base, b._focus(), b.n_focus, max(1, w.k), None if Kbar is not None else K,
                           Kbar, b.head_reduce, b.R, stream)
     fb.focus_select_blocks(ctx, b.shape, b.R, b.head_reduce, w.C, b.sink_idx, w.n_sink, b.sink_mode, b.block_idx,
                            b.max_blocks, b.block_cnt, b.sink_keep, stream)
-    fb.focus_sparse_attn(ctx, b.shape, Q, s.M, s.N, q_rows, n_rows, max_rows, K, V, b.head_reduce, b.block_idx,
+    fb.focus_sparse_attn(ctx, b.shape, Q, b.q_base, b.n_q, q_rows, n_rows, max_rows, K, V, b.head_reduce, b.block_idx,
                          b.max_blocks, b.block_cnt, b.sink_idx, b.sink_keep, w.n_sink, b.O if O is None else O,
                          b.lse if lse is None else lse, stream)
 

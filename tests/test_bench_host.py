@@ -1,8 +1,12 @@
 """Host-side pieces of the benchmark that need no GPU: the clock record keeps only samples stamped inside a
-timed region and reports throttle reasons seen there."""
+timed region and reports throttle reasons seen there; `--gpus N` started as a plain process starts its N ranks
+itself; the oracle arm's line says that its value is extrapolated from a bounded sample."""
 import datetime
 import importlib.util
+import json
 import pathlib
+import subprocess
+import sys
 
 _spec = importlib.util.spec_from_file_location("bench", pathlib.Path(__file__).resolve().parents[1] / "bench.py")
 bench = importlib.util.module_from_spec(_spec)
@@ -47,3 +51,36 @@ def test_a_region_between_two_samples_is_flagged():
     rec = _sampler([_line(ms(0), 1000), _line(ms(100), 1200)], [(ms(40), ms(60), True)]).stop()
     assert rec["samples"] == 2 and rec["samples_in_headline_region"] == 0 and "note" in rec
     assert rec["sm_mhz"] == 1100
+
+
+BENCH = str(pathlib.Path(__file__).resolve().parents[1] / "bench.py")
+
+
+def test_gpus_flag_starts_the_ranks_itself():
+    """No outer launcher, no WORLD_SIZE: `--gpus 2` must come back with a line from a 2-rank job (host-only stub step
+    over gloo: rank r sleeps r + 1 ms per step, so the reported time is the slower rank's)."""
+    import os
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, BENCH, "--gpus", "2", "--steps", "5", "--warmup", "0", "--stub-step"],
+                       capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(ln) for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                                            # rank 0 alone prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["steps"] == 5 and lines[0]["ms_per_step"] >= 2.0
+
+
+def test_reference_arm_says_that_its_value_is_extrapolated(monkeypatch, capsys):
+    class _Sample:
+        def __init__(self, w):
+            pass
+
+        def run(self):
+            return 7000.0, 16, "stub sample"
+    monkeypatch.setattr(bench, "OracleSample", _Sample)
+    monkeypatch.delenv("RANK", raising=False)
+    import argparse
+    bench.run_reference(argparse.Namespace(config=2, warmup=1, steps=3, gpus=1))
+    line = json.loads(capsys.readouterr().out.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["extrapolated"] is True and line["timed_passes"] == 3
+    assert line["timed_s"] < 1.0 and line["value"] == 7000.0 and line["steps"] == 3
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0

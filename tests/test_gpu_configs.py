@@ -1,9 +1,16 @@
 """GPU parity on the five benchmark configurations at their full sizes, through the C ABI, in the launch
-configuration the benchmark uses.  Index sets are compared in full (band rule for score-based sets); attention
-outputs are compared on sampled (layer, head) pairs that the oracle computes one by one, with the oracle given
-the index sets the GPU chose (after those have been validated), so that a legitimate in-band difference of a
-set does not masquerade as an attention error."""
+configuration the benchmark uses.  Index sets are compared in full: the query sets exactly, the sink set of every
+step and the block set of EVERY KV group of EVERY sparse layer / step / sweep point against the oracle's scores
+with the near-threshold band rule.  Attention outputs are compared on sampled (layer, head) pairs that the oracle
+computes one by one, with the oracle given the index sets the GPU chose (after those have been validated), so that
+a legitimate in-band difference of a set does not masquerade as an attention error.
+
+How many candidates sat inside the band of each check is collected in BAND_LOG and, when the environment variable
+FOCUS_BAND_REPORT names a file, written there as JSON at the end of the module (the band-occupancy table of the
+results document comes from it)."""
+import json
 import math
+import os
 
 import numpy as np
 import pytest
@@ -22,12 +29,24 @@ TOL_RMS = {"f32": 1e-5, "bf16": 1e-2}
 BAND = 1e-3
 
 
+BAND_LOG = []      # (case, stage, layer/step, group, candidates in band, set size, candidates)
+
+
+def log_band(case, stage, where, group, band, k, n_cand):
+    BAND_LOG.append({"case": case, "stage": stage, "where": where, "group": group, "in_band": int(band),
+                     "set_size": int(k), "candidates": int(n_cand)})
+
+
 @pytest.fixture(scope="module")
 def ctx():
     c = fb.Context(0, workspace_bytes=512 << 20)
     yield c
     assert c.poll_status() == 0
     c.close()
+    path = os.environ.get("FOCUS_BAND_REPORT")
+    if path:
+        with open(path, "w") as f:
+            json.dump(BAND_LOG, f)
 
 
 def f64(a, dtype, sl=slice(None)):
@@ -45,8 +64,26 @@ def oracle_sinks_by_head(Qa_store, K_store, dtype, scale):
     return acc / Hkv
 
 
+def check_block_sets(w, t, b_blocks, b_keep, sinks, focus, case, where):
+    """Block set and sink-keep flags of EVERY KV group of one sparse layer against the oracle (Eq. 7, Top-C, Eq. 8):
+    the oracle scores one group at a time (one mean-pool of that group's prompt keys)."""
+    s = w.shape
+    hpg = s.H // s.Hkv
+    for g in range(s.Hkv):
+        K = f64(t["K"], s.dtype, slice(g, g + 1))
+        Qf = f64(t["Q"][focus - s.M][:, g * hpg:(g + 1) * hpg], s.dtype)
+        R = fo.score_blocks(Qf, fo.pool_keys(K, s.M, s.B), fo.PER_KV_GROUP)
+        ora_blocks, _ = fo.select_blocks(R, w.C, sinks, s.B)
+        band = check_topk_band(b_blocks[g], ora_blocks[0], R[0], range(s.nb), BAND, scale_ref=np.abs(R[0]).max(),
+                               what=f"{case} {where}: blocks of group {g}")
+        log_band(case, "blocks", where, g, band, w.C, s.nb)
+        mine = {int(x) for x in b_blocks[g] if x >= 0}
+        assert b_keep[g].tolist() == [0 if (int(j) // s.B) in mine else 1 for j in sinks], f"{case} {where}: keep flags {g}"
+
+
 def check_layer(w, t, b_blocks, b_keep, sinks, focus, active, O_gpu, lse_gpu, heads, rows_pos, dense=False):
-    """Block sets (band rule, sampled groups) and attention outputs (sampled heads) of one layer."""
+    """Attention outputs of sampled heads of one layer; the oracle attends over the key set the GPU chose (its block
+    sets are validated for every group by check_block_sets)."""
     s = w.shape
     hpg = s.H // s.Hkv
     scale = 1.0 / math.sqrt(s.d)
@@ -58,13 +95,7 @@ def check_layer(w, t, b_blocks, b_keep, sinks, focus, active, O_gpu, lse_gpu, he
         if dense:
             O, lse = fo.dense_attn(Q[rows_pos - s.M][:, [h - g * hpg]], K, V, scale)
         else:
-            R = fo.score_blocks(Q[focus - s.M], fo.pool_keys(K, s.M, s.B), fo.PER_KV_GROUP)
-            ora_blocks, _ = fo.select_blocks(R, w.C, sinks, s.B)
-            band = check_topk_band(b_blocks[g], ora_blocks[0], R[0], range(s.nb), BAND, scale_ref=np.abs(R[0]).max(),
-                                   what=f"blocks head {h}")
             blocks_g = np.array([x for x in b_blocks[g] if x >= 0])
-            exp_keep = [0 if (int(j) // s.B) in set(blocks_g.tolist()) else 1 for j in sinks]
-            assert b_keep[g].tolist() == exp_keep
             O, lse = fo.sparse_attn(Q[rows_pos - s.M][:, [h - g * hpg]], K, V, s.M, s.B, [blocks_g], sinks, scale)
         got = O_gpu[:len(rows_pos), h]
         assert max_abs(got, O[:, 0]) <= TOL_ABS[s.dtype], f"head {h}"
@@ -101,6 +132,8 @@ def single_layer_case(ctx, w, rows, heads, head_reduce=fb.HEADS_PER_KV_GROUP, si
     S = oracle_sinks_by_head(t["Q"][active - s.M], t["K"], s.dtype, scale)
     sinks = fo.find_sinks(S, w.n_sink, 0, s.M)
     band = check_topk_band(ba.sink_idx.cpu().numpy(), sinks, S, range(s.M), BAND, what="sinks")
+    case = f"{w.name}/{rows}" + ("" if variant == "fix" else f"/{variant}")
+    log_band(case, "sinks", "layer 0", -1, band, w.n_sink, s.M)
     S_gpu = fstep.from_device(ba.sink_scores)
     assert np.max(np.abs(S_gpu - S) / S) < 2e-3
     planted = set(t["sink_pos"].tolist())
@@ -120,6 +153,7 @@ def single_layer_case(ctx, w, rows, heads, head_reduce=fb.HEADS_PER_KV_GROUP, si
     bi = b.block_idx.cpu().numpy().reshape(G, b.max_blocks)
     keep = b.sink_keep.cpu().numpy().reshape(G, -1)[:, :w.n_sink]
     if head_reduce == fb.HEADS_PER_KV_GROUP and sink_mode == fb.SINK_TOKENS:
+        check_block_sets(w, t, bi, keep, sinks_gpu, focus, case, "layer 0")
         check_layer(w, t, bi, keep, sinks_gpu, focus, active, fstep.from_device(b.O), fstep.from_device(b.lse), heads,
                     rows_pos)
     else:
@@ -188,12 +222,17 @@ def test_config2_full_32_layer_step(ctx):
                 fstep.find_sinks(ctx, b, dQ, dK, b.lse)
                 S = oracle_sinks_by_head(t["Q"][active - s.M], t["K"], s.dtype, scale)
                 sinks = fo.find_sinks(S, w.n_sink, 0, s.M)
-                check_topk_band(b.sink_idx.cpu().numpy(), sinks, S, range(s.M), BAND, what="sinks")
+                band = check_topk_band(b.sink_idx.cpu().numpy(), sinks, S, range(s.M), BAND, what="sinks")
+                log_band(w.name, "sinks", f"layer {l}", -1, band, w.n_sink, s.M)
                 sinks_gpu = b.sink_idx.cpu().numpy()
                 assert set(t["sink_pos"].tolist()) <= set(sinks_gpu.tolist())
         else:
             fb.focus_pool_keys(ctx, b.shape, dK, Kbar)
             fstep.sparse_layer(ctx, b, dQ, dK, dV, Kbar=Kbar)
+            torch.cuda.synchronize()
+            bi = b.block_idx.cpu().numpy().reshape(b.G, b.max_blocks)
+            keep = b.sink_keep.cpu().numpy().reshape(b.G, -1)[:, :w.n_sink]
+            check_block_sets(w, t, bi, keep, sinks_gpu, focus, w.name, f"layer {l}")     # all 32 groups of every sparse layer
         if l in check_layers:
             torch.cuda.synchronize()
             bi = b.block_idx.cpu().numpy().reshape(b.G, b.max_blocks)
@@ -235,12 +274,14 @@ def test_config3_gqa_16_steps(ctx):
         fstep.find_sinks(ctx, b, dQ, dK, b.lse)
         fstep.sparse_layer(ctx, b, dQ, dK, dV, Kbar=Kbar)
         torch.cuda.synchronize()
+        S = oracle_sinks_by_head(t["Q"][active - s.M], t["K"], s.dtype, scale)
+        sinks = fo.find_sinks(S, w.n_sink, 0, s.M)
+        band = check_topk_band(b.sink_idx.cpu().numpy(), sinks, S, range(s.M), BAND, what=f"sinks step {step}")
+        log_band(w.name, "sinks", f"step {step}", -1, band, w.n_sink, s.M)
+        bi = b.block_idx.cpu().numpy().reshape(b.G, b.max_blocks)
+        keep = b.sink_keep.cpu().numpy().reshape(b.G, -1)[:, :w.n_sink]
+        check_block_sets(w, t, bi, keep, b.sink_idx.cpu().numpy(), focus, w.name, f"step {step}")
         if step in (0, 7, 15):
-            S = oracle_sinks_by_head(t["Q"][active - s.M], t["K"], s.dtype, scale)
-            sinks = fo.find_sinks(S, w.n_sink, 0, s.M)
-            check_topk_band(b.sink_idx.cpu().numpy(), sinks, S, range(s.M), BAND, what=f"sinks step {step}")
-            bi = b.block_idx.cpu().numpy().reshape(b.G, b.max_blocks)
-            keep = b.sink_keep.cpu().numpy().reshape(b.G, -1)[:, :w.n_sink]
             check_layer(w, t, bi, keep, b.sink_idx.cpu().numpy(), focus, active, fstep.from_device(b.O),
                         fstep.from_device(b.lse), [0, 6, 13, 27], active)
         # harness-side stand-in for the transfer scheduler: unmask the 2 most confident masked positions
@@ -275,3 +316,51 @@ def test_paper_hyperparameters_one_layer(ctx, rows):
     Top-C path), 252 kept, paired two per 128-key tile by the attention kernel."""
     w = wl.config(5)
     single_layer_case(ctx, w, rows, heads=[0, 22], check_dense=False)
+
+
+# ---- the generator exactly as the benchmark text states it (sink keys x8, queries NOT shifted) ---------------------
+@pytest.mark.parametrize("rows", ["active", "gen"])
+def test_config0_with_the_literal_generator(ctx, rows):
+    """Config 0 with unshifted queries: the planted sinks then carry only a fraction of a percent more attention mass
+    than an ordinary key and sit inside the near-threshold band, so their recovery is not asserted; every index set
+    still obeys the band rule and the outputs the 1e-5 bound."""
+    w = wl.config(0)
+    single_layer_case(ctx, w, rows, heads=list(range(w.shape.H)), variant="lit")
+
+
+# ---- sink selection at the full config-2 shape with scores spread over decades: the band is empty ------------------
+def test_sink_set_is_exactly_the_oracles_when_nothing_sits_near_the_threshold(ctx):
+    """Config-2 shape (32 heads, 32K keys, the I_active rows) with keys whose logit against every query carries a
+    common per-key offset a_j ~ N(0, 3): the attention mass S_j is roughly log-normal, spreads over two decades in
+    the top percent alone, and for this seed no other candidate lies within 1e-3 of the 322nd largest score (the
+    nearest are 3e-3 above and 1e-2 below).  The band rule then has nothing to forgive: the GPU's sink set must be
+    the oracle's, index for index."""
+    w = wl.config(2)
+    s = w.shape
+    rng = np.random.default_rng(78)
+    c_prev, _ = wl.gen_confidence(w.seed, s.N)
+    conf, masked = wl.full_conf(s, c_prev), wl.gen_masked(w)
+    u = rng.standard_normal(s.d).astype(np.float32)
+    u /= np.linalg.norm(u)
+    a = (rng.standard_normal(s.L) * 3.0).astype(np.float32)
+    Qs = wl.to_storage(rng.standard_normal((s.N, s.H, s.d), dtype=np.float32) + 3.0 * u, s.dtype)
+    Ks = wl.to_storage(rng.standard_normal((s.Hkv, s.L, s.d), dtype=np.float32) +
+                       (a[:, None] * u[None, :] * (math.sqrt(s.d) / 3.0))[None], s.dtype)
+    dQ, dK = fstep.to_device(Qs, s.dtype), fstep.to_device(Ks, s.dtype)
+    b = fstep.StepBuffers(w, rows="active")
+    focus, active = run_selection(ctx, w, b, conf, masked)
+    fstep.find_sinks(ctx, b, dQ, dK, None)               # no dense pass here: the library computes the LSE itself
+    torch.cuda.synchronize()
+    S = oracle_sinks_by_head(Qs[active - s.M], Ks, s.dtype, 1.0 / math.sqrt(s.d))
+    sinks = fo.find_sinks(S, w.n_sink, 0, s.M)
+    got = b.sink_idx.cpu().numpy()
+    band = check_topk_band(got, sinks, S, range(s.M), BAND, what="spread sinks")
+    log_band("c2 shape, log-normal attention mass", "sinks", "one layer", -1, band, w.n_sink, s.M)
+    top = np.sort(S[:s.M])[::-1]
+    assert top[0] / top[w.n_sink] > 50.0                  # the scores do spread
+    assert band == 1                                      # the threshold element itself and nothing else
+    assert got.tolist() == sinks.tolist()
+    S_gpu = fstep.from_device(b.sink_scores)
+    big = S[:s.M] >= top[w.n_sink] * 0.1                  # relative error where the mass is
+    assert np.max(np.abs(S_gpu[:s.M][big] - S[:s.M][big]) / S[:s.M][big]) < 2e-3
+    assert ctx.poll_status() == 0
