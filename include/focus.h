@@ -286,6 +286,35 @@ focus_status focus_update_kv(focus_ctx* ctx, const focus_shape* shape, void* K_c
                              const void* K_new, const void* V_new, const int32_t* rows, const int32_t* n_rows,
                              int32_t max_rows, focus_stream stream);
 
+/* Incremental maintenance of the pooled keys after focus_update_kv (Eq. 3 applied to prompt rows, e.g. at a
+ * block-entry refresh; K-bar_b of "Block-wise token pruning"): K-bar[g, b, :] is recomputed for exactly the prompt
+ * blocks b that hold one of the listed positions, from the (already refreshed) K cache, with the arithmetic of
+ * focus_pool_keys -- the result equals a full focus_pool_keys of the refreshed cache bit for bit.  Listed positions in
+ * the response region change no pooled key.  rows int32[max_rows] ascending (device), n_rows int32[1] (device).
+ * Negative positions are skipped and reported through the status word. */
+focus_status focus_update_pooled_keys(focus_ctx* ctx, const focus_shape* shape, const void* K, float* Kbar,
+                                      const int32_t* rows, const int32_t* n_rows, int32_t max_rows,
+                                      focus_stream stream);
+
+/* The state update that ends a denoising step (Algorithm 1, last line of the step loop; the unmasking rule stated
+ * after Eq. 2), on the device, so that a multi-step loop needs no host-side mask handling.
+ *   conf_new, token_new  float / int32 [max_rows] as written by focus_confidence for the rows evaluated this step;
+ *                        the row list (rows, n_rows, max_rows; or NULL, NULL: positions pos_base .. pos_base+max_rows-1)
+ *                        is the one given to focus_confidence and must be ascending
+ *   conf    float[L]   c^(t) -> c^(t+1): conf[pos] = conf_new[r] for every evaluated position (others keep their value)
+ *   masked  uint8[L], x int32[L] (token ids): among the evaluated positions that are still masked and lie in the
+ *           decoding block [blk_lo, blk_hi), the n_unmask with the highest new confidence (ties: lower position; NaN
+ *           last; fewer if there are fewer candidates) get x[pos] = token_new[r] and masked[pos] = 0; every other
+ *           position stays as it is (the rest remains masked)
+ *   unmasked_idx int32[n_unmask] receives those positions ascending, padded with -1 (may be NULL when n_unmask == 0);
+ *           n_unmasked int32[1] their count (may be NULL)
+ * Requires max_rows <= 4096 and n_unmask <= 4096.  One launch.  Positions outside [0, L) are skipped and reported
+ * through the status word. */
+focus_status focus_commit_step(focus_ctx* ctx, const float* conf_new, const int32_t* token_new, int32_t pos_base,
+                               const int32_t* rows, const int32_t* n_rows, int32_t max_rows, int32_t L,
+                               int32_t blk_lo, int32_t blk_hi, int32_t n_unmask, float* conf, uint8_t* masked,
+                               int32_t* x, int32_t* unmasked_idx, int32_t* n_unmasked, focus_stream stream);
+
 #ifdef __cplusplus
 }
 #endif

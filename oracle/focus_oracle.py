@@ -22,6 +22,8 @@ Functions and the passages they follow
   dense_attn       "FullAttn" of Algorithm 1: plain bidirectional softmax attention.
   confidence       Section "Diffusion LLM inference", Eq. 2: predicted token and confidence of a position.
   update_kv        "Approximate KV cache in dLLMs", Eq. 3: refreshed rows replace the cached ones.
+  commit_step      Algorithm 1, the state update that ends a step, with the unmasking rule stated right after Eq. 2:
+                   the most confident masked positions receive their predicted tokens, the rest stay masked.
 
 Readings where the paper leaves a choice (parity unpinned by the paper for these):
   * Eq. 6 writes one softmax over an "aggregated query representation"; here every
@@ -250,3 +252,24 @@ def update_kv(K_cache: np.ndarray, V_cache: np.ndarray, K_new: np.ndarray, V_new
         K[:, int(pos), :] = K_new[r]
         V[:, int(pos), :] = V_new[r]
     return K, V
+
+
+# ----------------------------------------------------------------------------- end of a step (after Eq. 2; Algorithm 1)
+def commit_step(conf: np.ndarray, masked: np.ndarray, x: np.ndarray, pos: Sequence[int], conf_new: Sequence[float],
+                token_new: Sequence[int], blk_lo: int, blk_hi: int, n: int):
+    """x^(t) -> x^(t+1) and c^(t) -> c^(t+1) for the positions `pos` evaluated this step (conf_new[r], token_new[r]
+    belong to pos[r]; Eq. 2).  Every evaluated position takes its new confidence.  Among the evaluated positions
+    that are still masked and lie in the decoding block [blk_lo, blk_hi), the n with the highest new confidence
+    (ties: lower position, NaN last) are unmasked: they receive their predicted token and leave the masked set;
+    everything else stays as it was.  Returns new (conf, masked, x) and the unmasked positions, ascending."""
+    conf, masked, x = np.array(conf, copy=True), np.array(masked, copy=True), np.array(x, copy=True)
+    row_of = {int(p): r for r, p in enumerate(pos)}
+    cand = [int(p) for p in pos if masked[int(p)] != 0 and blk_lo <= int(p) < blk_hi]
+    order = _rank_desc([conf_new[row_of[p]] for p in cand], cand)
+    picks = sorted(order[:max(0, min(n, len(cand)))])
+    for p, r in row_of.items():
+        conf[p] = conf_new[r]
+    for p in picks:
+        x[p] = token_new[row_of[p]]
+        masked[p] = 0
+    return conf, masked, x, picks

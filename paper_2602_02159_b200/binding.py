@@ -60,6 +60,8 @@ _SIGS = {
                                 _P, _P]),
     "focus_confidence": (_I, [_P, _P, _I, C.c_int64, _I, _I, _I, _P, _P, _I, _P, _P, _P]),
     "focus_update_kv": (_I, [_P, _SH, _P, _P, _P, _P, _P, _P, _I, _P]),
+    "focus_update_pooled_keys": (_I, [_P, _SH, _P, _P, _P, _P, _I, _P]),
+    "focus_commit_step": (_I, [_P, _P, _P, _I, _P, _P, _I, _I, _I, _I, _I, _P, _P, _P, _P, _P, _P]),
     "focus_dense_attn": (_I, [_P, _SH, _P, _I, _I, _P, _P, _I, _P, _P, _P, _P, _P]),
 }
 
@@ -257,3 +259,15 @@ def focus_confidence(ctx, logits, dtype, row_stride, vocab, pos_base, n_pos, row
 def focus_update_kv(ctx, shape, K_cache, V_cache, K_new, V_new, rows, n_rows, max_rows, stream=None):
     _check(ctx._lib.focus_update_kv(ctx.handle, C.byref(shape), _ptr(K_cache), _ptr(V_cache), _ptr(K_new), _ptr(V_new),
                                     _ptr(rows), _ptr(n_rows), max_rows, _stream(stream)), "focus_update_kv")
+
+
+def focus_update_pooled_keys(ctx, shape, K, Kbar, rows, n_rows, max_rows, stream=None):
+    _check(ctx._lib.focus_update_pooled_keys(ctx.handle, C.byref(shape), _ptr(K), _ptr(Kbar), _ptr(rows), _ptr(n_rows),
+                                             max_rows, _stream(stream)), "focus_update_pooled_keys")
+
+
+def focus_commit_step(ctx, conf_new, token_new, pos_base, rows, n_rows, max_rows, L, blk_lo, blk_hi, n_unmask, conf,
+                      masked, x, unmasked_idx=None, n_unmasked=None, stream=None):
+    _check(ctx._lib.focus_commit_step(ctx.handle, _ptr(conf_new), _ptr(token_new), pos_base, _ptr(rows), _ptr(n_rows),
+                                      max_rows, L, blk_lo, blk_hi, n_unmask, _ptr(conf), _ptr(masked), _ptr(x),
+                                      _ptr(unmasked_idx), _ptr(n_unmasked), _stream(stream)), "focus_commit_step")

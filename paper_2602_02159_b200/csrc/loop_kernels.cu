@@ -1,10 +1,14 @@
-// The two per-step pieces that close the decoding loop around the attention path:
+// The per-step pieces that close the decoding loop around the attention path:
 //   focus_confidence  -- Eq. 2: predicted token and confidence c = max_v softmax(logits)_v of the active rows
 //                        (an HBM-bound streaming reduction over the vocabulary; its output is the conf_prev of the
 //                        next step's focus_select_queries, and with k = n, w = 0 the same call picks the tokens
 //                        to unmask);
 //   focus_update_kv   -- Eq. 3; Algorithm 1, the cache-update step of the non-block-entry branch: the refreshed
-//                        rows replace the cached K and V rows.
+//                        rows replace the cached K and V rows;
+//   focus_commit_step -- Algorithm 1, the state update at the end of a step, with the unmasking rule stated after
+//                        Eq. 2: the new confidences of the evaluated rows enter the confidence vector, the n most
+//                        confident still-masked evaluated positions of the decoding block receive their predicted
+//                        tokens and leave the masked set.
 #include "focus_common.cuh"
 
 namespace {
@@ -129,6 +133,76 @@ __global__ void update_kv_kernel(T* __restrict__ Kc, T* __restrict__ Vc, const T
   *reinterpret_cast<uint4*>(Vc + dst) = __ldg(reinterpret_cast<const uint4*>(Vn + src));
 }
 
+constexpr int CS_THREADS = 1024;
+constexpr int CS_MAX_ROWS = 4096;
+
+// One CTA.  Row r of (conf_new, token_new) belongs to position rows[r] (or pos_base + r).  Candidates for unmasking:
+// evaluated positions that are still masked and lie in [blk_lo, blk_hi); the n_unmask with the highest new confidence
+// win (ties: lower row, i.e. lower position for an ascending list; NaN last).  Every read of masked[] precedes every
+// write (one CTA, barriers in between).
+__global__ void __launch_bounds__(CS_THREADS)
+commit_step_kernel(const float* __restrict__ conf_new, const int32_t* __restrict__ token_new, int pos_base,
+                   const int32_t* __restrict__ rows, const int32_t* __restrict__ n_rows, int max_rows, int L, int blk_lo,
+                   int blk_hi, int n_unmask, float* __restrict__ conf, uint8_t* __restrict__ masked,
+                   int32_t* __restrict__ x, int32_t* __restrict__ unmasked_idx, int32_t* __restrict__ n_unmasked,
+                   int32_t* status) {
+  __shared__ uint32_t ckey[CS_MAX_ROWS];     // compacted candidates: order-preserving confidence key,
+  __shared__ int crow[CS_MAX_ROWS];          // the row they came from (ascending)
+  __shared__ uint8_t sel[CS_MAX_ROWS];
+  __shared__ int scan_s[33];
+  __shared__ int hist[258];
+  const int tid = threadIdx.x;
+  const int n = rows ? min(max(*n_rows, 0), max_rows) : max_rows;
+  int base = 0;
+  for (int r0 = 0; r0 < n; r0 += CS_THREADS) {
+    const int r = r0 + tid;
+    int is_cand = 0, pos = -1;
+    float c = 0.f;
+    if (r < n) {
+      pos = rows ? rows[r] : pos_base + r;
+      if (pos < 0 || pos >= L) {
+        set_status(status, FOCUS_ERR_INVALID_ARG);
+        pos = -1;
+      } else {
+        c = conf_new[r];
+        is_cand = (masked[pos] != 0 && pos >= blk_lo && pos < blk_hi) ? 1 : 0;
+      }
+    }
+    int tot;
+    const int pre = block_excl_scan(is_cand, scan_s, tot);
+    if (is_cand) { ckey[base + pre] = float_key(c); crow[base + pre] = r; }
+    base += tot;
+  }
+  __syncthreads();
+  const int n_cand = base;
+  const int n_take = min(max(n_unmask, 0), n_cand);
+  block_topc_mark(ckey, n_cand, n_take, sel, hist, scan_s);
+  // the new confidences enter the vector (every evaluated position, masked or not)
+  for (int r = tid; r < n; r += CS_THREADS) {
+    const int pos = rows ? rows[r] : pos_base + r;
+    if (pos >= 0 && pos < L) conf[pos] = conf_new[r];
+  }
+  // winners: token written, mask cleared, position reported (ascending)
+  int out_base = 0;
+  for (int j0 = 0; j0 < n_cand; j0 += CS_THREADS) {
+    const int j = j0 + tid;
+    const int f = (j < n_cand && sel[j]) ? 1 : 0;
+    int tot;
+    const int pre = block_excl_scan(f, scan_s, tot);
+    if (f) {
+      const int r = crow[j];
+      const int pos = rows ? rows[r] : pos_base + r;
+      x[pos] = token_new[r];
+      masked[pos] = 0;
+      if (unmasked_idx) unmasked_idx[out_base + pre] = pos;
+    }
+    out_base += tot;
+  }
+  if (unmasked_idx)
+    for (int i = out_base + tid; i < n_unmask; i += CS_THREADS) unmasked_idx[i] = -1;
+  if (tid == 0 && n_unmasked) *n_unmasked = out_base;
+}
+
 }  // namespace
 
 extern "C" focus_status focus_confidence(focus_ctx* ctx, const void* logits, int32_t dtype, int64_t row_stride,
@@ -189,6 +263,25 @@ extern "C" focus_status focus_update_kv(focus_ctx* ctx, const focus_shape* shape
                                                     (const float*)V_new, shape->kv_stride_tok, shape->kv_stride_head,
                                                     shape->L, shape->n_kv_heads, shape->head_dim, rows, n_rows, max_rows,
                                                     ctx->d_status);
+  FOCUS_CHECK_LAUNCH();
+  return FOCUS_OK;
+}
+
+extern "C" focus_status focus_commit_step(focus_ctx* ctx, const float* conf_new, const int32_t* token_new,
+                                          int32_t pos_base, const int32_t* rows, const int32_t* n_rows,
+                                          int32_t max_rows, int32_t L, int32_t blk_lo, int32_t blk_hi,
+                                          int32_t n_unmask, float* conf, uint8_t* masked, int32_t* x,
+                                          int32_t* unmasked_idx, int32_t* n_unmasked, focus_stream stream) {
+  if (!ctx || !conf_new || !token_new || !conf || !masked || !x) return FOCUS_ERR_INVALID_ARG;
+  if ((rows == nullptr) != (n_rows == nullptr)) return FOCUS_ERR_INVALID_ARG;
+  if (L <= 0 || pos_base < 0 || max_rows < 0 || max_rows > CS_MAX_ROWS || n_unmask < 0 || n_unmask > CS_MAX_ROWS)
+    return FOCUS_ERR_INVALID_ARG;
+  if (blk_lo < 0 || blk_hi < blk_lo || blk_hi > L) return FOCUS_ERR_INVALID_ARG;
+  if (!rows && pos_base + max_rows > L) return FOCUS_ERR_INVALID_ARG;
+  if (n_unmask > 0 && !unmasked_idx) return FOCUS_ERR_INVALID_ARG;
+  commit_step_kernel<<<1, CS_THREADS, 0, stream>>>(conf_new, token_new, pos_base, rows, n_rows, max_rows, L, blk_lo,
+                                                  blk_hi, n_unmask, conf, masked, x, unmasked_idx, n_unmasked,
+                                                  ctx->d_status);
   FOCUS_CHECK_LAUNCH();
   return FOCUS_OK;
 }

@@ -34,15 +34,14 @@ __global__ void qbar_kernel(const T* __restrict__ Q, int q_base, int n_q_rows_bo
 // One CTA per (block b, KV head g): 256 threads, each owning one 16-byte column chunk and striding over rows.
 // Writes Kbar (if non-NULL) and/or R[g][b] = qbar[g] . mean (if qbar non-NULL).
 template <typename T, int D>
-__global__ void __launch_bounds__(256)
-pool_score_kernel(const T* __restrict__ K, long long kv_stride_tok, long long kv_stride_head, int M, int B, int nb,
-                  float* __restrict__ Kbar, const float* __restrict__ qbar, float* __restrict__ R) {
+__device__ __forceinline__ void pool_score_block(const T* __restrict__ K, long long kv_stride_tok, long long kv_stride_head,
+                                                 int M, int B, int nb, float* __restrict__ Kbar,
+                                                 const float* __restrict__ qbar, float* __restrict__ R, int b, int g) {
   constexpr int EPC = 16 / sizeof(T);          // elements per 16-byte chunk
   constexpr int CPR = D / EPC;                 // chunks per row
   constexpr int RPI = 256 / CPR;               // rows per iteration
   __shared__ float red[RPI][D + 1];
   __shared__ float dotp[8];
-  const int b = blockIdx.x, g = blockIdx.y;
   const int lo = b * B, hi = min(lo + B, M);
   const int chunk = threadIdx.x % CPR, rsub = threadIdx.x / CPR;
   float acc[EPC];
@@ -91,6 +90,40 @@ pool_score_kernel(const T* __restrict__ K, long long kv_stride_tok, long long kv
   }
 }
 
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+pool_score_kernel(const T* __restrict__ K, long long kv_stride_tok, long long kv_stride_head, int M, int B, int nb,
+                  float* __restrict__ Kbar, const float* __restrict__ qbar, float* __restrict__ R) {
+  pool_score_block<T, D>(K, kv_stride_tok, kv_stride_head, M, B, nb, Kbar, qbar, R, blockIdx.x, blockIdx.y);
+}
+
+// Incremental maintenance of the pooled keys after a KV-cache refresh (Eq. 3): grid (max_rows, Hkv); CTA (r, g)
+// re-pools the prompt block that holds refreshed position rows[r] for KV head g, with the arithmetic of the full
+// pooling kernel (same reduction order: the result is bit-identical to pooling everything again).  Rows in the
+// response region touch no pooled key.  With an ascending list the CTA of the first listed row of a block does the
+// work and the others of that block leave; an unsorted list only costs repeated, identical work.
+template <typename T, int D>
+__global__ void __launch_bounds__(256)
+pool_rows_kernel(const T* __restrict__ K, long long kv_stride_tok, long long kv_stride_head, int M, int B, int nb,
+                 const int32_t* __restrict__ rows, const int32_t* __restrict__ n_rows, int max_rows,
+                 float* __restrict__ Kbar, int32_t* status) {
+  const int r = blockIdx.x, g = blockIdx.y;
+  const int n = min(max(*n_rows, 0), max_rows);
+  if (r >= n) return;
+  const int pos = rows[r];
+  if (pos < 0) {
+    if (threadIdx.x == 0) set_status(status, FOCUS_ERR_INVALID_ARG);
+    return;
+  }
+  if (pos >= M) return;
+  const int b = pos / B;
+  if (r > 0) {
+    const int prev = rows[r - 1];
+    if (prev >= 0 && prev < M && prev / B == b) return;
+  }
+  pool_score_block<T, D>(K, kv_stride_tok, kv_stride_head, M, B, nb, Kbar, nullptr, nullptr, b, g);
+}
+
 // Warm path: one warp per (block, group): R[g][b] = qbar[g] . Kbar[g][b].
 __global__ void score_from_kbar_kernel(const float* __restrict__ Kbar, const float* __restrict__ qbar, int nb, int d,
                                        int G, float* __restrict__ R) {
@@ -136,6 +169,32 @@ extern "C" focus_status focus_pool_keys(focus_ctx* ctx, const focus_shape* shape
   if (!shape_supported(shape)) return FOCUS_ERR_UNSUPPORTED;
   return shape->dtype == FOCUS_BF16 ? pool_score_launch<__nv_bfloat16>(shape, K, Kbar, nullptr, nullptr, stream)
                                     : pool_score_launch<float>(shape, K, Kbar, nullptr, nullptr, stream);
+}
+
+extern "C" focus_status focus_update_pooled_keys(focus_ctx* ctx, const focus_shape* shape, const void* K, float* Kbar,
+                                                 const int32_t* rows, const int32_t* n_rows, int32_t max_rows,
+                                                 focus_stream stream) {
+  if (!ctx || !shape_ok_basic(shape) || !K || !Kbar || !rows || !n_rows || !all_aligned16(K, Kbar)) return FOCUS_ERR_INVALID_ARG;
+  if (max_rows < 0) return FOCUS_ERR_INVALID_ARG;
+  if (!shape_supported(shape)) return FOCUS_ERR_UNSUPPORTED;
+  const int nb = shape_nb(shape);
+  if (max_rows == 0 || nb == 0) return FOCUS_OK;
+  dim3 grid(max_rows, shape->n_kv_heads);
+  const long long st = shape->kv_stride_tok, sh = shape->kv_stride_head;
+  const int M = shape->M, B = shape->kv_block;
+  if (shape->dtype == FOCUS_BF16) {
+    if (shape->head_dim == 128)
+      pool_rows_kernel<__nv_bfloat16, 128><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)K, st, sh, M, B, nb, rows, n_rows, max_rows, Kbar, ctx->d_status);
+    else
+      pool_rows_kernel<__nv_bfloat16, 64><<<grid, 256, 0, stream>>>((const __nv_bfloat16*)K, st, sh, M, B, nb, rows, n_rows, max_rows, Kbar, ctx->d_status);
+  } else {
+    if (shape->head_dim == 128)
+      pool_rows_kernel<float, 128><<<grid, 256, 0, stream>>>((const float*)K, st, sh, M, B, nb, rows, n_rows, max_rows, Kbar, ctx->d_status);
+    else
+      pool_rows_kernel<float, 64><<<grid, 256, 0, stream>>>((const float*)K, st, sh, M, B, nb, rows, n_rows, max_rows, Kbar, ctx->d_status);
+  }
+  FOCUS_CHECK_LAUNCH();
+  return FOCUS_OK;
 }
 
 extern "C" focus_status focus_score_blocks(focus_ctx* ctx, const focus_shape* shape, const void* Q, int32_t q_base,

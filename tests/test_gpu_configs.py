@@ -64,6 +64,13 @@ def oracle_sinks_by_head(Qa_store, K_store, dtype, scale):
     return acc / Hkv
 
 
+def check_sinks_exact_on_own_scores(sink_idx_gpu, S_gpu, n_sink, M, what):
+    """Complement of the band rule: on the float32 scores the GPU itself produced, its Top-n with the tie rule must be
+    exact -- whatever the band forgives, it forgives score rounding, never the selection."""
+    own = fo.find_sinks(np.asarray(S_gpu, dtype=np.float64), n_sink, 0, M)
+    assert [int(i) for i in sink_idx_gpu if i >= 0] == own.tolist(), f"{what}: selection differs on the GPU's own scores"
+
+
 def check_block_sets(w, t, b_blocks, b_keep, sinks, focus, case, where):
     """Block set and sink-keep flags of EVERY KV group of one sparse layer against the oracle (Eq. 7, Top-C, Eq. 8):
     the oracle scores one group at a time (one mean-pool of that group's prompt keys)."""
@@ -136,6 +143,7 @@ def single_layer_case(ctx, w, rows, heads, head_reduce=fb.HEADS_PER_KV_GROUP, si
     log_band(case, "sinks", "layer 0", -1, band, w.n_sink, s.M)
     S_gpu = fstep.from_device(ba.sink_scores)
     assert np.max(np.abs(S_gpu - S) / S) < 2e-3
+    check_sinks_exact_on_own_scores(ba.sink_idx.cpu().numpy(), S_gpu, w.n_sink, s.M, case)
     planted = set(t["sink_pos"].tolist())
     sinks_gpu = ba.sink_idx.cpu().numpy()
     if variant == "fix":
@@ -225,6 +233,7 @@ def test_config2_full_32_layer_step(ctx):
                 band = check_topk_band(b.sink_idx.cpu().numpy(), sinks, S, range(s.M), BAND, what="sinks")
                 log_band(w.name, "sinks", f"layer {l}", -1, band, w.n_sink, s.M)
                 sinks_gpu = b.sink_idx.cpu().numpy()
+                check_sinks_exact_on_own_scores(sinks_gpu, fstep.from_device(b.sink_scores), w.n_sink, s.M, w.name)
                 assert set(t["sink_pos"].tolist()) <= set(sinks_gpu.tolist())
         else:
             fb.focus_pool_keys(ctx, b.shape, dK, Kbar)
@@ -256,6 +265,10 @@ def test_config3_one_layer_with_all_gen_rows(ctx):
 
 # ---- config 3: Dream-like GQA, 16 consecutive steps with AR(1) confidences ------------------------------------
 def test_config3_gqa_16_steps(ctx):
+    """Sixteen consecutive steps with the decoding state (confidence vector, masked set, token ids) resident on the
+    device: every step ends with focus_commit_step, nothing of the state crosses to the host between steps.  The
+    oracle drives its own copy of the state from the same synthetic confidence process; focus / active sets, sink
+    and block sets, the unmasked positions and the final state are compared step by step."""
     w = wl.config(3)
     s = w.shape
     t = wl.gen_qkv(s, w.seed)
@@ -265,33 +278,45 @@ def test_config3_gqa_16_steps(ctx):
     Kbar = torch.zeros(s.Hkv, s.nb, s.d, dtype=torch.float32, device="cuda")
     fb.focus_pool_keys(ctx, b.shape, dK, Kbar)           # K/V are fixed over the steps: pooled once
     c_prev, c_cur = wl.gen_confidence(w.seed, s.N)
-    masked = wl.gen_masked(w)
+    # device-resident state and the oracle's own copy of it
+    o_conf, o_masked, o_x = wl.full_conf(s, c_prev), wl.gen_masked(w), np.zeros(s.L, dtype=np.int32)
+    d_conf, d_masked, d_x = (torch.from_numpy(a.copy()).cuda() for a in (o_conf, o_masked, o_x))
+    picked, n_picked = torch.zeros(2, dtype=torch.int32, device="cuda"), torch.zeros(1, dtype=torch.int32, device="cuda")
+    gen_pos = list(range(s.M, s.L))
     hits = total = 0
     for step in range(w.n_steps):
-        conf = wl.full_conf(s, c_prev)
-        focus, active = run_selection(ctx, w, b, conf, masked)
+        fstep.select_queries(ctx, b, d_conf, d_masked)
+        focus, active = fo.select_queries(o_conf, o_masked, w.blk_lo, w.blk_hi, w.k, w.w, s.M, s.L)
+        assert b.focus_idx.cpu().numpy()[:b.n_focus.item()].tolist() == focus.tolist()
+        assert b.active_idx.cpu().numpy()[:b.n_active.item()].tolist() == active.tolist()
         fstep.dense_layer(ctx, b, dQ, dK, dV)
         fstep.find_sinks(ctx, b, dQ, dK, b.lse)
         fstep.sparse_layer(ctx, b, dQ, dK, dV, Kbar=Kbar)
+        # the model's output for this step is synthetic: the AR(1) confidence of every gen position and a token id
+        tok = (1000 + step * s.N + np.arange(s.N)).astype(np.int32)
+        fb.focus_commit_step(ctx, torch.from_numpy(c_cur).cuda(), torch.from_numpy(tok).cuda(), s.M, None, None, s.N,
+                             s.L, s.M, s.L, 2, d_conf, d_masked, d_x, picked, n_picked)
         torch.cuda.synchronize()
         S = oracle_sinks_by_head(t["Q"][active - s.M], t["K"], s.dtype, scale)
         sinks = fo.find_sinks(S, w.n_sink, 0, s.M)
         band = check_topk_band(b.sink_idx.cpu().numpy(), sinks, S, range(s.M), BAND, what=f"sinks step {step}")
         log_band(w.name, "sinks", f"step {step}", -1, band, w.n_sink, s.M)
+        check_sinks_exact_on_own_scores(b.sink_idx.cpu().numpy(), fstep.from_device(b.sink_scores), w.n_sink, s.M,
+                                        f"{w.name} step {step}")
         bi = b.block_idx.cpu().numpy().reshape(b.G, b.max_blocks)
         keep = b.sink_keep.cpu().numpy().reshape(b.G, -1)[:, :w.n_sink]
         check_block_sets(w, t, bi, keep, b.sink_idx.cpu().numpy(), focus, w.name, f"step {step}")
         if step in (0, 7, 15):
             check_layer(w, t, bi, keep, b.sink_idx.cpu().numpy(), focus, active, fstep.from_device(b.O),
                         fstep.from_device(b.lse), [0, 6, 13, 27], active)
-        # harness-side stand-in for the transfer scheduler: unmask the 2 most confident masked positions
-        cur = wl.full_conf(s, c_cur)
-        unmasked = wl.unmask_two(masked, cur, s.M, s.L)
+        o_conf, o_masked, o_x, unmasked = fo.commit_step(o_conf, o_masked, o_x, gen_pos, c_cur, tok, s.M, s.L, 2)
+        assert n_picked.item() == 2 and picked.cpu().numpy().tolist() == unmasked
         hits += len(set(unmasked) & set(focus.tolist()))
         total += len(unmasked)
-        c_prev = c_cur
         c_cur = wl.ar1_next(w.seed, step, c_cur)
-    assert masked[s.M:].sum() == s.N - 2 * w.n_steps
+    assert np.array_equal(d_masked.cpu().numpy(), o_masked) and np.array_equal(d_x.cpu().numpy(), o_x)
+    assert np.array_equal(d_conf.cpu().numpy(), o_conf.astype(np.float32))
+    assert o_masked[s.M:].sum() == s.N - 2 * w.n_steps and (o_x[s.M:] != 0).sum() == 2 * w.n_steps
     assert hits / total > 0.5                          # indicator recall on this synthetic process (logged, loose)
     assert ctx.poll_status() == 0
 

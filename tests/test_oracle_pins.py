@@ -426,6 +426,49 @@ def test_update_kv_replaces_exactly_the_listed_rows():
     assert np.array_equal(O1, O2)
 
 
+# ------------------------------------------------------------------ commit_step (end of a step)
+def test_commit_step_hand_worked_cases():
+    n = 0
+    for conf, masked, x, pos, cn, tn, par, conf2, masked2, x2, picks in _cases("commit_cases.txt"):
+        blk_lo, blk_hi, k = map(int, par)
+        c, m, xx, p = fo.commit_step(np.array(conf, dtype=np.float32), np.array(masked, dtype=np.uint8),
+                                     np.array(x, dtype=np.int64), list(map(int, pos)), list(map(float, cn)),
+                                     list(map(int, tn)), blk_lo, blk_hi, k)
+        assert np.allclose(c, np.array(conf2, dtype=np.float32), atol=0) and m.tolist() == list(map(int, masked2))
+        assert xx.tolist() == list(map(int, x2)) and p == list(map(int, picks))
+        n += 1
+    assert n == 5
+
+
+def test_commit_step_is_the_indicator_with_k_n_and_no_window():
+    """The unmasking pick is the same top-k rule as Eq. 4 (already pinned by hand-worked cases and brute force), applied
+    to the new confidences with w = 0; inputs are left untouched; NaN ranks last."""
+    rng = np.random.default_rng(53)
+    for trial in range(20):
+        L = int(rng.integers(8, 60))
+        masked = (rng.random(L) < 0.6).astype(np.uint8)
+        conf = rng.random(L).astype(np.float32)
+        x = rng.integers(1, 100, size=L)
+        pos = sorted(rng.choice(L, size=int(rng.integers(1, L)), replace=False).tolist())
+        cn = (np.round(rng.random(len(pos)) * 6) / 6).astype(np.float32)          # ties
+        if trial % 4 == 0:
+            cn[0] = np.nan
+        tn = rng.integers(100, 200, size=len(pos))
+        lo = int(rng.integers(0, L // 2)); hi = int(rng.integers(lo, L + 1)); n = int(rng.integers(0, 6))
+        keep = (conf.copy(), masked.copy(), x.copy())
+        c2, m2, x2, picks = fo.commit_step(conf, masked, x, pos, cn, tn, lo, hi, n)
+        assert np.array_equal(conf, keep[0]) and np.array_equal(masked, keep[1]) and np.array_equal(x, keep[2])
+        full = np.full(L, -1.0, dtype=np.float32); full[pos] = cn
+        evaluated = np.zeros(L, dtype=np.uint8); evaluated[pos] = 1
+        f, _ = fo.select_queries(full, masked & evaluated, lo, hi, n, 0, 0, L)
+        assert picks == f.tolist()
+        untouched = [i for i in range(L) if i not in picks]
+        assert np.array_equal(m2[untouched], masked[untouched]) and np.array_equal(x2[untouched], x[untouched])
+        assert all(m2[p] == 0 and x2[p] == tn[pos.index(p)] for p in picks)
+        exp_c = conf.copy(); exp_c[pos] = cn
+        assert np.array_equal(c2, exp_c, equal_nan=True)
+
+
 # ------------------------------------------------------------------ generators (inputs only)
 def test_bf16_round_trip_and_rne():
     x = np.array([1.0, 1.00390625, 1.01171875, -2.5, 3.140625], dtype=np.float32)   # 1+2^-8 ties to even
