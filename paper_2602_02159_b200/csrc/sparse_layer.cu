@@ -72,6 +72,18 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
     kpre[u] = b < nb ? __ldg(reinterpret_cast<const float4*>(kb + (size_t)b * FS_HD)) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   const int my_sink = tid < n_sink ? sink_idx[tid] : -1;
+  // The gather CTAs of this launch mostly run only after the previous attention launch has left the SMs: bring the
+  // sink rows of this head into L2 now, while that launch is still streaming, so that they find them there.
+  for (int s = tid; s < n_sink; s += FS_THREADS) {
+    const int j = s == tid ? my_sink : sink_idx[s];
+    if (j >= 0 && j < L) {
+      const size_t off = (size_t)g * kv_stride_head + (size_t)j * kv_stride_tok;
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(K + off));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(K + off + 64));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(V + off));
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(V + off + 64));
+    }
+  }
   const int c = tid & 127, y = tid >> 7;
   const int pos0 = y < max_focus ? focus_idx[y] : -1;
   const int nf = min(max(*n_focus, 0), max_focus);
