@@ -389,3 +389,48 @@ def test_sink_set_is_exactly_the_oracles_when_nothing_sits_near_the_threshold(ct
     big = S[:s.M] >= top[w.n_sink] * 0.1                  # relative error where the mass is
     assert np.max(np.abs(S_gpu[:s.M][big] - S[:s.M][big]) / S[:s.M][big]) < 2e-3
     assert ctx.poll_status() == 0
+
+
+# ---- Dream-7B's layer schedule: the last four layers stay dense ---------------------------------------------------
+def test_dream_schedule_keeps_the_final_four_layers_dense(ctx):
+    """Config-3 shape, 28 layers, layer_schedule(28, probe 5, final_dense 4) (the paper keeps the last four layers of
+    Dream-7B dense): layers 0..5 dense (5 = probe), 6..23 sparse with the shared sink set, 24..27 dense again.  Per-layer
+    Q/K/V seeded by the layer index; sampled layers of every kind are checked against the oracle, block sets of every
+    group of the sampled sparse layers included."""
+    w = wl.config(3)
+    s = w.shape
+    NL, probe = 28, 5
+    sched = fstep.layer_schedule(NL, probe, final_dense=4)
+    assert sched.count("sparse") == 18 and sched[24:] == ["dense"] * 4 and sched[probe] == "probe"
+    check = {0: [0], probe: [13], 6: [0, 27], 23: [6], 24: [20], 27: [27]}
+    c_prev, _ = wl.gen_confidence(w.seed, s.N)
+    conf, masked = wl.full_conf(s, c_prev), wl.gen_masked(w)
+    b = fstep.StepBuffers(w, rows="active")
+    focus, active = run_selection(ctx, w, b, conf, masked)
+    Kbar = torch.zeros(s.Hkv, s.nb, s.d, dtype=torch.float32, device="cuda")
+    scale = 1.0 / math.sqrt(s.d)
+    sinks_gpu = None
+    for l, kind in enumerate(sched):
+        t = wl.gen_qkv(s, 100 + l)
+        dQ, dK, dV = (fstep.to_device(t[n], s.dtype) for n in "QKV")
+        if kind in ("dense", "probe"):
+            fstep.dense_layer(ctx, b, dQ, dK, dV)
+            if kind == "probe":
+                fstep.find_sinks(ctx, b, dQ, dK, b.lse)
+                S = oracle_sinks_by_head(t["Q"][active - s.M], t["K"], s.dtype, scale)
+                sinks = fo.find_sinks(S, w.n_sink, 0, s.M)
+                band = check_topk_band(b.sink_idx.cpu().numpy(), sinks, S, range(s.M), BAND, what="sinks")
+                log_band("dream schedule", "sinks", f"layer {l}", -1, band, w.n_sink, s.M)
+                sinks_gpu = b.sink_idx.cpu().numpy()
+        else:
+            fb.focus_pool_keys(ctx, b.shape, dK, Kbar)
+            fstep.sparse_layer(ctx, b, dQ, dK, dV, Kbar=Kbar)
+        if l in check:
+            torch.cuda.synchronize()
+            bi = b.block_idx.cpu().numpy().reshape(b.G, b.max_blocks)
+            keep = b.sink_keep.cpu().numpy().reshape(b.G, -1)[:, :w.n_sink]
+            if kind == "sparse":
+                check_block_sets(w, t, bi, keep, sinks_gpu, focus, "dream schedule", f"layer {l}")
+            check_layer(w, t, bi, keep, sinks_gpu, focus, active, fstep.from_device(b.O), fstep.from_device(b.lse),
+                        check[l], active, dense=kind != "sparse")
+    assert ctx.poll_status() == 0
