@@ -846,6 +846,18 @@ def run_stages(args):
         Kn = torch.randn(ba.max_active, s.Hkv, s.d, device="cuda").to(torch.bfloat16)
         u["update_kv (Eq. 3), I_active rows"] = graph_time(lambda l: fb.focus_update_kv(
             ctx, ba.shape, Ks[l], Vs[l], Kn, Kn, ba.active_idx, ba.n_active, ba.max_active))
+        # a block-entry style refresh of 64 prompt rows spread over the prompt, then the pooled keys of their blocks
+        prow = torch.arange(0, s.M, max(1, s.M // 64), dtype=torch.int32, device="cuda")[:64].contiguous()
+        pn = torch.tensor([prow.numel()], dtype=torch.int32, device="cuda")
+        u["update_pooled_keys (64 refreshed prompt rows)"] = graph_time(lambda l: fb.focus_update_pooled_keys(
+            ctx, ba.shape, Ks[l], Kb[l], prow, pn, prow.numel()))
+    # the state update that ends a step: new confidences of the I_active rows in, two positions unmasked
+    st_conf, st_masked = conf.clone(), masked.clone()
+    st_x = torch.zeros(s.L, dtype=torch.int32, device="cuda")
+    picked = torch.zeros(2, dtype=torch.int32, device="cuda"); n_picked = torch.zeros(1, dtype=torch.int32, device="cuda")
+    u["commit_step (end of a step, I_active rows, 2 unmasked)"] = graph_time(lambda l: fb.focus_commit_step(
+        ctx, cconf, ctok, s.M, ba.active_idx, ba.n_active, ba.max_active, s.L, w.blk_lo, w.blk_hi, 2, st_conf, st_masked,
+        st_x, picked, n_picked))
     for name, b in (("I_active rows", ba), ("gen rows", bg)):
         q_rows, n_rows, max_rows = b._rows()
         n_q = na if b is ba else s.N
