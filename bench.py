@@ -324,6 +324,10 @@ def run_focus(args):
     sampler = None
 
     def timed(fn, steps, warmup, with_marks=False, headline=False):
+        # every timed region starts from an idle part: what ran before (seconds of gen-row attention, say) would
+        # otherwise decide under which power state this region is measured; the back-to-back figure is `sustained`
+        sync_all()
+        time.sleep(args.cooldown_s)
         for _ in range(warmup):
             fn(None)
         sync_all()
@@ -697,6 +701,8 @@ def graph_time_us(fn, n_layers, warm=10, reps=50):
     with torch.cuda.graph(gr):
         for l in range(n_layers):
             fn(l)
+    torch.cuda.synchronize()
+    time.sleep(0.3)                                  # start from an idle part (see `timed` in run_focus)
     for _ in range(warm):
         gr.replay()
     torch.cuda.synchronize()
@@ -925,6 +931,7 @@ def main():
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle baseline leg")
     ap.add_argument("--sustain-s", type=float, default=2.0,
                     help="seconds of back-to-back graph replays for the sustained figure (0 = skip)")
+    ap.add_argument("--cooldown-s", type=float, default=0.5, help="idle time before each timed region")
     ap.add_argument("--stub-step", action="store_true", help=argparse.SUPPRESS)   # host-only step: tests of the launcher
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not (args.stages or args.sweep):

@@ -933,67 +933,21 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   extern __shared__ uint8_t smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
-  // Programmatic dependent launch, as in attn_tc_kernel: the successor may start early; this launch may itself have
-  // started before its predecessor finished.  p.pdl = 2 (predecessor unknown): only the private set-up (barriers,
-  // TMEM) runs ahead of griddepcontrol.wait.  p.pdl = 1 (predecessor = the selection kernel of the same sparse
-  // layer): the row list and the query rows do not come from that kernel, so they are read and staged ahead of the
-  // wait as well; block lists, gathered sink rows and their mask are read after it.
+  // programmatic dependent launch: let the successor start early; wait for the predecessor before touching memory
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (p.pdl) warm_params(p, &tmK, &tmV, &tmSK, &tmSV);
+  if (p.pdl) {
+    warm_params(p, &tmK, &tmV, &tmSK, &tmSV);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+  }
 
   constexpr int TMQ = KP ? TM : TMW;                             // query rows of this CTA
   constexpr int QCH = HD * 2 / 16;                               // 16-byte chunks per query row
-  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* sptr = smem_raw + (sbase - smem_u32(smem_raw));
-  const uint32_t sQ = sbase;
-  const uint32_t sSlot = sbase + Q_BYTES_W;
-  const uint32_t sBar = sSlot + NSLOT_W * SLOT_BYTES;
-  auto bar_full = [&](int s) { return sBar + 8u * s; };
-  auto bar_empty = [&](int s) { return sBar + 8u * (NSLOT_W + s); };
-  auto bar_sfull = [&](int x) { return sBar + 8u * (2 * NSLOT_W + x); };
-  auto bar_pready = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 2 + x); };    // P_x columns of keys 0..63 stored
-  auto bar_pready2 = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 7 + x); };   // ... of keys 64..127
-  auto bar_pvdone = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 4 + x); };
-  const uint32_t bar_alldone = sBar + 8u * (2 * NSLOT_W + 6);   // every MMA of this CTA has completed
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(sptr + Q_BYTES_W + NSLOT_W * SLOT_BYTES + NBAR_W * 8);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
-  int2* tlist = reinterpret_cast<int2*>(tmem_holder + 16);
-  float* ps = reinterpret_cast<float*>(sptr + Q_BYTES_W);        // split partial (cluster mode), over the K/V ring
-
-  auto arm_barriers = [&]() {                                    // warp 0, lane 0
-    for (int s = 0; s < NSLOT_W; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
-    for (int x = 0; x < 2; ++x) {
-      mbar_init(bar_sfull(x), 1); mbar_init(bar_pready(x), 128); mbar_init(bar_pready2(x), 128); mbar_init(bar_pvdone(x), 1);
-    }
-    mbar_init(bar_alldone, 1);
-    *abort_flag = 0;
-    fence_barrier_init();
-    fence_proxy_async();
-  };
-  auto alloc_tmem = [&]() {                                      // warp 1, all lanes
-    tmem_alloc(smem_u32(tmem_holder), 512);
-    tmem_relinquish();
-  };
-  auto free_tmem_early = [&]() {                                 // every thread: TMEM allocated ahead of an early exit
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    if (warp == 1) {
-      __syncwarp();
-      tmem_dealloc(*tmem_holder, 512);
-    }
-  };
-  if (p.pdl) {
-    if (warp == 0 && lane == 0) arm_barriers();
-    if (warp == 1) alloc_tmem();
-  }
-  if (p.pdl == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
-
   // one query row per softmax thread (the key-pair form has 128 rows for 256 such threads: the upper half idles);
   // the row is requested as soon as its position is known, without waiting for the row count
   const int qtid = (int)threadIdx.x - 128;
   const bool stager = qtid >= 0 && qtid < TMQ;
   const int nrows_raw = p.q_rows ? ld_ordered(p.n_rows) : p.n_q;
+  const int cnt_raw = p.dense ? 0 : ld_ordered(p.block_cnt + g * p.group_stride);
   const int my_fr = mt * TMQ + qtid;
   const int my_qr = my_fr / p.hpg, my_hh = my_fr - my_qr * p.hpg;
   const int my_pos = (stager && my_qr < p.rows_bound) ? (p.q_rows ? ld_ordered(p.q_rows + my_qr) : p.q_base + my_qr) : -1;
@@ -1009,31 +963,28 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   }
   const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
   const int total_fr = nrows * p.hpg;
-  if (mt * TMQ >= total_fr) {                                    // uniform over the CTA (and over its cluster)
-    if (p.pdl) free_tmem_early();
-    return;
-  }
-  auto store_q = [&]() {                                         // query tile X at X * 32 KB, swizzled K-major
-    if (my_fr < total_fr && !pos_ok) set_status(p.status, FOCUS_ERR_INVALID_ARG);
-    const bool live = my_fr < total_fr;                          // rows beyond the count are staged as zeros
-    const int x = qtid >> 7, rr = qtid & 127;
-#pragma unroll
-    for (int c = 0; c < QCH; ++c) {
-      const int half = c >> 3, cc = c & 7;
-      *reinterpret_cast<uint4*>(sptr + x * Q_BYTES + half * HALF_BYTES + rr * 128 + ((cc ^ (rr & 7)) << 4)) =
-          live ? qv[c] : make_uint4(0, 0, 0, 0);
-    }
-  };
-  if (p.pdl == 1) {
-    if (stager) store_q();
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-  }
-  const int cnt_raw = p.dense ? 0 : ld_ordered(p.block_cnt + g * p.group_stride);
+  if (mt * TMQ >= total_fr) return;
 
   const TileEnum te = make_enum(p, g, cnt_raw);
   const int t0 = split_lo(te.total, split, p.n_splits);
   const int t1 = split_lo(te.total, split + 1, p.n_splits);
   const int nt = t1 - t0;
+
+  const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sptr = smem_raw + (sbase - smem_u32(smem_raw));
+  const uint32_t sQ = sbase;
+  const uint32_t sSlot = sbase + Q_BYTES_W;
+  const uint32_t sBar = sSlot + NSLOT_W * SLOT_BYTES;
+  auto bar_full = [&](int s) { return sBar + 8u * s; };
+  auto bar_empty = [&](int s) { return sBar + 8u * (NSLOT_W + s); };
+  auto bar_sfull = [&](int x) { return sBar + 8u * (2 * NSLOT_W + x); };
+  auto bar_pready = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 2 + x); };    // P_x columns of keys 0..63 stored
+  auto bar_pready2 = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 7 + x); };   // ... of keys 64..127
+  auto bar_pvdone = [&](int x) { return sBar + 8u * (2 * NSLOT_W + 4 + x); };
+  const uint32_t bar_alldone = sBar + 8u * (2 * NSLOT_W + 6);   // every MMA of this CTA has completed
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(sptr + Q_BYTES_W + NSLOT_W * SLOT_BYTES + NBAR_W * 8);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  int2* tlist = reinterpret_cast<int2*>(tmem_holder + 16);
   const bool use_list = !p.dense && nt <= MAXT_W;
   auto get_tile = [&](int idx) -> TileInfo {
     if (use_list) {
@@ -1041,9 +992,9 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     }
     return tile_info(p, te, t0 + idx);
   };
+  float* ps = reinterpret_cast<float*>(sptr + Q_BYTES_W);        // split partial (cluster mode), over the K/V ring
 
   if (nt <= 0) {                                                 // empty split (cluster mode only: see the launcher)
-    if (p.pdl) free_tmem_early();
     for (int r = threadIdx.x; r < TMQ; r += NTHREADS_W) { ps[TMQ * PROW + 2 * r] = -INFINITY; ps[TMQ * PROW + 2 * r + 1] = 0.f; }
     cluster_merge<TMQ, 256>(p, g, mt, total_fr, split, sSlot, (int)threadIdx.x - 128);
     return;
@@ -1061,7 +1012,16 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   const int n_loads = 2 * nt;
   const int n_early = n_loads < NSLOT_W ? n_loads : NSLOT_W;
   if (warp == 0) {
-    if (lane == 0 && !p.pdl) arm_barriers();
+    if (lane == 0) {
+      for (int s = 0; s < NSLOT_W; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+      for (int x = 0; x < 2; ++x) {
+        mbar_init(bar_sfull(x), 1); mbar_init(bar_pready(x), 128); mbar_init(bar_pready2(x), 128); mbar_init(bar_pvdone(x), 1);
+      }
+      mbar_init(bar_alldone, 1);
+      *abort_flag = 0;
+      fence_barrier_init();
+      fence_proxy_async();
+    }
     if (use_list) {
       for (int t = lane; t < nt; t += 32) {
         const TileInfo ti = tile_info(p, te, t0 + t);
@@ -1073,8 +1033,21 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (lane < n_early) issue(lane);                             // one copy per lane
     __syncwarp();
   }
-  if (warp == 1 && !p.pdl) alloc_tmem();
-  if (stager && p.pdl != 1) store_q();
+  if (warp == 1) {
+    tmem_alloc(smem_u32(tmem_holder), 512);
+    tmem_relinquish();
+  }
+  if (stager) {                                                  // query tile X at X * 32 KB, swizzled K-major
+    if (my_fr < total_fr && !pos_ok) set_status(p.status, FOCUS_ERR_INVALID_ARG);
+    const bool live = my_fr < total_fr;                          // rows beyond the count are staged as zeros
+    const int x = qtid >> 7, rr = qtid & 127;
+#pragma unroll
+    for (int c = 0; c < QCH; ++c) {
+      const int half = c >> 3, cc = c & 7;
+      *reinterpret_cast<uint4*>(sptr + x * Q_BYTES + half * HALF_BYTES + rr * 128 + ((cc ^ (rr & 7)) << 4)) =
+          live ? qv[c] : make_uint4(0, 0, 0, 0);
+    }
+  }
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();
@@ -1674,7 +1647,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.cluster = use_cluster ? 1 : 0;
   p.pair = pair ? 1 : 0;
   // 1: called right after the selection kernel of a fused sparse layer (pre-gathered sinks); 2: predecessor unknown
-  p.pdl = ctx->no_pdl ? 0 : (pre != nullptr ? 1 : 2);
+  p.pdl = ctx->no_pdl ? 0 : ((pre != nullptr && !wg3) ? 1 : 2);
   p.counters = (n_splits > 1 && !use_cluster && !wg3 && ctx->merge_mode != 2 && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
                    ? ctx->d_counters : nullptr;
   p.q_stride_row = sh.q_stride_row; p.q_stride_head = sh.q_stride_head;

@@ -208,25 +208,6 @@ __device__ __forceinline__ void fadd2(float& d0, float& d1, float a0, float a1, 
       "add.rn.f32x2 rd, ra, rb;\n\tmov.b64 {%0, %1}, rd;\n\t}"
       : "=f"(d0), "=f"(d1) : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
 }
-// 2^x for a pair of arguments without the special-function unit, which is the narrowest pipe of the softmax loop
-// (four lanes per scheduler): x is clamped to >= -126, split as n + f by a magic-number rounding (n integer,
-// |f| <= 0.5), 2^f comes from a degree-3 polynomial (relative error 7.5e-5, far below the bf16 rounding of the
-// probabilities it feeds) and n is added to the exponent field as an integer.  Arguments up to about +120 are fine;
-// -inf gives a value below 2^-125.  Used for part of the exponentials so that both pipes stay busy.
-__device__ __forceinline__ void ex2_poly2(float& r0, float& r1, float x0, float x1) {
-  constexpr float MAGIC = 12582912.f;            // 1.5 * 2^23: adding it rounds to the nearest integer in the low mantissa bits
-  x0 = fmaxf(x0, -126.f);
-  x1 = fmaxf(x1, -126.f);
-  float t0, t1, n0, n1, f0, f1, p0, p1;
-  fadd2(t0, t1, x0, x1, MAGIC, MAGIC);
-  fadd2(n0, n1, t0, t1, -MAGIC, -MAGIC);
-  ffma2(f0, f1, n0, n1, -1.f, -1.f, x0, x1);
-  ffma2(p0, p1, f0, f1, 0.05517211f, 0.05517211f, 0.24261113f, 0.24261113f);
-  ffma2(p0, p1, p0, p1, f0, f1, 0.69326085f, 0.69326085f);
-  ffma2(p0, p1, p0, p1, f0, f1, 0.99992806f, 0.99992806f);
-  r0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
-  r1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
-}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
