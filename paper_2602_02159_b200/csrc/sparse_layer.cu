@@ -141,33 +141,57 @@ fused_select_kernel(const __nv_bfloat16* __restrict__ Q, int q_base, long long q
   } else {
     block_topc_mark(key, nb, C, sel, hist, scan_s);
   }
+  // Everything that can be computed ahead of the dependency wait is: with at most one block and one sink slot per
+  // thread (every benchmark shape) the list position of this thread's block and the flags of its sink token sit in
+  // registers, and what follows the wait is a handful of independent stores, no loop, no barrier.
+  const bool one_pass = nb <= FS_THREADS && ns_pad <= FS_THREADS;
+  int my_f = 0, my_posn = 0, base = 0;
+  uint8_t my_keep = 0, my_mk = 0;
+  if (one_pass) {
+    my_f = (tid < nb && sel[tid]) ? 1 : 0;
+    my_posn = block_excl_scan(my_f, scan_s, base);
+    if (tid < n_sink && my_sink >= 0 && my_sink < L) {
+      const int b = my_sink / B;
+      my_keep = (b < nb && !sel[b]) ? 1 : 0;
+      my_mk = (my_keep && my_sink < M) ? 1 : 0;
+    }
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   // every store comes after the wait: the previous layer's selection kernel (which may still have been storing when
   // this one started) wrote the same R, lists and flags
-  if (R)
-    for (int b = tid; b < nb; b += FS_THREADS) R[(size_t)g * nb + b] = key_to_float(key[b]);
-  for (int s = tid; s < ns_pad; s += FS_THREADS) {
-    uint8_t keep = 0, mk = 0;
-    if (s < n_sink) {
-      const int j = s == tid ? my_sink : sink_idx[s];
-      if (j >= 0 && j < L) {
-        const int b = j / B;
-        keep = (b < nb && !sel[b]) ? 1 : 0;
-        mk = (keep && j < M) ? 1 : 0;
-      }
-      if (sink_keep) sink_keep[(size_t)g * n_sink + s] = keep;
-    }
-    mask[(size_t)g * ns_pad + s] = mk;
-  }
-  int base = 0;
   int32_t* out = block_idx + (size_t)g * C;
-  for (int c0 = 0; c0 < nb; c0 += FS_THREADS) {
-    const int i = c0 + tid;
-    const int f = (i < nb && sel[i]) ? 1 : 0;
-    int tot;
-    const int pre = block_excl_scan(f, scan_s, tot);
-    if (f && base + pre < C) out[base + pre] = i;
-    base += tot;
+  if (one_pass) {
+    if (R && tid < nb) R[(size_t)g * nb + tid] = key_to_float(key[tid]);
+    if (tid < ns_pad) {
+      if (tid < n_sink && sink_keep) sink_keep[(size_t)g * n_sink + tid] = my_keep;
+      mask[(size_t)g * ns_pad + tid] = my_mk;
+    }
+    if (my_f && my_posn < C) out[my_posn] = tid;
+  } else {
+    if (R)
+      for (int b = tid; b < nb; b += FS_THREADS) R[(size_t)g * nb + b] = key_to_float(key[b]);
+    for (int s = tid; s < ns_pad; s += FS_THREADS) {
+      uint8_t keep = 0, mk = 0;
+      if (s < n_sink) {
+        const int j = s == tid ? my_sink : sink_idx[s];
+        if (j >= 0 && j < L) {
+          const int b = j / B;
+          keep = (b < nb && !sel[b]) ? 1 : 0;
+          mk = (keep && j < M) ? 1 : 0;
+        }
+        if (sink_keep) sink_keep[(size_t)g * n_sink + s] = keep;
+      }
+      mask[(size_t)g * ns_pad + s] = mk;
+    }
+    base = 0;
+    for (int c0 = 0; c0 < nb; c0 += FS_THREADS) {
+      const int i = c0 + tid;
+      const int f = (i < nb && sel[i]) ? 1 : 0;
+      int tot;
+      const int pre = block_excl_scan(f, scan_s, tot);
+      if (f && base + pre < C) out[base + pre] = i;
+      base += tot;
+    }
   }
   if (tid == 0) block_cnt[g] = min(base, C);
 }
