@@ -107,7 +107,7 @@ uint64_t focus_launch_count(void);
  * and >= 4 key tiles per CTA, where 3 does not apply); 0 = none yet. */
 int32_t focus_last_attn_variant(focus_ctx* ctx);
 
-/* Selects the attention implementation for bf16 / head_dim 128 inputs: 0 = automatic (tensor-core
+/* Selects the attention implementation for bf16 inputs (head_dim 128 or 64): 0 = automatic (tensor-core
  * kernel where supported), 1 = force the generic SIMT kernels.  Returns the previous value. */
 int32_t focus_set_force_simt(focus_ctx* ctx, int32_t force);
 

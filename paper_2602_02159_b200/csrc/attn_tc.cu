@@ -67,6 +67,7 @@ struct TcParams {
   int n_mtiles, n_splits, lse_stride;
   int cluster;                 // 1: the splits of a tile are one thread-block cluster and merge through shared memory
   int pdl;                     // 1: launched as a programmatic dependent of the selection kernel (see the wait below)
+  int hd;                      // head dim: 128, or 64 (the upper 64 columns of every operand tile are then zeros)
   int pair;                    // 1: 64-token KV blocks, two selected blocks per 128-key tile; tmK / tmV have 64-row boxes
   float scale_log2;            // softmax scale * log2(e)
   int32_t* status;
@@ -182,15 +183,18 @@ __device__ __forceinline__ TileInfo tile_info(const TcParams& p, const TileEnum&
 // 8 KB, a whole number of swizzle atoms, after rows 0..63).
 __device__ __forceinline__ void load_tile(const TcParams& p, const TileInfo& ti, const CUtensorMap* map, uint32_t dst,
                                           uint32_t bar, int g, uint64_t l2_pol) {
-  mbar_expect_tx(bar, SLOT_BYTES);
+  const bool two = p.hd > 64;                     // head dim 64: only the lower half of the slot is filled (and read)
+  mbar_expect_tx(bar, two ? SLOT_BYTES : HALF_BYTES);
   if (p.pair && ti.kind == 0) {
     tma_load_3d_hint(dst, map, bar, 0, ti.start, g, l2_pol);
     tma_load_3d_hint(dst + HALF_BYTES / 2, map, bar, 0, ti.start2, g, l2_pol);
-    tma_load_3d_hint(dst + HALF_BYTES, map, bar, 64, ti.start, g, l2_pol);
-    tma_load_3d_hint(dst + HALF_BYTES + HALF_BYTES / 2, map, bar, 64, ti.start2, g, l2_pol);
+    if (two) {
+      tma_load_3d_hint(dst + HALF_BYTES, map, bar, 64, ti.start, g, l2_pol);
+      tma_load_3d_hint(dst + HALF_BYTES + HALF_BYTES / 2, map, bar, 64, ti.start2, g, l2_pol);
+    }
   } else {
     tma_load_3d_hint(dst, map, bar, 0, ti.start, g, l2_pol);
-    tma_load_3d_hint(dst + HALF_BYTES, map, bar, 64, ti.start, g, l2_pol);
+    if (two) tma_load_3d_hint(dst + HALF_BYTES, map, bar, 64, ti.start, g, l2_pol);
   }
 }
 
@@ -228,6 +232,7 @@ __device__ __forceinline__ void merge_rows(const TcParams& p, int tile, int g, i
 #pragma unroll 2
   for (int item = threadIdx.x; item < rows * 32; item += NTHREADS) {
     const int row = item >> 5, cg = item & 31;
+    if (cg * 4 >= p.hd) continue;
     const float4* po = reinterpret_cast<const float4*>(p.part_O) + ((size_t)tile * S * TM + row) * (HD / 4) + cg;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 4
@@ -238,7 +243,7 @@ __device__ __forceinline__ void merge_rows(const TcParams& p, int tile, int g, i
     }
     const float inv = inv_s[row];
     const int fr = mt * TM + row;
-    __nv_bfloat16* orow = p.O + ((size_t)(fr / p.hpg) * p.H + (size_t)(g * p.hpg + fr % p.hpg)) * HD + cg * 4;
+    __nv_bfloat16* orow = p.O + ((size_t)(fr / p.hpg) * p.H + (size_t)(g * p.hpg + fr % p.hpg)) * p.hd + cg * 4;
     uint2 v;
     v.x = pack_bf16(acc.x * inv, acc.y * inv);
     v.y = pack_bf16(acc.z * inv, acc.w * inv);
@@ -329,7 +334,7 @@ __device__ __forceinline__ void cluster_merge_items(const TcParams& p, int g, in
     for (int s = 0; s < SMAX; ++s) wgt[s] *= inv;
     const int fr = mt * ROWS + row;
     const int qr = fr / p.hpg, hh = fr % p.hpg;
-    __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD;
+    __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * p.hd;
 #pragma unroll
     for (int k0 = 0; k0 < 4; k0 += KB) {
       float4 o[KB][SMAX];
@@ -353,7 +358,7 @@ __device__ __forceinline__ void cluster_merge_items(const TcParams& p, int g, in
         uint2 v;
         v.x = pack_bf16(acc.x, acc.y);
         v.y = pack_bf16(acc.z, acc.w);
-        *reinterpret_cast<uint2*>(orow + (c8 + 8 * (k0 + k)) * 4) = v;
+        if ((k0 + k) * 32 < p.hd) *reinterpret_cast<uint2*>(orow + (c8 + 8 * (k0 + k)) * 4) = v;
       }
     }
     if (p.lse && c8 == 0)
@@ -446,8 +451,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       const int total = (p.L + TN - 1) / TN;
       const int pt0 = split_lo(total, split, p.n_splits), pt1 = split_lo(total, split + 1, p.n_splits);
       for (int t = pt0; t < pt1 && t < pt0 + PREF_TILES; ++t) {
-        tma_prefetch_3d(&tmK, 0, t * TN, g); tma_prefetch_3d(&tmK, 64, t * TN, g);
-        tma_prefetch_3d(&tmV, 0, t * TN, g); tma_prefetch_3d(&tmV, 64, t * TN, g);
+        tma_prefetch_3d(&tmK, 0, t * TN, g); tma_prefetch_3d(&tmV, 0, t * TN, g);
+        if (p.hd > 64) { tma_prefetch_3d(&tmK, 64, t * TN, g); tma_prefetch_3d(&tmV, 64, t * TN, g); }
       }
     }
     if (warp >= 2) {
@@ -461,7 +466,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         }
         if (pos >= p.q_base && pos < p.q_base + p.n_q) {
           const __nv_bfloat16* row = p.Q + (long long)(pos - p.q_base) * p.q_stride_row + (long long)(g * p.hpg + hh) * p.q_stride_head;
-          prefetch_l2(row); prefetch_l2(row + 64);
+          prefetch_l2(row);
+          if (p.hd > 64) prefetch_l2(row + 64);
         }
       }
     }
@@ -514,7 +520,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     const uint4* src = reinterpret_cast<const uint4*>(p.Q + (long long)(my_pos - p.q_base) * p.q_stride_row +
                                                       (long long)(g * p.hpg + my_hh) * p.q_stride_head);
 #pragma unroll
-    for (int c = 0; c < QCH; ++c) qv[c] = ld_ordered(src + c);
+    for (int c = 0; c < QCH; ++c)
+      if (c * 8 < p.hd) qv[c] = ld_ordered(src + c);
   }
   const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
   const int total_fr = nrows * p.hpg;                    // stacked (row, head-of-group) rows of this KV head
@@ -673,7 +680,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     // ================================ MMA issuer ==================================================
     if (lane == 0) {
       constexpr uint32_t IDESC_QK = make_idesc(TM, TN, 0);
-      constexpr uint32_t IDESC_PV = make_idesc(TM, HD, 1);
+      const uint32_t IDESC_PV = p.hd > 64 ? make_idesc(TM, HD, 1) : make_idesc(TM, 64, 1);   // head dim 64: O is 64 columns wide
       const uint64_t qdesc = make_sdesc(sQ, 16, 1024);
       uint32_t q = 0;
       bool ok = true;
@@ -708,6 +715,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         for (int half = 0; half < 2; ++half)
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
+            if (half == 1 && p.hd <= 64) continue;                   // head dim 64: one half of the contraction
             const uint64_t off = (uint64_t)((half * HALF_BYTES + ks * 32) >> 4);
             mma_ss(tmem + b * 128, qdesc + off, kdesc + off, IDESC_QK, (half | ks) ? 1u : 0u);
           }
@@ -835,7 +843,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       if (p.n_splits == 1) {
         const float inv = l > 0.f ? 1.f / l : 0.f;
         const int qr = valid ? fr / p.hpg : 0, hh = valid ? fr % p.hpg : 0;
-        __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD;
+        __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * p.hd;
 #pragma unroll
         for (int cb = 0; cb < 4; ++cb) {
           uint32_t oreg[32];
@@ -849,7 +857,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
               v.y = pack_bf16(__uint_as_float(oreg[c + 2]) * inv, __uint_as_float(oreg[c + 3]) * inv);
               v.z = pack_bf16(__uint_as_float(oreg[c + 4]) * inv, __uint_as_float(oreg[c + 5]) * inv);
               v.w = pack_bf16(__uint_as_float(oreg[c + 6]) * inv, __uint_as_float(oreg[c + 7]) * inv);
-              *reinterpret_cast<uint4*>(orow + cb * 32 + c) = v;
+              if (cb * 32 < p.hd) *reinterpret_cast<uint4*>(orow + cb * 32 + c) = v;
             }
           }
         }
@@ -959,7 +967,8 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     const uint4* src = reinterpret_cast<const uint4*>(p.Q + (long long)(my_pos - p.q_base) * p.q_stride_row +
                                                       (long long)(g * p.hpg + my_hh) * p.q_stride_head);
 #pragma unroll
-    for (int c = 0; c < QCH; ++c) qv[c] = ld_ordered(src + c);
+    for (int c = 0; c < QCH; ++c)
+      if (c * 8 < p.hd) qv[c] = ld_ordered(src + c);
   }
   const int nrows = p.q_rows ? min(max(nrows_raw, 0), p.rows_bound) : p.n_q;
   const int total_fr = nrows * p.hpg;
@@ -1076,7 +1085,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
   } else if (warp == 1) {
     if (lane == 0) {
       constexpr uint32_t IDESC_QK = make_idesc(TM, TN, 0);
-      constexpr uint32_t IDESC_PV = make_idesc(TM, HD, 1);
+      const uint32_t IDESC_PV = p.hd > 64 ? make_idesc(TM, HD, 1) : make_idesc(TM, 64, 1);   // head dim 64: O is 64 columns wide
       bool ok = true;
       auto wait_load = [&](int q) { return mbar_wait(bar_full(q % NSLOT_W), (uint32_t)(q / NSLOT_W) & 1u, abort_flag, p.status); };
       auto do_qk = [&](int x, int j) {                              // S_x = Q_x K_j^T (KP: the one query tile)
@@ -1086,6 +1095,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         for (int half = 0; half < 2; ++half)
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
+            if (half == 1 && p.hd <= 64) continue;                   // head dim 64: one half of the contraction
             const uint64_t off = (uint64_t)((half * HALF_BYTES + ks * 32) >> 4);
             mma_ss(tmem + x * 128, qdesc + off, kdesc + off, IDESC_QK, (half | ks) ? 1u : 0u);
           }
@@ -1297,7 +1307,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
         const float inv = p.n_splits == 1 ? (tot > 0.f ? 1.f / tot : 0.f) : 1.f;
         const float fa = wa * inv, fb = wb * inv;
         const uint32_t toa = tmem + lane_off + 256, tob = tmem + lane_off + 384;
-        __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD;
+        __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * p.hd;
         float* prow = ps + row * PROW;
 #pragma unroll
         for (int cb = 2 * x; cb < 2 * x + 2; ++cb) {                 // this warpgroup's 64 output columns
@@ -1320,7 +1330,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
                 v.y = pack_bf16(__uint_as_float(oa[c + 2]), __uint_as_float(oa[c + 3]));
                 v.z = pack_bf16(__uint_as_float(oa[c + 4]), __uint_as_float(oa[c + 5]));
                 v.w = pack_bf16(__uint_as_float(oa[c + 6]), __uint_as_float(oa[c + 7]));
-                *reinterpret_cast<uint4*>(orow + cb * 32 + c) = v;
+                if (cb * 32 < p.hd) *reinterpret_cast<uint4*>(orow + cb * 32 + c) = v;
               }
             } else {
 #pragma unroll
@@ -1345,7 +1355,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
       if (p.n_splits == 1) {
         const float inv = l > 0.f ? 1.f / l : 0.f;
         const int qr = valid ? fr / p.hpg : 0, hh = valid ? fr % p.hpg : 0;
-        __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * HD;
+        __nv_bfloat16* orow = p.O + ((size_t)qr * p.H + (size_t)(g * p.hpg + hh)) * p.hd;
 #pragma unroll
         for (int cb = 0; cb < 4; ++cb) {
           uint32_t oreg[32];
@@ -1359,7 +1369,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
               v.y = pack_bf16(__uint_as_float(oreg[c + 2]) * inv, __uint_as_float(oreg[c + 3]) * inv);
               v.z = pack_bf16(__uint_as_float(oreg[c + 4]) * inv, __uint_as_float(oreg[c + 5]) * inv);
               v.w = pack_bf16(__uint_as_float(oreg[c + 6]) * inv, __uint_as_float(oreg[c + 7]) * inv);
-              *reinterpret_cast<uint4*>(orow + cb * 32 + c) = v;
+              if (cb * 32 < p.hd) *reinterpret_cast<uint4*>(orow + cb * 32 + c) = v;
             }
           }
         }
@@ -1395,7 +1405,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
 __global__ void __launch_bounds__(256)
 attn_combine_kernel(const float* __restrict__ part_O, const float* __restrict__ part_ml, int n_splits, int n_mtiles,
                     int hpg, int H, const int32_t* q_rows, const int32_t* n_rows, int rows_bound, int n_q,
-                    __nv_bfloat16* __restrict__ O, float* __restrict__ lse, int lse_stride) {
+                    __nv_bfloat16* __restrict__ O, float* __restrict__ lse, int lse_stride, int hd) {
   const int lane = threadIdx.x & 31;
   const int wrow = blockIdx.x * 8 + (threadIdx.x >> 5);        // global stacked-row slot: tile * 128 + row
   const int tile = wrow / TM, row = wrow % TM;
@@ -1421,11 +1431,11 @@ attn_combine_kernel(const float* __restrict__ part_O, const float* __restrict__ 
   }
   const float inv = tot > 0.f ? 1.f / tot : 0.f;
   const int qr = fr / hpg, hh = fr % hpg;
-  __nv_bfloat16* orow = O + ((size_t)qr * H + (size_t)(g * hpg + hh)) * HD + lane * 4;
+  __nv_bfloat16* orow = O + ((size_t)qr * H + (size_t)(g * hpg + hh)) * hd + lane * 4;
   uint2 v;
   v.x = pack_bf16(acc.x * inv, acc.y * inv);
   v.y = pack_bf16(acc.z * inv, acc.w * inv);
-  *reinterpret_cast<uint2*>(orow) = v;
+  if (lane * 4 < hd) *reinterpret_cast<uint2*>(orow) = v;
   if (lse && lane == 0) lse[(size_t)(g * hpg + hh) * lse_stride + qr] = (m + log2f(tot)) * 0.6931471805599453f;
 }
 
@@ -1436,10 +1446,10 @@ __global__ void __launch_bounds__(256)
 sink_gather_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V, long long kv_stride_tok,
                    long long kv_stride_head, const int32_t* __restrict__ sink_idx, const uint8_t* __restrict__ sink_keep,
                    int n_sink, int ns_pad, int group_stride, int M, int L, __nv_bfloat16* __restrict__ gK,
-                   __nv_bfloat16* __restrict__ gV, uint8_t* __restrict__ mask, int32_t* status) {
+                   __nv_bfloat16* __restrict__ gV, uint8_t* __restrict__ mask, int32_t* status, int hd) {
   const int g = blockIdx.y;
   const int s = blockIdx.x * 16 + (threadIdx.x >> 4), c = threadIdx.x & 15;
-  if (s >= ns_pad) return;
+  if (s >= ns_pad || c * 8 >= hd) return;
   uint4 kv = make_uint4(0, 0, 0, 0), vv = kv;
   uint8_t mk = 0;
   if (s < n_sink) {
@@ -1453,7 +1463,7 @@ sink_gather_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __r
       mk = (j < M && sink_keep[(size_t)g * group_stride * n_sink + s]) ? 1 : 0;
     }
   }
-  const size_t o = ((size_t)g * ns_pad + s) * HD + c * 8;
+  const size_t o = ((size_t)g * ns_pad + s) * hd + c * 8;
   *reinterpret_cast<uint4*>(gK + o) = kv;
   *reinterpret_cast<uint4*>(gV + o) = vv;
   if (c == 0) mask[(size_t)g * ns_pad + s] = mk;
@@ -1512,7 +1522,7 @@ static focus_status launch_ex(K kernel, dim3 grid, int threads, int smem, int cl
 }  // namespace
 
 bool attn_tc_supported(const focus_ctx* ctx, const AttnArgs& a) {
-  return ctx->encode_tiled != nullptr && a.sh.dtype == FOCUS_BF16 && a.sh.head_dim == HD && a.O != nullptr &&
+  return ctx->encode_tiled != nullptr && a.sh.dtype == FOCUS_BF16 && (a.sh.head_dim == HD || a.sh.head_dim == 64) && a.O != nullptr &&
          (a.sh.n_q_heads / a.sh.n_kv_heads) <= TM && a.sh.L >= 1;
 }
 
@@ -1620,20 +1630,23 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   }
   if (!ws.ok) return FOCUS_ERR_WORKSPACE_TOO_SMALL;
 
+  // head dim 64: the maps' inner extent is 64, so the copy of a tile's upper 64 columns lies wholly outside the
+  // tensor and arrives as zeros -- the kernels run their 128-wide geometry on operands padded for free
+  const int hd = sh.head_dim;
   CUtensorMap tmK, tmV, tmSK, tmSV;
   const int box_rows = pair ? 64 : TN;
-  if (!encode_kv_map(ctx->encode_tiled, &tmK, a.K, HD, sh.L, Hkv, sh.kv_stride_tok, sh.kv_stride_head, 64, box_rows) ||
-      !encode_kv_map(ctx->encode_tiled, &tmV, a.V, HD, sh.L, Hkv, sh.kv_stride_tok, sh.kv_stride_head, 64, box_rows))
+  if (!encode_kv_map(ctx->encode_tiled, &tmK, a.K, hd, sh.L, Hkv, sh.kv_stride_tok, sh.kv_stride_head, 64, box_rows) ||
+      !encode_kv_map(ctx->encode_tiled, &tmV, a.V, hd, sh.L, Hkv, sh.kv_stride_tok, sh.kv_stride_head, 64, box_rows))
     return FOCUS_ERR_INVALID_ARG;
   if (ns_pad > 0) {
-    if (!encode_kv_map(ctx->encode_tiled, &tmSK, gK, HD, ns_pad, Hkv, HD, (long long)ns_pad * HD, 64, TN) ||
-        !encode_kv_map(ctx->encode_tiled, &tmSV, gV, HD, ns_pad, Hkv, HD, (long long)ns_pad * HD, 64, TN))
+    if (!encode_kv_map(ctx->encode_tiled, &tmSK, gK, hd, ns_pad, Hkv, hd, (long long)ns_pad * hd, 64, TN) ||
+        !encode_kv_map(ctx->encode_tiled, &tmSV, gV, hd, ns_pad, Hkv, hd, (long long)ns_pad * hd, 64, TN))
       return FOCUS_ERR_CUDA;
     if (!pre) {
       dim3 gg((ns_pad + 15) / 16, Hkv);
       sink_gather_kernel<<<gg, 256, 0, st>>>((const __nv_bfloat16*)a.K, (const __nv_bfloat16*)a.V, sh.kv_stride_tok,
                                              sh.kv_stride_head, a.sink_idx, a.sink_keep, a.n_sink, ns_pad,
-                                             a.group_stride, sh.M, sh.L, gK, gV, mask, ctx->d_status);
+                                             a.group_stride, sh.M, sh.L, gK, gV, mask, ctx->d_status, hd);
       FOCUS_CHECK_LAUNCH();
     }
   } else {
@@ -1646,6 +1659,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.sink_mask = mask; p.part_O = part_O; p.part_ml = part_ml;
   p.cluster = use_cluster ? 1 : 0;
   p.pair = pair ? 1 : 0;
+  p.hd = hd;
   // 1: called right after the selection kernel of a fused sparse layer (pre-gathered sinks); 2: predecessor unknown
   p.pdl = ctx->no_pdl ? 0 : ((pre != nullptr && !wg3) ? 1 : 2);
   p.counters = (n_splits > 1 && !use_cluster && !wg3 && ctx->merge_mode != 2 && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
@@ -1677,7 +1691,7 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
     const int rows_total = base * TM;
     attn_combine_kernel<<<rows_total / 8, 256, 0, st>>>(part_O, part_ml, n_splits, n_mtiles, hpg, sh.n_q_heads,
                                                         a.q_rows, a.n_rows, a.max_rows, a.n_q,
-                                                        (__nv_bfloat16*)a.O, a.lse, a.lse_stride);
+                                                        (__nv_bfloat16*)a.O, a.lse, a.lse_stride, hd);
     FOCUS_CHECK_LAUNCH();
   }
   return FOCUS_OK;

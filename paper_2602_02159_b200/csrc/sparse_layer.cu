@@ -222,7 +222,8 @@ extern "C" focus_status focus_sparse_layer(focus_ctx* ctx, const focus_shape* sh
   a.dense = 0; a.group_stride = 1; a.block_idx = block_idx; a.max_blocks = C; a.block_cnt = block_cnt;
   a.sink_idx = sink_idx; a.sink_keep = sink_keep; a.n_sink = n_sink;
 
-  const bool fused = !ctx->force_simt && attn_tc_supported(ctx, a) && nb <= FS_MAX_NB && nb > 0 && a.max_rows > 0;
+  const bool fused = !ctx->force_simt && attn_tc_supported(ctx, a) && shape->head_dim == FS_HD && nb <= FS_MAX_NB &&
+                     nb > 0 && a.max_rows > 0;
   if (!fused) {
     // generic route: the stand-alone stages, one after the other
     if (!R) return FOCUS_ERR_INVALID_ARG;

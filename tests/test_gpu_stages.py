@@ -351,6 +351,77 @@ def test_64_token_blocks_are_paired_into_key_tiles(ctx, rows, lists):
     assert ctx.poll_status() == 0
 
 
+@pytest.mark.parametrize("merge", ["cluster", "counters", "kernel"])
+@pytest.mark.parametrize("rows", [40, 128, 512])
+@pytest.mark.parametrize("keys", ["dense", "sparse_B64", "sparse_B128"])
+def test_head_dim_64_runs_on_the_tensor_core_kernels(keys, rows, merge):
+    """bf16 with head dim 64 (Dream-style heads are 128 wide, smaller models 64): the tensor-core kernels keep their
+    128-wide geometry and receive the missing upper half of every K/V tile as zeros (a copy that lies wholly outside
+    the tensor), the upper half of the query tile is staged as zeros, and only 64 output columns are written.  All
+    three kernel forms (40 / 128 / 512 stacked rows per KV head), dense and sparse key sets with both block sizes,
+    sink tiles, a ragged last block, key splits merged in all three ways, row lists, lse -- against the oracle; the
+    output buffer is twice as long as needed and its tail must stay untouched."""
+    if merge != "cluster" and rows != 40:
+        pytest.skip("only the one-tile kernel merges through global memory")
+    B = 64 if keys == "sparse_B64" else 128
+    # 512 stacked rows: GQA 4:1 with 128 rows; the dense case has enough KV heads and keys for the two-tile form
+    wide = rows == 512 and keys == "dense"
+    M = 64 * (200 if wide else 150) + 40
+    H, Hkv = ((64, 16) if wide else (8, 2)) if rows == 512 else (4, 4)
+    n = 128 if rows == 512 else rows
+    s = wl.Shape(M + n, M, H, Hkv, 64, B, "bf16")
+    rng = np.random.default_rng(5)
+    Qs, Ks, Vs = _rand_qkv(s, 61, qk_scale=1.5)
+    dQ, dK, dV = (fstep.to_device(x, s.dtype) for x in (Qs, Ks, Vs))
+    # a row list: every row but three, in order
+    q_rows = np.array([r for r in range(n) if r not in (3, 17, n - 1)], dtype=np.int32) + M
+    n_rows = len(q_rows)
+    d_rows = torch.from_numpy(np.concatenate([q_rows, np.full(3, -1, np.int32)])).cuda()
+    d_nrows = torch.tensor([n_rows], dtype=torch.int32, device="cuda")
+    O = torch.full((2 * n, s.H, s.d), 7.0, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(s.H, n, dtype=torch.float32, device="cuda")
+    c = fb.Context(0, workspace_bytes=64 << 20)
+    try:
+        if merge != "cluster":
+            c.set_option(fb.OPT_MERGE_MODE, fb.MERGE_COUNTERS if merge == "counters" else fb.MERGE_KERNEL)
+        sh = fstep.c_shape(s)
+        if keys == "dense":
+            fb.focus_dense_attn(c, sh, dQ, s.M, n, d_rows, d_nrows, n, dK, dV, O, lse)
+        else:
+            nb = s.nb
+            blocks = [np.sort(np.concatenate([rng.choice(nb - 1, size=(100 if B == 64 else 50) + g, replace=False), [nb - 1]])) for g in range(Hkv)]
+            C = max(len(b) for b in blocks) + 1
+            bidx = np.full((Hkv, C), -1, dtype=np.int32)
+            for g, b in enumerate(blocks):
+                bidx[g, :len(b)] = b
+            sinks = np.sort(rng.choice(s.M, size=70, replace=False)).astype(np.int32)
+            keep = np.array([[0 if (j // B) in set(blocks[g].tolist()) else 1 for j in sinks] for g in range(Hkv)],
+                            dtype=np.uint8)
+            fb.focus_sparse_attn(c, sh, dQ, s.M, n, d_rows, d_nrows, n, dK, dV, fb.HEADS_PER_KV_GROUP,
+                                 torch.from_numpy(bidx.reshape(-1)).cuda(), C,
+                                 torch.tensor([len(b) for b in blocks], dtype=torch.int32, device="cuda"),
+                                 torch.from_numpy(sinks).cuda(), torch.from_numpy(keep.reshape(-1)).cuda(), len(sinks),
+                                 O, lse)
+        torch.cuda.synchronize()
+        assert c.last_attn_variant() == (3 if wide else {40: 2, 128: 4, 512: 4}[rows])
+        assert c.poll_status() == 0
+    finally:
+        c.close()
+    assert bool((O[n_rows:].float() == 7.0).all()), "rows past the row count (and the spare half) stay untouched"
+    hpg = s.H // s.Hkv
+    scale = 1.0 / math.sqrt(s.d)
+    f64h = lambda a, h, kv=True: wl.storage_to_f64(a[h // hpg:h // hpg + 1] if kv else a[:, h:h + 1], s.dtype)
+    got, got_lse = fstep.from_device(O)[:n_rows], fstep.from_device(lse)[:, :n_rows]
+    for h in (0, s.H - 1):
+        Qh = f64h(Qs, h, False)[q_rows - M]
+        if keys == "dense":
+            Oh, lh = fo.dense_attn(Qh, f64h(Ks, h), f64h(Vs, h), scale)
+        else:
+            Oh, lh = fo.sparse_attn(Qh, f64h(Ks, h), f64h(Vs, h), s.M, s.B, [blocks[h // hpg]], sinks, scale)
+        assert max_abs(got[:, h], Oh[:, 0]) <= 2e-2 and rel_rms(got[:, h], Oh[:, 0]) <= 1e-2
+        assert max_abs(got_lse[h], lh[0]) <= 2e-3
+
+
 @pytest.mark.parametrize("cfg", [SHAPES[0], SHAPES[3], SHAPES[5]])
 def test_token_major_cache_and_padded_query_rows(ctx, cfg):
     """Strides are part of the shape: K/V cache stored token-major ([L, Hkv, d]: token stride Hkv*d, head stride d)
