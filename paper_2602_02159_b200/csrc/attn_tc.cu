@@ -5,7 +5,7 @@
 // are stacked, so every K/V tile is read once per group) x one contiguous range ("split") of that head's key
 // tiles.  Key tiles are 128 keys wide and are enumerated from the selected block list (one 128-token block, or two
 // 64-token blocks side by side, per tile), the gathered sink tokens and the response region; K/V tiles arrive by
-// TMA through a six-slot ring.
+// TMA through a ring of four slots, three of them in use when the key loop is short (see the launcher).
 //
 // Warp roles (192 threads):
 //   warp 0        TMA producer (one lane): K0, K1, V0, K2, V1, ... in the order the MMA warp consumes them
@@ -35,7 +35,10 @@ namespace {
 constexpr int TM = 128;            // query rows per CTA
 constexpr int TN = 128;            // keys per tile
 constexpr int HD = 128;            // head dim
-constexpr int NSLOT = 6;           // K/V ring slots
+constexpr int NSLOT = 4;           // K/V ring slots
+constexpr int EARLY = 3;           // copies requested when a CTA starts (K0, K1, V0); the others follow once K0 has landed
+constexpr int RING_SHORT = 3, RING_LONG = 4;   // ring slots in use: key loops of fewer than 12 tiles per CTA, longer ones
+static_assert(EARLY <= RING_SHORT && RING_LONG <= NSLOT, "ring");
 constexpr int SLOT_BYTES = TN * HD * 2;
 constexpr int HALF_BYTES = SLOT_BYTES / 2;     // one 64-wide half of a tile: 128 rows x 128 bytes
 constexpr int Q_BYTES = TM * HD * 2;
@@ -67,6 +70,7 @@ struct TcParams {
   int n_mtiles, n_splits, lse_stride;
   int cluster;                 // 1: the splits of a tile are one thread-block cluster and merge through shared memory
   int pdl;                     // 1: launched as a programmatic dependent of the selection kernel (see the wait below)
+  int ring;                    // one-tile kernel: K/V ring slots in use (EARLY <= ring <= NSLOT)
   int hd;                      // head dim: 128, or 64 (the upper 64 columns of every operand tile are then zeros)
   int pair;                    // 1: 64-token KV blocks, two selected blocks per 128-key tile; tmK / tmV have 64-row boxes
   float scale_log2;            // softmax scale * log2(e)
@@ -404,6 +408,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   extern __shared__ uint8_t smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.x / p.n_mtiles, mt = blockIdx.x % p.n_mtiles, split = blockIdx.y;
+  const int W = p.ring;                              // ring slots in use (EARLY <= W <= NSLOT)
 
   const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sptr = smem_raw + (sbase - smem_u32(smem_raw));
@@ -445,7 +450,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     if (warp == 1) alloc_tmem();
     // While the predecessor drains (a CTA is resident a few microseconds before the wait returns), warm L2 with what
     // the chain of dependent loads after the wait will ask for: the row count and row list, this tile's query rows
-    // and, for the dense key set (known without reading anything), the first ring-full of K/V tiles.  Values read
+    // and, for the dense key set (known without reading anything), the first K/V tiles.  Values read
     // here serve as prefetch addresses only (bounds-checked) and are read again after the wait.
     if (warp == 0 && lane == 0 && p.dense) {
       const int total = (p.L + TN - 1) / TN;
@@ -473,9 +478,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
   }
-  // Dense key set: which tiles this split streams is known without reading anything, so the first ring-full of
-  // K/V copies starts right here, ahead of the chain row count -> row list -> query rows (about 3 us sooner than
-  // from their usual place further down).  Should the tile then turn out to have no rows, the copies are awaited
+  // Dense key set: which tiles this split streams is known without reading anything, so the first K/V copies
+  // start right here, ahead of the chain row count -> row list -> query rows (about 3 us sooner than from their
+  // usual place further down).  Should the tile then turn out to have no rows, the copies are awaited
   // before the CTA leaves.
   // the two loads every thread's set-up hangs on are requested first (their values are consumed further down)
   constexpr int QCH = HD * 2 / 16;                               // 16-byte chunks per query row
@@ -489,7 +494,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     const int total = (p.L + TN - 1) / TN;
     const int pt0 = split_lo(total, split, p.n_splits), pt1 = split_lo(total, split + 1, p.n_splits);
     const int ntd = pt1 - pt0;
-    const int n_e = 2 * ntd < NSLOT ? 2 * ntd : NSLOT;
+    const int n_e = 2 * ntd < EARLY ? 2 * ntd : EARLY;
     const uint64_t pol = l2_policy_evict_first();
     if (lane < n_e) {                                // lane q issues copy q: K0, K1, V0, K2, V1, ... as in seq_tile below
       const int q = lane;
@@ -500,7 +505,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       else { isV = true; idx = (q >> 1) - 1; }
       TileInfo ti;
       ti.kind = 0; ti.start = (pt0 + idx) * TN; ti.nvalid = min(TN, p.L - ti.start); ti.start2 = ti.start + 64;
-      load_tile(p, ti, isV ? &tmV : &tmK, sSlot + (q % NSLOT) * SLOT_BYTES, bar_full(q % NSLOT), g, pol);
+      load_tile(p, ti, isV ? &tmV : &tmK, sSlot + q * SLOT_BYTES, bar_full(q), g, pol);
     }
     early_issued = n_e;
     __syncwarp();
@@ -529,7 +534,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     if (p.pdl == 2) {                                    // TMEM was allocated ahead of the row count
       if (lane == 0)
         for (int q = 0; q < early_issued; ++q)           // copies already on their way land before the CTA leaves
-          mbar_wait(bar_full(q % NSLOT), 0u, abort_flag, p.status);
+          mbar_wait(bar_full(q), 0u, abort_flag, p.status);
       tc_fence_before();
       __syncthreads();
       tc_fence_after();
@@ -611,8 +616,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   }
 
   // ---- set-up -------------------------------------------------------------------------------------
-  // Warp 0 arms the barriers, stages the tile list and puts the first ring-full of K/V tiles in flight right
-  // away: those copies need nothing from the other warps, which meanwhile allocate TMEM and stage Q.
+  // Warp 0 arms the barriers, stages the tile list and requests the first copies (K0, K1, V0) right away: they
+  // need nothing from the other warps, which meanwhile allocate TMEM and stage Q.
   // Load sequence q -> (tile, K or V), the order the MMA warp consumes: K0, K1, V0, K2, V1, ..., V(nt-1).
   auto seq_tile = [&](int q, bool& isV) -> int {
     if (q == 0) { isV = false; return 0; }
@@ -621,16 +626,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     isV = true; return (q >> 1) - 1;
   };
   const uint64_t l2_pol = l2_policy_evict_first();
-  auto issue = [&](int q) {
+  auto issue = [&](int q, int slot) {
     bool isV;
     const int idx = seq_tile(q, isV);
     const TileInfo ti = get_tile(idx);
-    const int slot = q % NSLOT;
     const CUtensorMap* map = ti.kind ? (isV ? &tmSV : &tmSK) : (isV ? &tmV : &tmK);
     load_tile(p, ti, map, sSlot + slot * SLOT_BYTES, bar_full(slot), g, l2_pol);
   };
   const int n_loads = 2 * nt;
-  const int n_early = n_loads < NSLOT ? n_loads : NSLOT;
+  const int n_early = n_loads < EARLY ? n_loads : EARLY;
   if (warp == 0) {
     if (lane == 0 && !p.pdl) arm_barriers();
     if (use_list) {
@@ -641,7 +645,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
     }
     __syncwarp();
-    if (lane >= early_issued && lane < n_early) issue(lane);       // one copy per lane
+    if (lane >= early_issued && lane < n_early) issue(lane, lane);   // one copy per lane (EARLY <= W: slot = copy index)
     __syncwarp();
   }
   if (warp == 1 && !p.pdl) alloc_tmem();
@@ -660,17 +664,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     if (lane == 0) {
       int issued = n_early;
       bool ok = true;
-      for (int q = n_early; q < n_loads; ++q) {
-        if (!mbar_wait(bar_empty(q % NSLOT), (uint32_t)((q / NSLOT) & 1) ^ 1u, abort_flag, p.status)) { ok = false; break; }
-        issue(q);
+      // All CTAs of a launch start together: with a whole ring requested at once the first key tile shares the
+      // memory system with five others per CTA and lands when they all do.  The first score tile needs K0 only,
+      // so the copies beyond the first three wait for it.
+      if (n_early < n_loads) ok = mbar_wait(bar_full(0), 0u, abort_flag, p.status);
+      int slot = n_early == W ? 0 : n_early;                 // slot and round of copy q, kept without dividing by W
+      uint32_t round = n_early == W ? 1u : 0u;
+      for (int q = n_early; q < n_loads && ok; ++q) {
+        if (!mbar_wait(bar_empty(slot), (round & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+        issue(q, slot);
         ++issued;
+        if (++slot == W) { slot = 0; ++round; }
       }
       if (!ok) {
         // unwinding: let the copies already issued land before the CTA's shared memory is released
-        const uint32_t first = issued > NSLOT ? (uint32_t)(issued - NSLOT) : 0u;
+        const uint32_t first = issued > W ? (uint32_t)(issued - W) : 0u;
         for (uint32_t i = first; i < (uint32_t)issued; ++i) {
           uint64_t t_start = global_ns();
-          while (!mbar_try_wait(bar_full(i % NSLOT), (i / NSLOT) & 1u)) {
+          while (!mbar_try_wait(bar_full(i % W), (i / W) & 1u)) {
             if (global_ns() - t_start > WAIT_LIMIT_NS) break;
           }
         }
@@ -682,13 +693,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       constexpr uint32_t IDESC_QK = make_idesc(TM, TN, 0);
       const uint32_t IDESC_PV = p.hd > 64 ? make_idesc(TM, HD, 1) : make_idesc(TM, 64, 1);   // head dim 64: O is 64 columns wide
       const uint64_t qdesc = make_sdesc(sQ, 16, 1024);
-      uint32_t q = 0;
+      int slot = 0;                                          // ring slot and round of the next tile to consume
+      uint32_t round = 0;
       bool ok = true;
       auto do_pv = [&](int idx) -> bool {
         const int b = idx & 1;
         if (!mbar_wait(bar_pready(b), (uint32_t)(idx >> 1) & 1u, abort_flag, p.status)) return false;
-        const int slot = q % NSLOT;
-        if (!mbar_wait(bar_full(slot), (q / NSLOT) & 1u, abort_flag, p.status)) return false;
+        if (!mbar_wait(bar_full(slot), round & 1u, abort_flag, p.status)) return false;
         tc_fence_after();
         const uint64_t vdesc = make_sdesc(sSlot + slot * SLOT_BYTES, HALF_BYTES, 1024);
         const uint32_t pt = tmem + b * 128;
@@ -702,13 +713,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           mma_ts(tmem_O, pt + ks * 8, vdesc + (uint64_t)(ks * (2048 >> 4)), IDESC_PV, 1u);
         tc_commit(bar_empty(slot));
         tc_commit(bar_pvdone);
-        ++q;
+        if (++slot == W) { slot = 0; ++round; }
         return true;
       };
       for (int idx = 0; idx < nt && ok; ++idx) {
         const int b = idx & 1;
-        const int slot = q % NSLOT;
-        if (!mbar_wait(bar_full(slot), (q / NSLOT) & 1u, abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(bar_full(slot), round & 1u, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         const uint64_t kdesc = make_sdesc(sSlot + slot * SLOT_BYTES, 16, 1024);
 #pragma unroll
@@ -721,7 +731,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           }
         tc_commit(bar_empty(slot));
         tc_commit(bar_sfull(b));
-        ++q;
+        if (++slot == W) { slot = 0; ++round; }
         if (idx > 0) ok = do_pv(idx - 1);
       }
       if (ok) ok = do_pv(nt - 1);
@@ -1660,6 +1670,11 @@ focus_status launch_attn_tc_ws(focus_ctx* ctx, const AttnArgs& a, WsAlloc& ws, c
   p.cluster = use_cluster ? 1 : 0;
   p.pair = pair ? 1 : 0;
   p.hd = hd;
+  // K/V ring slots the one-tile kernel keeps in flight: a short key loop is a chain of latencies and wants the tile it
+  // needs next delivered first (every copy in flight takes its share of the CTA's bandwidth); a long one wants one
+  // more slot to ride out the jitter.  Measured, I_active rows, 128 CTAs: 5-6 tiles per CTA 24.9 us with six slots,
+  // 23.2 with four, 22.9 with three; 64 tiles per CTA (dense) 87.0 / 85.7 / 87.7 us; 33 tiles 61.1 / 59.4 / 61.1.
+  p.ring = max_tiles / n_splits >= 12 ? RING_LONG : RING_SHORT;
   // 1: called right after the selection kernel of a fused sparse layer (pre-gathered sinks); 2: predecessor unknown
   p.pdl = ctx->no_pdl ? 0 : ((pre != nullptr && !wg3) ? 1 : 2);
   p.counters = (n_splits > 1 && !use_cluster && !wg3 && ctx->merge_mode != 2 && base <= FOCUS_N_COUNTERS && (size_t)(TM * n_splits + TM) * 4 <= (size_t)NSLOT * SLOT_BYTES)
