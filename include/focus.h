@@ -22,12 +22,16 @@
  *   - Stream order.  The attention kernels and the selection kernel of focus_sparse_layer are launched with
  *     programmatic stream serialization and let their successor in the stream begin early; each of them waits
  *     for its predecessor to complete before it writes anything, and before it reads anything that another of
- *     these kernels may have written (outputs, lists, workspace).  Caller-visible ordering is plain stream
- *     order: a kernel of another library placed before or after a call sees complete results, and inputs
- *     produced on the same stream before a call by any kernel that does not release its successor early -- every
- *     kernel outside this library, and every kernel of this library except the attention kernels and the selection
- *     kernel of focus_sparse_layer -- are complete when the call's kernels read them.  The one thing not to do is
- *     to feed the O or lse of one attention call straight in as the Q, q_rows or n_rows of the next attention or
+ *     these kernels may have written (outputs, lists, workspace).  A kernel of another library placed after a call
+ *     sees complete results.  Ahead of that wait these kernels read only inputs that none of them writes:
+ *     focus_sparse_layer reads Q, the focus and sink index lists, the pooled keys and the sinks' K/V rows there,
+ *     its attention kernel the row list and Q; focus_dense_attn and focus_sparse_attn read nothing ahead of it.
+ *     Such an input is complete if its producer finished before the call's predecessor in the stream started, or if
+ *     the producer is a kernel of this library (those make their outputs visible before they exit).  An input
+ *     written by a foreign kernel that runs immediately before a focus_sparse_layer call, with nothing in between
+ *     on the stream, would be read in the window between that kernel's last block exiting and its writes being
+ *     guaranteed visible: put any other kernel or an event wait in between, or set FOCUS_OPT_NO_PDL.  And do not
+ *     feed the O or lse of one attention call straight in as the Q, q_rows or n_rows of the next attention or
  *     focus_sparse_layer call with no other kernel in between: those three are read ahead of the wait.
  *   - Results are deterministic run to run (fixed reduction order, no floating-point atomics).
  *   - A device-side anomaly (index out of range, a bounded wait that ran out) never traps: the kernel

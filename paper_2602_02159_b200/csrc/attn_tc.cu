@@ -933,6 +933,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 // ================================================================================================================
 constexpr int TMW = 256;
 constexpr int NSLOT_W = 5;
+constexpr int EARLY_W = 2;                      // copies requested when a CTA starts (K0, V0); the others follow once K0 has landed
 constexpr int Q_BYTES_W = TMW * HD * 2;
 constexpr int NBAR_W = 2 * NSLOT_W + 9;
 constexpr int MAXT_W = 96;
@@ -1029,7 +1030,7 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     load_tile(p, ti, map, sSlot + slot * SLOT_BYTES, bar_full(slot), g, l2_pol);
   };
   const int n_loads = 2 * nt;
-  const int n_early = n_loads < NSLOT_W ? n_loads : NSLOT_W;
+  const int n_early = n_loads < EARLY_W ? n_loads : EARLY_W;
   if (warp == 0) {
     if (lane == 0) {
       for (int s = 0; s < NSLOT_W; ++s) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
@@ -1078,7 +1079,8 @@ attn_tc_wide_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_consta
     if (lane == 0) {
       int issued = n_early;
       bool ok = true;
-      for (int q = n_early; q < n_loads; ++q) {
+      if (n_early < n_loads) ok = mbar_wait(bar_full(0), 0u, abort_flag, p.status);   // K0 first (see the one-tile kernel)
+      for (int q = n_early; q < n_loads && ok; ++q) {
         if (!mbar_wait(bar_empty(q % NSLOT_W), (uint32_t)((q / NSLOT_W) & 1) ^ 1u, abort_flag, p.status)) { ok = false; break; }
         issue(q);
         ++issued;

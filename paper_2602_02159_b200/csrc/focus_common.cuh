@@ -85,6 +85,12 @@ static inline int shape_nb(const focus_shape* s) { return (s->M + s->kv_block - 
 #ifdef __CUDACC__
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
 
+// Last statement of a kernel whose outputs a later kernel of this library reads ahead of its dependency wait (index
+// lists, pooled keys, refreshed cache rows).  A programmatic dependent may start once every CTA of its predecessor has
+// exited, which is not yet the point where the predecessor's writes are guaranteed visible; with this fence every
+// thread's writes are visible before its CTA can exit.
+__device__ __forceinline__ void publish_outputs() { __threadfence(); }
+
 // Order-preserving map float -> uint32 (larger float => larger key).  NaN ranks below everything;
 // -0 and +0 compare equal.
 __device__ __forceinline__ uint32_t float_key(float x) {

@@ -131,6 +131,7 @@ __global__ void update_kv_kernel(T* __restrict__ Kc, T* __restrict__ Vc, const T
   const size_t dst = (size_t)g * kv_stride_head + (size_t)pos * kv_stride_tok + c * EPC;
   *reinterpret_cast<uint4*>(Kc + dst) = __ldg(reinterpret_cast<const uint4*>(Kn + src));
   *reinterpret_cast<uint4*>(Vc + dst) = __ldg(reinterpret_cast<const uint4*>(Vn + src));
+  publish_outputs();
 }
 
 constexpr int CS_THREADS = 1024;

@@ -95,6 +95,7 @@ __global__ void __launch_bounds__(256)
 pool_score_kernel(const T* __restrict__ K, long long kv_stride_tok, long long kv_stride_head, int M, int B, int nb,
                   float* __restrict__ Kbar, const float* __restrict__ qbar, float* __restrict__ R) {
   pool_score_block<T, D>(K, kv_stride_tok, kv_stride_head, M, B, nb, Kbar, qbar, R, blockIdx.x, blockIdx.y);
+  publish_outputs();
 }
 
 // Incremental maintenance of the pooled keys after a KV-cache refresh (Eq. 3): grid (max_rows, Hkv); CTA (r, g)
@@ -122,6 +123,7 @@ pool_rows_kernel(const T* __restrict__ K, long long kv_stride_tok, long long kv_
     if (prev >= 0 && prev < M && prev / B == b) return;
   }
   pool_score_block<T, D>(K, kv_stride_tok, kv_stride_head, M, B, nb, Kbar, nullptr, nullptr, b, g);
+  publish_outputs();
 }
 
 // Warm path: one warp per (block, group): R[g][b] = qbar[g] . Kbar[g][b].

@@ -99,6 +99,7 @@ select_queries_kernel(const float* __restrict__ conf, const uint8_t* __restrict_
   }
   for (int i = abase + tid; i < k * span; i += SQ_THREADS) active_idx[i] = -1;
   if (tid == 0) *n_active = abase;
+  publish_outputs();
 }
 
 extern "C" focus_status focus_select_queries(focus_ctx* ctx, const float* conf_prev, const uint8_t* masked, int32_t L,
@@ -251,10 +252,12 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
   if (*n_active <= 0) {                      // undefined scores: report and emit an empty set
     if (tid == 0) set_status(status, FOCUS_ERR_INVALID_ARG);
     for (int i = tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
+    publish_outputs();
     return;
   }
   if (want == 0) {
     for (int i = tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
+    publish_outputs();
     return;
   }
   if (tid < 40) cnt[tid] = 0;
@@ -332,6 +335,7 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
       sink_idx[rank] = mine;
     }
     for (int i = want + tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
+    publish_outputs();
     return;
   }
   // ordered compaction: warp w owns candidates [w*seg, (w+1)*seg), seg a multiple of 32
@@ -362,6 +366,7 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
     eq_seen += __popc(m_eq);
   }
   for (int i = tot_sel + tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
+  publish_outputs();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -422,6 +427,7 @@ sink_select_cluster_kernel(const float* __restrict__ S, const int32_t* n_active,
   if (n_act <= 0 || want == 0) {                        // undefined scores or nothing asked for: an empty set
     if (n_act <= 0 && tid == 0 && rank == 0) set_status(status, FOCUS_ERR_INVALID_ARG);
     for (int i = (int)rank * SC_THREADS + tid; i < n_sink; i += SC_CTAS * SC_THREADS) sink_idx[i] = -1;
+    publish_outputs();
     return;                                             // uniform over the cluster: nobody waits at a barrier
   }
   if (tid < 256) { hist[0][tid] = 0u; hist[1][tid] = 0u; }
@@ -548,6 +554,7 @@ sink_select_cluster_kernel(const float* __restrict__ S, const int32_t* n_active,
     eq_seen += __popc(m_eq);
   }
   for (int i = want + (int)rank * SC_THREADS + tid; i < n_sink; i += SC_CTAS * SC_THREADS) sink_idx[i] = -1;
+  publish_outputs();
   sc_sync();                                            // nobody leaves while its shared memory may still be read
 }
 
