@@ -519,8 +519,14 @@ def run_focus(args):
     sel_dev = torch.zeros(2 + max(1, w.k) + MA, dtype=torch.int32, device=dev)
     sel_host = torch.zeros(2 + max(1, w.k) + MA, dtype=torch.int32).pin_memory()
     sink_host = torch.zeros(bc.sink_idx.numel(), dtype=torch.int32).pin_memory()
-    n_chunks = max(1, min(4, NL // 2))
-    bounds = [round(i * NL / n_chunks) for i in range(n_chunks + 1)]
+    # chunk sizes: what precedes the first graph (indicator, read-back, gather and upload of the first chunk's rows) and
+    # what follows the last (its outputs going home) is serial, so the first and the last chunk are short
+    if NL >= 12:
+        bounds = [0] + [2 + round(i * (NL - 4) / 3) for i in range(4)] + [NL]
+    else:
+        nc = max(1, min(4, NL // 2))
+        bounds = [round(i * NL / nc) for i in range(nc + 1)]
+    n_chunks = len(bounds) - 1
     chunk_ready = [torch.cuda.Event() for _ in range(n_chunks)]
 
     def chunk_layers(c, home_prev):
@@ -556,8 +562,11 @@ def run_focus(args):
                 chunk_layers(c, True)
             chunk_graphs.append(g_)
 
+    e2e_marks = []                                       # host clock at the phase boundaries of every end-to-end step
+
     def e2e_compact_step(_m):
         main = torch.cuda.current_stream()
+        tm = [time.perf_counter()]
         conf.copy_(conf_host, non_blocking=True)
         masked.copy_(masked_host, non_blocking=True)
         fstep.select_queries(ctx, bc, conf, masked)
@@ -566,6 +575,7 @@ def run_focus(args):
         sel_dev[2 + bc.focus_idx.numel():].copy_(bc.active_idx, non_blocking=True)
         sel_host.copy_(sel_dev, non_blocking=True)
         main.synchronize()
+        tm.append(time.perf_counter())                   # indicator done, index sets on the host
         nf_, na_ = int(sel_host[0]), int(sel_host[1])
         fpos = sel_host[2:2 + nf_]
         apos = sel_host[2 + bc.focus_idx.numel():2 + bc.focus_idx.numel() + na_]
@@ -577,19 +587,32 @@ def run_focus(args):
             with torch.cuda.stream(copy_stream):
                 if c == 0:
                     copy_stream.wait_stream(main)
-                Qc[bounds[c]:bounds[c + 1], :na_].copy_(Qc_host[bounds[c]:bounds[c + 1], :na_], non_blocking=True)
+                for l in range(bounds[c], bounds[c + 1]):    # one contiguous block per layer: plain DMA from pinned memory
+                    Qc[l, :na_].copy_(Qc_host[l, :na_], non_blocking=True)
                 chunk_ready[c].record(copy_stream)
             main.wait_event(chunk_ready[c])
             if chunk_graphs is not None:
                 chunk_graphs[c].replay()
             else:
                 chunk_layers(c, True)
+            if c == 0:
+                tm.append(time.perf_counter())           # first chunk gathered, uploaded and launched
         Oc_host[bounds[-2]:].copy_(Oc[bounds[-2]:], non_blocking=True)
         sink_host.copy_(bc.sink_idx, non_blocking=True)
+        tm.append(time.perf_counter())                   # everything enqueued
         main.synchronize()
+        tm.append(time.perf_counter())
+        e2e_marks.append(tm)
 
     ms_e2e, _, _ = timed(e2e_compact_step, max(2, K // 2), 2)
     h2d_c = conf_host.numel() * 4 + masked_host.numel() + NL * na * s.H * s.d * 2 + 4 * max(1, w.k)
+    e2e_phases = None
+    if e2e_marks:
+        tail = e2e_marks[-max(2, K // 2):]               # the timed steps
+        med = lambda i: float(np.median([(t[i + 1] - t[i]) * 1e3 for t in tail]))
+        e2e_phases = {"indicator_and_readback_ms": round(med(0), 3), "first_chunk_gather_upload_launch_ms": round(med(1), 3),
+                      "remaining_enqueue_ms": round(med(2), 3), "wait_for_the_device_ms": round(med(3), 3),
+                      "note": "host clock between the phase boundaries of the timed end-to-end steps (medians)"}
     d2h_c = Oc_host.numel() * 2 + sel_host.numel() * 4 + sink_host.numel() * 4
 
     # ---- sustained leg: the same graph replayed back to back for >= 2 s of device time, clocks sampled inside --------
@@ -668,7 +691,8 @@ def run_focus(args):
                             "those rows of every layer's Q in pinned memory and uploads only them (chunks of layers, the "
                             "gather of the next chunk overlapping the GPU work of the current one); outputs of the "
                             "I_active rows of every layer and the index sets go back to pinned memory",
-                "launch_mode": f"{n_chunks} CUDA graphs of {NL // n_chunks} layers per step + eager indicator call"
+                "host_phases": e2e_phases,
+                "launch_mode": f"{n_chunks} CUDA graphs of {[bounds[i + 1] - bounds[i] for i in range(n_chunks)]} layers per step + eager indicator call"
                                if chunk_graphs is not None else "eager C-ABI calls"},
         "e2e_all_gen_rows": {"value": ms_e2e_all, "unit": "ms", "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                              "note": "all 512 gen rows of Q of every layer uploaded although only the I_active rows are read "
