@@ -42,7 +42,7 @@ static_assert(EARLY <= RING_SHORT && RING_LONG <= NSLOT, "ring");
 constexpr int SLOT_BYTES = TN * HD * 2;
 constexpr int HALF_BYTES = SLOT_BYTES / 2;     // one 64-wide half of a tile: 128 rows x 128 bytes
 constexpr int Q_BYTES = TM * HD * 2;
-constexpr int NBAR = 2 * NSLOT + 7;
+constexpr int NBAR = 2 * NSLOT + 8;
 constexpr int MAXT = 128;            // key tiles of a split whose descriptors are staged in shared memory
 constexpr int SMEM_BYTES = 1024 + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8 + 64 + MAXT * 8;
 constexpr int NTHREADS = 192;
@@ -419,7 +419,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   auto bar_empty = [&](int s) { return sBar + 8u * (NSLOT + s); };
   auto bar_sfull = [&](int b) { return sBar + 8u * (2 * NSLOT + b); };
   auto bar_pready = [&](int b) { return sBar + 8u * (2 * NSLOT + 2 + b); };
-  const uint32_t bar_pvdone = sBar + 8u * (2 * NSLOT + 4);
+  // P V of key tile idx commits to bar_pvdone(idx & 1): a softmax thread that has seen S of tile idx knows P V of
+  // tile idx - 2 (and so idx - 3) complete, i.e. it is at most one phase behind on either barrier and a parity wait
+  // cannot mistake a phase two further on for the one it asks for (with a single barrier it could: had the last
+  // product retired before a delayed thread's first test, the test read "not yet" until the wait ran out)
+  auto bar_pvdone = [&](int b) { return sBar + 8u * (b ? 2 * NSLOT + 7 : 2 * NSLOT + 4); };
   auto bar_pready2 = [&](int b) { return sBar + 8u * (2 * NSLOT + 5 + b); };   // second half (keys 64..127) of P_b stored
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(sptr + Q_BYTES + NSLOT * SLOT_BYTES + NBAR * 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
@@ -436,7 +440,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   auto arm_barriers = [&]() {                        // warp 0, lane 0
     for (int sl = 0; sl < NSLOT; ++sl) { mbar_init(bar_full(sl), 1); mbar_init(bar_empty(sl), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(bar_sfull(b), 1); mbar_init(bar_pready(b), 128); mbar_init(bar_pready2(b), 128); }
-    mbar_init(bar_pvdone, 1);
+    mbar_init(bar_pvdone(0), 1); mbar_init(bar_pvdone(1), 1);
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async();
@@ -712,7 +716,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         for (int ks = TN / 32; ks < TN / 16; ++ks)
           mma_ts(tmem_O, pt + ks * 8, vdesc + (uint64_t)(ks * (2048 >> 4)), IDESC_PV, 1u);
         tc_commit(bar_empty(slot));
-        tc_commit(bar_pvdone);
+        tc_commit(bar_pvdone(b));
         if (++slot == W) { slot = 0; ++round; }
         return true;
       };
@@ -801,9 +805,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       // p = 2^(s*scale_log2 - m_ref); a fully masked row so far (m_ref = -inf) contributes zeros
       const float mneg = m_ref == -INFINITY ? 0.f : -m_ref;
       if (idx > 0 && __any_sync(0xffffffffu, rescale)) {   // tcgen05.ld/st are warp-collective: the whole warp takes the branch
-        // P_{idx-1} V_{idx-1} must have left the tensor core before O is touched.  Phases that were not waited for
-        // cannot alias: phase idx of this barrier needs this thread's own arrival below.
-        if (!__all_sync(0xffffffffu, mbar_wait(bar_pvdone, (uint32_t)(idx - 1) & 1u, abort_flag, p.status))) { ok = false; break; }
+        // P_{idx-1} V_{idx-1} must have left the tensor core before O is touched (its barrier is at most one phase
+        // behind: see bar_pvdone).
+        if (!__all_sync(0xffffffffu, mbar_wait(bar_pvdone((idx - 1) & 1), (uint32_t)((idx - 1) >> 1) & 1u, abort_flag, p.status))) { ok = false; break; }
         tc_fence_after();
 #pragma unroll
         for (int cb = 0; cb < 4; ++cb) {
@@ -841,11 +845,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       l = l * alpha + ((acc[0] + acc[1]) + (acc[2] + acc[3]));
     }
     // ---- epilogue: wait for the last P V, normalise, write out -----------------------------------
-    // The loop waits on this barrier only before a rescale, so it may still be in phase nt-2 here (S_{nt-1} being
-    // complete says no more than that P_{nt-3} V_{nt-3} is): take the last two phases in order, or the parity of
-    // phase nt-1 would be mistaken for complete.
-    if (ok && nt >= 2) ok = __all_sync(0xffffffffu, mbar_wait(bar_pvdone, (uint32_t)(nt - 2) & 1u, abort_flag, p.status));
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_pvdone, (uint32_t)(nt - 1) & 1u, abort_flag, p.status));
+    // The loop waits for a P V product only before a rescale: S_{nt-1} being complete says no more than that
+    // P_{nt-3} V_{nt-3} is, which is the previous phase of the barrier of tile nt-1's parity.
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_pvdone((nt - 1) & 1), (uint32_t)((nt - 1) >> 1) & 1u, abort_flag, p.status));
     if (ok) {
       tc_fence_after();
       const int fr = mt * TM + row;
