@@ -650,7 +650,7 @@ def run_focus(args):
 
     # dram__bytes_read.sum + dram__bytes_write.sum of one dense-layer launch of this shape (32 heads, L = 32768,
     # I_active rows) from the ncu capture of that kernel summarised under profiles/
-    traffic = 541_858_304 if (args.config == 2 and not args.layers) else None
+    traffic = 541_483_264 if (args.config == 2 and not args.layers) else None
     out = {
         "metric": METRIC, "value": ms_step, "unit": "ms", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
