@@ -165,13 +165,22 @@ focus_status focus_select_queries(focus_ctx* ctx, const float* conf_prev, const 
  *   K          [Hkv, L, d] by strides
  *   lse        float[H * max_active] (lse[h*max_active + r], natural log, as written by focus_dense_attn
  *              for the same rows) or NULL: the library then computes it (one more pass over K)
- *   sink_idx   int32[n_sink]; scores float[L] or NULL (receives S)
+ *   sink_idx   int32[n_sink] (may be NULL when n_sink == 0: scores only); scores float[L] or NULL (receives S)
  * n_active == 0 on the device is recorded as INVALID_ARG in the status word (outputs are -1). */
 focus_status focus_find_sinks(focus_ctx* ctx, const focus_shape* shape, const void* Q, int32_t q_base,
                               const int32_t* active_idx, const int32_t* n_active, int32_t max_active,
                               const void* K, const float* lse, int32_t n_sink,
                               int32_t cand_lo, int32_t cand_hi,
                               int32_t* sink_idx, float* scores, focus_stream stream);
+
+/* The Top-N_sink step of Eq. 6 on its own: I_sink = the n_sink positions of [cand_lo, cand_hi) with the highest
+ * scores[j] (ties: lower index), ascending, padded with -1 when the range is shorter than n_sink.  For a layer whose
+ * heads live on several devices (equal head counts): each device computes S over its own heads with
+ * focus_find_sinks (n_sink = 0, sink_idx NULL, scores = its S), the S are averaged over the devices -- L floats, the
+ * only exchange of a denoising step -- and every device selects from the average with this call.
+ *   scores float[L], sink_idx int32[n_sink] (device) */
+focus_status focus_select_sinks(focus_ctx* ctx, const float* scores, int32_t L, int32_t cand_lo, int32_t cand_hi,
+                                int32_t n_sink, int32_t* sink_idx, focus_stream stream);
 
 /* ---- stage 3: block relevance (Eq. 7) and Top-C selection (Eq. 8) --------------------------- */
 

@@ -51,6 +51,7 @@ _SIGS = {
     "focus_last_attn_variant": (_I, [_P]),
     "focus_select_queries": (_I, [_P, _P, _P, _I, _I, _I, _I, _I, _I, _I, _P, _P, _P, _P, _P]),
     "focus_find_sinks": (_I, [_P, _SH, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _P, _P, _P]),
+    "focus_select_sinks": (_I, [_P, _P, _I, _I, _I, _I, _P, _P]),
     "focus_pool_keys": (_I, [_P, _SH, _P, _P, _P]),
     "focus_score_blocks": (_I, [_P, _SH, _P, _I, _P, _P, _I, _P, _P, _I, _P, _P]),
     "focus_score_blocks_static": (_I, [_SH, _P, _I, _P, _P, _I, _P, _P, _I, _P, _P, _P]),
@@ -195,6 +196,11 @@ def focus_find_sinks(ctx, shape, Q, q_base, active_idx, n_active, max_active, K,
     _check(ctx._lib.focus_find_sinks(ctx.handle, C.byref(shape), _ptr(Q), q_base, _ptr(active_idx), _ptr(n_active),
                                      max_active, _ptr(K), _ptr(lse), n_sink, cand_lo, cand_hi, _ptr(sink_idx),
                                      _ptr(scores), _stream(stream)), "focus_find_sinks")
+
+
+def focus_select_sinks(ctx, scores, L, cand_lo, cand_hi, n_sink, sink_idx, stream=None):
+    _check(ctx._lib.focus_select_sinks(ctx.handle, _ptr(scores), L, cand_lo, cand_hi, n_sink, _ptr(sink_idx),
+                                       _stream(stream)), "focus_select_sinks")
 
 
 def focus_pool_keys(ctx, shape, K, Kbar, stream=None):

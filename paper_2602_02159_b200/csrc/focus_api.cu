@@ -10,6 +10,8 @@
 
 focus_status launch_sink_select(focus_ctx* ctx, const float* part, int H, int L, const int32_t* n_active, float* S,
                                 int cand_lo, int cand_hi, int n_sink, int32_t* sink_idx, cudaStream_t st);
+focus_status launch_sink_topn(focus_ctx* ctx, const float* S, const int32_t* n_active, int cand_lo, int cand_hi,
+                              int n_sink, int32_t* sink_idx, cudaStream_t st);
 focus_status launch_sink_colsum_simt(focus_ctx* ctx, const focus_shape* s, const void* Q, int q_base,
                                      const int32_t* active_idx, const int32_t* n_active, int max_active,
                                      const void* K, const float* lse, float* part, cudaStream_t st);
@@ -187,7 +189,8 @@ extern "C" focus_status focus_find_sinks(focus_ctx* ctx, const focus_shape* shap
                                          const int32_t* active_idx, const int32_t* n_active, int32_t max_active,
                                          const void* K, const float* lse, int32_t n_sink, int32_t cand_lo,
                                          int32_t cand_hi, int32_t* sink_idx, float* scores, focus_stream stream) {
-  if (!ctx || !shape_ok_basic(shape) || !Q || !active_idx || !n_active || !K || !sink_idx) return FOCUS_ERR_INVALID_ARG;
+  if (!ctx || !shape_ok_basic(shape) || !Q || !active_idx || !n_active || !K) return FOCUS_ERR_INVALID_ARG;
+  if (n_sink > 0 && !sink_idx) return FOCUS_ERR_INVALID_ARG;      // n_sink == 0: scores only
   if (!all_aligned16(Q, K)) return FOCUS_ERR_INVALID_ARG;
   if (max_active <= 0 || n_sink < 0 || q_base < 0 || q_base > shape->L) return FOCUS_ERR_INVALID_ARG;
   if (cand_lo < 0 || cand_hi < cand_lo || cand_hi > shape->L) return FOCUS_ERR_INVALID_ARG;
@@ -224,5 +227,13 @@ extern "C" focus_status focus_find_sinks(focus_ctx* ctx, const focus_shape* shap
   else s = launch_sink_colsum_simt(ctx, shape, Q, q_base, active_idx, n_active, max_active, K, lse, part, stream);
   if (s != FOCUS_OK) return s;
   return launch_sink_select(ctx, part, H, L, n_active, S, cand_lo, cand_hi, n_sink, sink_idx, stream);
+}
+
+extern "C" focus_status focus_select_sinks(focus_ctx* ctx, const float* scores, int32_t L, int32_t cand_lo,
+                                           int32_t cand_hi, int32_t n_sink, int32_t* sink_idx, focus_stream stream) {
+  if (!ctx || !scores || L <= 0 || n_sink < 0 || (n_sink > 0 && !sink_idx)) return FOCUS_ERR_INVALID_ARG;
+  if (cand_lo < 0 || cand_hi < cand_lo || cand_hi > L) return FOCUS_ERR_INVALID_ARG;
+  if (n_sink == 0) return FOCUS_OK;
+  return launch_sink_topn(ctx, scores, nullptr, cand_lo, cand_hi, n_sink, sink_idx, (cudaStream_t)stream);
 }
 

@@ -249,7 +249,7 @@ sink_topn_kernel(const float* __restrict__ S, int lo, int hi, int n_sink, const 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int n = hi - lo;
   const int want = min(n_sink, n);
-  if (*n_active <= 0) {                      // undefined scores: report and emit an empty set
+  if (n_active && *n_active <= 0) {          // undefined scores: report and emit an empty set (NULL: scores as given)
     if (tid == 0) set_status(status, FOCUS_ERR_INVALID_ARG);
     for (int i = tid; i < n_sink; i += TN_THREADS) sink_idx[i] = -1;
     publish_outputs();
@@ -414,7 +414,7 @@ sink_select_cluster_kernel(const float* __restrict__ S, const int32_t* n_active,
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
   const int n = hi - lo;
   const int want = min(n_sink, n);
-  const int n_act = *n_active;
+  const int n_act = n_active ? *n_active : 1;           // NULL: the scores are taken as given
   const int chunk = (n + SC_CTAS - 1) / SC_CTAS;
   const int c_lo = min((int)rank * chunk, n), c_hi = min(c_lo + chunk, n), cn = c_hi - c_lo;
   uint32_t a = 0xFFFFFFFFu, o = 0u;
@@ -558,10 +558,20 @@ sink_select_cluster_kernel(const float* __restrict__ S, const int32_t* n_active,
   sc_sync();                                            // nobody leaves while its shared memory may still be read
 }
 
+focus_status launch_sink_topn(focus_ctx* ctx, const float* S, const int32_t* n_active, int cand_lo, int cand_hi,
+                              int n_sink, int32_t* sink_idx, cudaStream_t st);
+
 focus_status launch_sink_select(focus_ctx* ctx, const float* part, int H, int L, const int32_t* n_active, float* S,
                                 int cand_lo, int cand_hi, int n_sink, int32_t* sink_idx, cudaStream_t st) {
   sink_reduce_heads_kernel<<<(L + 255) / 256, 256, 0, st>>>(part, H, L, n_active, S);
   FOCUS_CHECK_LAUNCH();
+  if (n_sink == 0) return FOCUS_OK;                     // scores only
+  return launch_sink_topn(ctx, S, n_active, cand_lo, cand_hi, n_sink, sink_idx, st);
+}
+
+// Exact Top-n of given scores (n_active NULL: the scores are defined whatever produced them).
+focus_status launch_sink_topn(focus_ctx* ctx, const float* S, const int32_t* n_active, int cand_lo, int cand_hi,
+                              int n_sink, int32_t* sink_idx, cudaStream_t st) {
   const int n = cand_hi - cand_lo;
   const int chunk = (n + SC_CTAS - 1) / SC_CTAS;
   int& cluster_state = ctx->ls.select_cluster;        // 0 not tried, 1 works, 2 the cluster launch was refused once

@@ -115,6 +115,19 @@ def find_sinks(ctx, b: StepBuffers, Q, K, lse: Optional[torch.Tensor], stream=No
                         b.sink_idx, b.sink_scores, stream)
 
 
+def find_sinks_sharded(ctx, b: StepBuffers, Q, K, lse: Optional[torch.Tensor], group=None, stream=None):
+    """find_sinks for a rank that holds only its own heads of the layer (b.shape, Q, K and lse describe those heads):
+    S over the local heads, mean over the ranks of `group` (the one exchange of a step), Top-N_sink from the mean.
+    Every rank ends up with the same b.sink_idx and b.sink_scores."""
+    from . import head_shards
+    w, s = b.wl, b.wl.shape
+    act = b.row_ids if b.rows == "compact" else b.active_idx
+    fb.focus_find_sinks(ctx, b.shape, Q, b.q_base, act, b.n_active, b.max_active, K, lse, 0, 0, s.M, None,
+                        b.sink_scores, stream)
+    head_shards.mean_over_ranks(b.sink_scores, group)
+    fb.focus_select_sinks(ctx, b.sink_scores, s.L, 0, s.M, w.n_sink, b.sink_idx, stream)
+
+
 def sparse_layer(ctx, b: StepBuffers, Q, K, V, Kbar: Optional[torch.Tensor] = None, O=None, lse=None, stream=None,
                  fused: bool = True):
     """score_blocks -> select_blocks -> sparse_attn for one sparse layer (Algorithm 1, sparse branch); with cached

@@ -422,6 +422,51 @@ def test_head_dim_64_runs_on_the_tensor_core_kernels(keys, rows, merge):
         assert max_abs(got_lse[h], lh[0]) <= 2e-3
 
 
+@pytest.mark.parametrize("world", [2, 4])
+@pytest.mark.parametrize("cfg", [("bf16", 128, 128, 8, 4), ("f32", 64, 64, 8, 8)])
+def test_sinks_of_a_layer_whose_heads_are_dealt_out_to_several_ranks(ctx, cfg, world):
+    """Eq. 6 is a mean over all heads: the one step of the path that needs an exchange when the heads of a layer
+    live on several GPUs.  Here the ranks run one after the other on one GPU -- every rank computes S over its own
+    heads (focus_find_sinks with n_sink = 0), the mean over ranks stands in for the all-reduce, focus_select_sinks
+    takes the Top-N_sink -- and the result is held against the oracle over all heads (band rule), against the
+    single-device call, and against an exact selection on the averaged float32 scores themselves."""
+    from paper_2602_02159_b200 import head_shards
+    dtype, d, B, H, Hkv = cfg
+    w = small_workload(dtype, d, B, H=H, Hkv=Hkv, L=2600, M=2100, n_sink=21)
+    s = w.shape
+    host, dev = make_inputs(w)
+    b = fstep.StepBuffers(w)
+    fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
+    fstep.find_sinks(ctx, b, dev["Q"], dev["K"], None)
+    single = b.sink_idx.cpu().numpy().copy()
+    S_single = fstep.from_device(b.sink_scores).copy()
+    S_sum = torch.zeros(s.L, dtype=torch.float32, device="cuda")
+    for r in range(world):
+        qh, kvh = head_shards.local_heads(H, Hkv, r, world)
+        shape_r = fb.make_shape(s.L, s.M, H // world, Hkv // world, d, B, fb.F32 if dtype == "f32" else fb.BF16,
+                                q_stride_row=H * d, q_stride_head=d, kv_stride_tok=d, kv_stride_head=s.L * d)
+        S_r = torch.full((s.L,), 9.0, dtype=torch.float32, device="cuda")
+        fb.focus_find_sinks(ctx, shape_r, dev["Q"][:, qh], s.M, b.active_idx, b.n_active, b.max_active, dev["K"][kvh],
+                            None, 0, 0, s.M, None, S_r)
+        S_sum += S_r
+    S_mean = (S_sum * (1.0 / world)).contiguous()
+    sink = torch.full((w.n_sink,), -7, dtype=torch.int32, device="cuda")
+    fb.focus_select_sinks(ctx, S_mean, s.L, 0, s.M, w.n_sink, sink)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    got, S_got = sink.cpu().numpy(), fstep.from_device(S_mean)
+    na = int(b.n_active.item())
+    active = b.active_idx.cpu().numpy()[:na]
+    S_ora = fo.sink_scores(host["Q"][active - s.M], host["K"], 1.0 / math.sqrt(d))
+    ora = fo.find_sinks(S_ora, w.n_sink, 0, s.M)
+    assert np.max(np.abs(S_got - S_ora) / S_ora) < 2e-3                     # the bar of the single-device scores
+    assert max_abs(S_got, S_single) <= 1e-6 * float(S_ora.max())          # same scores up to the order of the head sum
+    check_topk_band(got, ora, S_ora, range(s.M), BAND, what=f"sharded sinks, {world} ranks")
+    check_topk_band(got, [int(i) for i in single if i >= 0], S_single.astype(np.float64), range(s.M), BAND,
+                    what="sharded against single device")
+    assert got.tolist() == fo.find_sinks(S_got.astype(np.float64), w.n_sink, 0, s.M).tolist(), "exact on its own scores"
+
+
 @pytest.mark.parametrize("cfg", [SHAPES[0], SHAPES[3], SHAPES[5]])
 def test_token_major_cache_and_padded_query_rows(ctx, cfg):
     """Strides are part of the shape: K/V cache stored token-major ([L, Hkv, d]: token stride Hkv*d, head stride d)
