@@ -467,6 +467,66 @@ def test_sinks_of_a_layer_whose_heads_are_dealt_out_to_several_ranks(ctx, cfg, w
     assert got.tolist() == fo.find_sinks(S_got.astype(np.float64), w.n_sink, 0, s.M).tolist(), "exact on its own scores"
 
 
+def test_a_rank_of_a_head_sharded_layer_computes_what_the_single_device_computes_for_its_heads(ctx):
+    """Two ranks, one after the other on one GPU, each with its half of the KV heads (views into the full tensors by
+    strides): dense layer, sink scores over the own heads, the mean over ranks (a sum here), Top-N_sink, sparse
+    layer.  Given the same sink set, everything else is per KV group: the rank's block lists and keep flags must be
+    exactly those of the single-device run for its groups, its attention outputs those of the single-device run for
+    its heads (to rounding: fewer heads per launch means other key splits, i.e. another summation order)."""
+    import dataclasses
+    from paper_2602_02159_b200 import head_shards
+    world = 2
+    w = small_workload("bf16", 128, 128, H=8, Hkv=4, L=2600, M=2100, n_sink=21, C=5)
+    s = w.shape
+    host, dev = make_inputs(w)
+    Kbar = torch.zeros(s.Hkv, s.nb, s.d, dtype=torch.float32, device="cuda")
+    fb.focus_pool_keys(ctx, fstep.c_shape(s), dev["K"], Kbar)
+    ranks = []
+    S_sum = torch.zeros(s.L, dtype=torch.float32, device="cuda")
+    for r in range(world):
+        qh, kvh = head_shards.local_heads(s.H, s.Hkv, r, world)
+        w_r = dataclasses.replace(w, shape=wl.Shape(s.L, s.M, s.H // world, s.Hkv // world, s.d, s.B, s.dtype))
+        b = fstep.StepBuffers(w_r)
+        b.shape = fb.make_shape(s.L, s.M, s.H // world, s.Hkv // world, s.d, s.B, fb.BF16, q_stride_row=s.H * s.d,
+                                q_stride_head=s.d, kv_stride_tok=s.d, kv_stride_head=s.L * s.d)
+        Q, K, V = dev["Q"][:, qh], dev["K"][kvh], dev["V"][kvh]
+        fstep.select_queries(ctx, b, dev["conf"], dev["masked"])
+        fstep.dense_layer(ctx, b, Q, K, V)
+        dense = b.O.clone()
+        fstep.find_sinks_sharded(ctx, b, Q, K, b.lse)          # no process group: the local scores stay in b.sink_scores
+        S_sum += b.sink_scores
+        ranks.append(dict(b=b, Q=Q, K=K, V=V, qh=qh, kvh=kvh, dense=dense))
+    S_mean = (S_sum * (1.0 / world)).contiguous()
+    for rk in ranks:                                           # what the all-reduce leaves on every rank
+        rk["b"].sink_scores.copy_(S_mean)
+        fb.focus_select_sinks(ctx, rk["b"].sink_scores, s.L, 0, s.M, w.n_sink, rk["b"].sink_idx)
+        fstep.sparse_layer(ctx, rk["b"], rk["Q"], rk["K"], rk["V"], Kbar=Kbar[rk["kvh"]].contiguous())
+    assert torch.equal(ranks[0]["b"].sink_idx, ranks[1]["b"].sink_idx)
+    # the single device, with the same sink set
+    b1 = fstep.StepBuffers(w)
+    fstep.select_queries(ctx, b1, dev["conf"], dev["masked"])
+    fstep.dense_layer(ctx, b1, dev["Q"], dev["K"], dev["V"])
+    dense1 = b1.O.clone()
+    fstep.find_sinks(ctx, b1, dev["Q"], dev["K"], b1.lse)
+    assert float((b1.sink_scores - S_mean).abs().max()) <= 1e-6 * float(S_mean.max())
+    b1.sink_idx.copy_(ranks[0]["b"].sink_idx)
+    fstep.sparse_layer(ctx, b1, dev["Q"], dev["K"], dev["V"], Kbar=Kbar)
+    torch.cuda.synchronize()
+    assert ctx.poll_status() == 0
+    na = int(b1.n_active.item())
+    per = s.Hkv // world
+    for r, rk in enumerate(ranks):
+        b = rk["b"]
+        assert torch.equal(b.active_idx, b1.active_idx) and torch.equal(b.focus_idx, b1.focus_idx)
+        assert torch.equal(b.block_cnt, b1.block_cnt[r * per:(r + 1) * per])
+        assert torch.equal(b.block_idx.view(per, -1), b1.block_idx.view(s.Hkv, -1)[r * per:(r + 1) * per])
+        assert torch.equal(b.sink_keep.view(per, -1), b1.sink_keep.view(s.Hkv, -1)[r * per:(r + 1) * per])
+        assert torch.equal(b.R.view(per, -1), b1.R.view(s.Hkv, -1)[r * per:(r + 1) * per])
+        for mine, ref in ((rk["dense"], dense1), (b.O, b1.O)):
+            a, c = fstep.from_device(mine)[:na], fstep.from_device(ref)[:na, rk["qh"]]
+            assert max_abs(a, c) <= 2e-2 and rel_rms(a, c) <= 5e-3
+
+
 @pytest.mark.parametrize("cfg", [SHAPES[0], SHAPES[3], SHAPES[5]])
 def test_token_major_cache_and_padded_query_rows(ctx, cfg):
     """Strides are part of the shape: K/V cache stored token-major ([L, Hkv, d]: token stride Hkv*d, head stride d)
