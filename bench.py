@@ -39,20 +39,66 @@ def peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed regions run.
+    """Samples SM clock, power and throttle reasons while the timed regions run: through NVML from a thread of this
+    process (a sample every 2 ms, so that a region of tens of milliseconds holds a dozen), else with nvidia-smi
+    (25 ms).  Both only read.
 
-    Every sample carries nvidia-smi's own timestamp; `window()` brackets a timed region with host wall-clock times
-    (same machine clock), and `stop()` keeps only the samples that fall inside a window, so that the median is a
-    clock under load and not one taken while the host was building a graph."""
+    Every sample carries a timestamp of the machine clock; `window()` brackets a timed region with host wall-clock
+    times, and `stop()` keeps only the samples that fall inside a window, so that the median is a clock under load
+    and not one taken while the host was building a graph."""
     Q = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
     INTERVAL_MS = 25
+    NVML_INTERVAL_MS = 2
 
     def __init__(self, index: int):
-        self.index, self.proc, self.lines, self.windows = index, None, [], []
+        self.index, self.proc, self.lines, self.windows, self.source = index, None, [], [], "nvidia-smi"
+
+    def _start_nvml(self) -> bool:
+        """One line per sample, in nvidia-smi's own CSV layout, appended to self.lines by a thread."""
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            try:                                                   # the device torch calls `index`, whatever NVML's order
+                uuid = str(torch.cuda.get_device_properties(self.index).uuid)
+                h = nv.nvmlDeviceGetHandleByUUID(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+            except Exception:
+                h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            cmax = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+        except Exception:
+            return False
+        stop = threading.Event()
+        act = lambda r, m: "Active" if r & m else "Not Active"
+
+        def loop():
+            while not stop.is_set():
+                try:
+                    ts = datetime.datetime.now()
+                    clk = nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
+                    watts = nv.nvmlDeviceGetPowerUsage(h) / 1000.0
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                    # bits: 0x4 sw power cap, 0x8 hw slowdown, 0x20 sw thermal slowdown, 0x40 hw thermal slowdown
+                    self.lines.append(f"{ts:%Y/%m/%d %H:%M:%S.%f}, {self.index}, {clk}, {cmax}, {watts:.2f}, {r:#x}, "
+                                      f"{act(r, 0x8)}, {act(r, 0x40)}, {act(r, 0x20)}, {act(r, 0x4)}\n")
+                except Exception:
+                    pass
+                stop.wait(self.NVML_INTERVAL_MS / 1000)
+
+        class _Stopper:
+            terminate = staticmethod(stop.set)
+        self.proc, self.INTERVAL_MS, self.source = _Stopper(), self.NVML_INTERVAL_MS, "nvml"
+        self.t = threading.Thread(target=loop, daemon=True)
+        self.t.start()
+        t0 = time.time()
+        while not self.lines and time.time() - t0 < 2.0:
+            time.sleep(0.005)
+        return True
 
     def start(self):
+        if self._start_nvml():
+            return
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
                                           "-i", str(self.index), "-lms", str(self.INTERVAL_MS)],
@@ -122,7 +168,7 @@ class ClockSampler:
                 "samples": len(sm), "samples_in_headline_region": len(sm_head),
                 "sm_mhz_headline_region": statistics.median(sm_head) if sm_head else None,
                 "power_w": statistics.median(watts) if watts else None,
-                "interval_ms": self.INTERVAL_MS, "reasons": sorted(reasons),
+                "interval_ms": self.INTERVAL_MS, "source": self.source, "reasons": sorted(reasons),
                 "reason_share": {n: round(c / len(sm), 3) for n, c in counts.items() if c and sm}}
         if note:
             out["note"] = note
@@ -620,7 +666,7 @@ def run_focus(args):
     if graph is not None and args.sustain_s > 0:
         n_rep = max(K, int(math.ceil(args.sustain_s * 1e3 / ms_step)))
         sus = ClockSampler(local)
-        sus.INTERVAL_MS = 25
+        sus.INTERVAL_MS, sus.NVML_INTERVAL_MS = 25, 10
         sus.start()
         a, z = ev(), ev()
         sync_all()
