@@ -143,6 +143,18 @@ __device__ __forceinline__ TileEnum make_enum(const TcParams& p, int g, int cnt_
   return e;
 }
 
+// First key tile of split s of n for a sparse key set, tiles weighed by what their softmax costs: a sink tile (one
+// mask test per column) counts 3, a block or response tile 2.  With equal tile counts the split that got the sink
+// tiles finished last and its cluster waited for it (config 2, four splits of 22 tiles: loops of 11.4 / 13.6 / 12.7 /
+// 16.4 thousand cycles).  s = 0 gives 0, s = n the tile count; monotonic in s.
+__device__ __forceinline__ int split_lo_cost(const TileEnum& e, int s, int n) {
+  const unsigned wb = 2u * (unsigned)e.n_blk, ws = 3u * (unsigned)e.n_sinkt, W = wb + ws + 2u * (unsigned)e.n_resp;
+  const unsigned x = (W * (unsigned)s + (unsigned)n - 1u) / (unsigned)n;          // ceil(W s / n)
+  if (x <= wb) return (int)((x + 1u) / 2u);
+  if (x <= wb + ws) return e.n_blk + (int)((x - wb + 2u) / 3u);
+  return e.n_blk + e.n_sinkt + (int)((x - wb - ws + 1u) / 2u);
+}
+
 __device__ __forceinline__ TileInfo tile_info(const TcParams& p, const TileEnum& e, int t) {
   TileInfo ti;
   ti.start2 = -1;
@@ -576,8 +588,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   const int cnt_raw = p.dense ? 0 : ld_ordered(p.block_cnt + g * p.group_stride);
 
   const TileEnum te = make_enum(p, g, cnt_raw);
-  const int t0 = split_lo(te.total, split, p.n_splits);
-  const int t1 = split_lo(te.total, split + 1, p.n_splits);
+  const int t0 = p.dense ? split_lo(te.total, split, p.n_splits) : split_lo_cost(te, split, p.n_splits);
+  const int t1 = p.dense ? split_lo(te.total, split + 1, p.n_splits) : split_lo_cost(te, split + 1, p.n_splits);
   const int nt = t1 - t0;
   const int cta_lin = blockIdx.x * p.n_splits + split;
 
