@@ -1,5 +1,6 @@
 // Block-sparse / dense bidirectional attention on the 5th-generation tensor cores (Eq. 9; FullAttn of
-// Algorithm 1).  bf16 inputs, head_dim 128, fp32 accumulation in TMEM.
+// Algorithm 1).  bf16 inputs, head_dim 128 (or 64: the kernels keep their 128-wide geometry and leave the upper half
+// of every operand tile out), fp32 accumulation in TMEM.
 //
 // attn_tc_kernel: one CTA = one 128-row query tile of one KV head (GQA: the rows of all query heads of the group
 // are stacked, so every K/V tile is read once per group) x one contiguous range ("split") of that head's key
