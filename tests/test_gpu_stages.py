@@ -527,6 +527,31 @@ def test_a_rank_of_a_head_sharded_layer_computes_what_the_single_device_computes
             assert max_abs(a, c) <= 2e-2 and rel_rms(a, c) <= 5e-3
 
 
+@pytest.mark.parametrize("heads", [1, 74])
+@pytest.mark.parametrize("tiles", [1, 2, 3, 4, 5, 7, 8, 10, 12, 21, 24, 26])
+def test_one_tile_kernel_with_every_short_key_loop(ctx, heads, tiles):
+    """The one-tile kernel's K/V ring has three or four slots in use depending on the key tiles per CTA (cross-over at
+    12), requests three copies at the start and the rest once the first has landed, and its P V products commit to two
+    barriers by tile parity: dense attention with key loops of 1 to 13 tiles per CTA, odd and even, a ragged last
+    tile, with one head (many splits of few tiles) and with 74 heads (two splits: tiles / 2 per CTA)."""
+    L = tiles * 128 - 37
+    n = 24
+    s = wl.Shape(L, L - n, heads, heads, 128, 128, "bf16")
+    Qs, Ks, Vs = _rand_qkv(s, 100 + tiles, qk_scale=1.5)
+    dQ, dK, dV = (fstep.to_device(x, s.dtype) for x in (Qs, Ks, Vs))
+    O = torch.zeros(n, s.H, s.d, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(s.H, n, dtype=torch.float32, device="cuda")
+    fb.focus_dense_attn(ctx, fstep.c_shape(s), dQ, s.M, n, None, None, 0, dK, dV, O, lse)
+    torch.cuda.synchronize()
+    assert ctx.last_attn_variant() == 2 and ctx.poll_status() == 0
+    got, got_lse = fstep.from_device(O), fstep.from_device(lse)
+    f64h = lambda a, h, kv=True: wl.storage_to_f64(a[h:h + 1] if kv else a[:, h:h + 1], s.dtype)
+    for h in sorted({0, heads - 1}):
+        Oh, lh = fo.dense_attn(f64h(Qs, h, False), f64h(Ks, h), f64h(Vs, h), 1.0 / math.sqrt(s.d))
+        assert max_abs(got[:, h], Oh[:, 0]) <= 2e-2 and rel_rms(got[:, h], Oh[:, 0]) <= 1e-2, (tiles, h)
+        assert max_abs(got_lse[h], lh[0]) <= 2e-3, (tiles, h)
+
+
 @pytest.mark.parametrize("cfg", [SHAPES[0], SHAPES[3], SHAPES[5]])
 def test_token_major_cache_and_padded_query_rows(ctx, cfg):
     """Strides are part of the shape: K/V cache stored token-major ([L, Hkv, d]: token stride Hkv*d, head stride d)
