@@ -1135,6 +1135,55 @@ def test_step_replayed_from_a_cuda_graph_matches_eager_calls(ctx, rows):
             assert torch.equal(getattr(b_e, name), getattr(b_g, name)), name
 
 
+@pytest.mark.parametrize("rows", ["active", "gen"])
+def test_launch_options_change_nothing_but_the_launches(rows):
+    """focus_set_option: without programmatic dependent launches (plain stream order: what a caller sets when a foreign
+    kernel produces an input immediately before a fused layer) the same kernels run the same arithmetic, so a small
+    step must come out bit for bit as by default; without the three-warpgroup kernels the one-tile kernel takes
+    their launches and the outputs agree to rounding, index sets exactly."""
+    w = small_workload("bf16", 128, 128, H=8, Hkv=2, L=2600, M=2100, n_sink=21, C=5)
+    host, dev = make_inputs(w)
+    s = w.shape
+    Kbar = torch.zeros(s.Hkv, s.nb, s.d, dtype=torch.float32, device="cuda")
+    runs = {}
+    for name, opts in (("default", []), ("no_pdl", [(fb.OPT_NO_PDL, 1)]), ("no_wide", [(fb.OPT_NO_WIDE, 1)])):
+        c = fb.Context(0)
+        try:
+            for o, v in opts:
+                assert c.set_option(o, v) == 0
+            b = fstep.StepBuffers(w, rows=rows)
+            fb.focus_pool_keys(c, b.shape, dev["K"], Kbar)
+            fstep.select_queries(c, b, dev["conf"], dev["masked"])
+            outs = []
+            for l in range(2):
+                fstep.dense_layer(c, b, dev["Q"], dev["K"], dev["V"])
+                outs.append(b.O.clone())
+            variants = [c.last_attn_variant()]
+            fstep.find_sinks(c, b, dev["Q"], dev["K"], b.lse if rows == "active" else None)
+            for l in range(3):
+                fstep.sparse_layer(c, b, dev["Q"], dev["K"], dev["V"], Kbar=Kbar)
+                outs.append(b.O.clone())
+            variants.append(c.last_attn_variant())
+            torch.cuda.synchronize()
+            assert c.poll_status() == 0
+            runs[name] = dict(outs=outs, sinks=b.sink_idx.clone(), blocks=b.block_idx.clone(), keep=b.sink_keep.clone(),
+                              lse=b.lse.clone(), variants=variants)
+        finally:
+            c.close()
+    d, p, nw = runs["default"], runs["no_pdl"], runs["no_wide"]
+    assert p["variants"] == d["variants"]
+    for a, z in zip(d["outs"], p["outs"]):
+        assert torch.equal(a.view(torch.int16), z.view(torch.int16))
+    assert torch.equal(d["lse"], p["lse"])
+    for r in (p, nw):
+        assert torch.equal(d["sinks"], r["sinks"]) and torch.equal(d["blocks"], r["blocks"]) and torch.equal(d["keep"], r["keep"])
+    assert nw["variants"] == [2, 2]
+    if rows == "gen":
+        assert d["variants"][0] in (3, 4), "the default dense layer was meant to take a three-warpgroup kernel"
+    for a, z in zip(d["outs"], nw["outs"]):
+        assert max_abs(fstep.from_device(a), fstep.from_device(z)) <= 2e-2
+
+
 def test_step_with_nothing_left_to_unmask(ctx):
     """No masked position in the decoding block: I_focus and I_active are empty.  The attention calls have no rows to
     compute (outputs stay untouched), sink identification and the fused layer report the undefined inputs through
