@@ -37,6 +37,8 @@
  *   - A device-side anomaly (index out of range, a bounded wait that ran out) never traps: the kernel
  *     skips the access, records a code in the context's device status word and returns; read it with
  *     focus_poll_status.
+ *   - Every compute entry point opens an NVTX range of its own name around its launches (host side), so a profiler
+ *     attached to the process can group kernels by stage.
  *   - There is no CPU fallback: without a CUDA device every compute entry point fails.
  */
 #ifndef FOCUS_H_

@@ -158,6 +158,7 @@ static focus_status attn_dispatch(focus_ctx* ctx, const AttnArgs& a, cudaStream_
 extern "C" focus_status focus_dense_attn(focus_ctx* ctx, const focus_shape* shape, const void* Q, int32_t q_base,
                                          int32_t n_q, const int32_t* q_rows, const int32_t* n_rows, int32_t max_rows,
                                          const void* K, const void* V, void* O, float* lse, focus_stream stream) {
+  FOCUS_STAGE("focus_dense_attn");
   AttnArgs a{};
   focus_status s = attn_common(ctx, shape, Q, q_base, n_q, q_rows, n_rows, max_rows, K, V, O, lse, a);
   if (s != FOCUS_OK) return s;
@@ -171,6 +172,7 @@ extern "C" focus_status focus_sparse_attn(focus_ctx* ctx, const focus_shape* sha
                                           int32_t max_blocks, const int32_t* block_cnt, const int32_t* sink_idx,
                                           const uint8_t* sink_keep, int32_t n_sink, void* O, float* lse,
                                           focus_stream stream) {
+  FOCUS_STAGE("focus_sparse_attn");
   AttnArgs a{};
   focus_status s = attn_common(ctx, shape, Q, q_base, n_q, q_rows, n_rows, max_rows, K, V, O, lse, a);
   if (s != FOCUS_OK) return s;
@@ -189,6 +191,7 @@ extern "C" focus_status focus_find_sinks(focus_ctx* ctx, const focus_shape* shap
                                          const int32_t* active_idx, const int32_t* n_active, int32_t max_active,
                                          const void* K, const float* lse, int32_t n_sink, int32_t cand_lo,
                                          int32_t cand_hi, int32_t* sink_idx, float* scores, focus_stream stream) {
+  FOCUS_STAGE("focus_find_sinks");
   if (!ctx || !shape_ok_basic(shape) || !Q || !active_idx || !n_active || !K) return FOCUS_ERR_INVALID_ARG;
   if (n_sink > 0 && !sink_idx) return FOCUS_ERR_INVALID_ARG;      // n_sink == 0: scores only
   if (!all_aligned16(Q, K)) return FOCUS_ERR_INVALID_ARG;
@@ -231,6 +234,7 @@ extern "C" focus_status focus_find_sinks(focus_ctx* ctx, const focus_shape* shap
 
 extern "C" focus_status focus_select_sinks(focus_ctx* ctx, const float* scores, int32_t L, int32_t cand_lo,
                                            int32_t cand_hi, int32_t n_sink, int32_t* sink_idx, focus_stream stream) {
+  FOCUS_STAGE("focus_select_sinks");
   if (!ctx || !scores || L <= 0 || n_sink < 0 || (n_sink > 0 && !sink_idx)) return FOCUS_ERR_INVALID_ARG;
   if (cand_lo < 0 || cand_hi < cand_lo || cand_hi > L) return FOCUS_ERR_INVALID_ARG;
   if (n_sink == 0) return FOCUS_OK;

@@ -3,6 +3,7 @@
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <stdint.h>
 
 #include "focus.h"
@@ -52,6 +53,17 @@ struct WsAlloc {
 // Every kernel launch of the library goes through this macro: it counts the launch and maps a failed
 // launch to FOCUS_ERR_CUDA.
 extern unsigned long long g_focus_launches;
+// One NVTX range per public compute call (host side, around the enqueue): a profiler attached to the process can
+// filter or group launches by stage (ncu: --nvtx --nvtx-include "focus_find_sinks/").  NVTX is header-only and costs a
+// call through a null hook when no tool is attached.
+struct FocusStageRange {
+  explicit FocusStageRange(const char* name) { nvtxRangePushA(name); }
+  ~FocusStageRange() { nvtxRangePop(); }
+  FocusStageRange(const FocusStageRange&) = delete;
+  FocusStageRange& operator=(const FocusStageRange&) = delete;
+};
+#define FOCUS_STAGE(name) FocusStageRange focus_stage_range_(name)
+
 #define FOCUS_CHECK_LAUNCH()                                      \
   do {                                                            \
     ++g_focus_launches;                                           \

@@ -210,6 +210,7 @@ extern "C" focus_status focus_confidence(focus_ctx* ctx, const void* logits, int
                                          int32_t vocab, int32_t pos_base, int32_t n_pos, const int32_t* rows,
                                          const int32_t* n_rows, int32_t max_rows, float* conf, int32_t* token,
                                          focus_stream stream) {
+  FOCUS_STAGE("focus_confidence");
   if (!ctx || !logits || !conf || !token || !aligned16(logits)) return FOCUS_ERR_INVALID_ARG;
   if (dtype != FOCUS_F32 && dtype != FOCUS_BF16) return FOCUS_ERR_INVALID_ARG;
   if (vocab <= 0 || row_stride < vocab || pos_base < 0 || n_pos < 0 || max_rows < 0) return FOCUS_ERR_INVALID_ARG;
@@ -246,6 +247,7 @@ extern "C" focus_status focus_confidence(focus_ctx* ctx, const void* logits, int
 extern "C" focus_status focus_update_kv(focus_ctx* ctx, const focus_shape* shape, void* K_cache, void* V_cache,
                                         const void* K_new, const void* V_new, const int32_t* rows,
                                         const int32_t* n_rows, int32_t max_rows, focus_stream stream) {
+  FOCUS_STAGE("focus_update_kv");
   if (!ctx || !shape_ok_basic(shape) || !K_cache || !V_cache || !K_new || !V_new || !rows || !n_rows)
     return FOCUS_ERR_INVALID_ARG;
   if (!all_aligned16(K_cache, V_cache, K_new, V_new)) return FOCUS_ERR_INVALID_ARG;
@@ -273,6 +275,7 @@ extern "C" focus_status focus_commit_step(focus_ctx* ctx, const float* conf_new,
                                           int32_t max_rows, int32_t L, int32_t blk_lo, int32_t blk_hi,
                                           int32_t n_unmask, float* conf, uint8_t* masked, int32_t* x,
                                           int32_t* unmasked_idx, int32_t* n_unmasked, focus_stream stream) {
+  FOCUS_STAGE("focus_commit_step");
   if (!ctx || !conf_new || !token_new || !conf || !masked || !x) return FOCUS_ERR_INVALID_ARG;
   if ((rows == nullptr) != (n_rows == nullptr)) return FOCUS_ERR_INVALID_ARG;
   if (L <= 0 || pos_base < 0 || max_rows < 0 || max_rows > CS_MAX_ROWS || n_unmask < 0 || n_unmask > CS_MAX_ROWS)

@@ -167,6 +167,7 @@ static focus_status pool_score_launch(const focus_shape* s, const void* K, float
 
 extern "C" focus_status focus_pool_keys(focus_ctx* ctx, const focus_shape* shape, const void* K, float* Kbar,
                                         focus_stream stream) {
+  FOCUS_STAGE("focus_pool_keys");
   if (!ctx || !shape_ok_basic(shape) || !K || !Kbar || !all_aligned16(K, Kbar)) return FOCUS_ERR_INVALID_ARG;
   if (!shape_supported(shape)) return FOCUS_ERR_UNSUPPORTED;
   return shape->dtype == FOCUS_BF16 ? pool_score_launch<__nv_bfloat16>(shape, K, Kbar, nullptr, nullptr, stream)
@@ -176,6 +177,7 @@ extern "C" focus_status focus_pool_keys(focus_ctx* ctx, const focus_shape* shape
 extern "C" focus_status focus_update_pooled_keys(focus_ctx* ctx, const focus_shape* shape, const void* K, float* Kbar,
                                                  const int32_t* rows, const int32_t* n_rows, int32_t max_rows,
                                                  focus_stream stream) {
+  FOCUS_STAGE("focus_update_pooled_keys");
   if (!ctx || !shape_ok_basic(shape) || !K || !Kbar || !rows || !n_rows || !all_aligned16(K, Kbar)) return FOCUS_ERR_INVALID_ARG;
   if (max_rows < 0) return FOCUS_ERR_INVALID_ARG;
   if (!shape_supported(shape)) return FOCUS_ERR_UNSUPPORTED;
@@ -203,6 +205,7 @@ extern "C" focus_status focus_score_blocks(focus_ctx* ctx, const focus_shape* sh
                                            const int32_t* focus_idx, const int32_t* n_focus, int32_t max_focus,
                                            const void* K, const float* Kbar, int32_t head_reduce, float* R,
                                            focus_stream stream) {
+  FOCUS_STAGE("focus_score_blocks");
   if (!ctx || !shape_ok_basic(shape) || !Q || !focus_idx || !n_focus || !R) return FOCUS_ERR_INVALID_ARG;
   if ((K == nullptr) == (Kbar == nullptr) || !all_aligned16(Q, K, Kbar)) return FOCUS_ERR_INVALID_ARG;
   if (max_focus <= 0 || q_base < 0 || q_base > shape->L) return FOCUS_ERR_INVALID_ARG;

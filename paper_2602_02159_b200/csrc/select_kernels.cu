@@ -106,6 +106,7 @@ extern "C" focus_status focus_select_queries(focus_ctx* ctx, const float* conf_p
                                              int32_t blk_lo, int32_t blk_hi, int32_t k, int32_t w, int32_t clip_lo,
                                              int32_t clip_hi, int32_t* focus_idx, int32_t* n_focus,
                                              int32_t* active_idx, int32_t* n_active, focus_stream stream) {
+  FOCUS_STAGE("focus_select_queries");
   if (!ctx || !conf_prev || !masked || !focus_idx || !n_focus || !active_idx || !n_active) return FOCUS_ERR_INVALID_ARG;
   if (L <= 0 || blk_lo < 0 || blk_hi < blk_lo || blk_hi > L || k < 0 || w < 0) return FOCUS_ERR_INVALID_ARG;
   if (clip_lo < 0 || clip_hi > L || clip_hi < clip_lo) return FOCUS_ERR_INVALID_ARG;
@@ -186,6 +187,7 @@ extern "C" focus_status focus_select_blocks(focus_ctx* ctx, const focus_shape* s
                                             int32_t head_reduce, int32_t C, const int32_t* sink_idx, int32_t n_sink,
                                             int32_t sink_mode, int32_t* block_idx, int32_t max_blocks,
                                             int32_t* block_cnt, uint8_t* sink_keep, focus_stream stream) {
+  FOCUS_STAGE("focus_select_blocks");
   if (!ctx || !shape_ok_basic(shape) || !R || !block_idx || !block_cnt) return FOCUS_ERR_INVALID_ARG;
   const int nb = shape_nb(shape);
   if (C < 0 || C > nb || max_blocks < C || n_sink < 0) return FOCUS_ERR_INVALID_ARG;

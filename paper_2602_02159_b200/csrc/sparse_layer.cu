@@ -203,6 +203,7 @@ extern "C" focus_status focus_sparse_layer(focus_ctx* ctx, const focus_shape* sh
                                            const int32_t* sink_idx, int32_t n_sink, float* R, int32_t* block_idx,
                                            int32_t* block_cnt, uint8_t* sink_keep, void* O, float* lse,
                                            focus_stream stream) {
+  FOCUS_STAGE("focus_sparse_layer");
   if (!ctx || !shape_ok_basic(shape) || !Q || !K || !V || !Kbar || !O || !focus_idx || !n_focus || !block_idx ||
       !block_cnt)
     return FOCUS_ERR_INVALID_ARG;
